@@ -1,0 +1,204 @@
+/*
+ * ngc.h -- C ABI of the B200 (sm_100a) hot path of Neural Garbage Collection:
+ * batched rollout decoding over a KV cache that the policy itself prunes.
+ *
+ * One eviction round is   ngc_score_evict -> ngc_sample_evict -> ngc_evict_logprob
+ * -> ngc_compact_kv,   after which generation continues with
+ * ngc_decode_attn_ragged over the surviving entries (paper Section 4.1,
+ * "grow-then-evict").
+ *
+ * Conventions
+ * -----------
+ * - Plain C.  No global state except the last CUDA error code.
+ * - Every data pointer is a DEVICE pointer owned by the caller unless the
+ *   comment says "host".  The library never allocates, frees or synchronises;
+ *   scratch comes from a caller-supplied workspace sized by
+ *   ngc_workspace_bytes().  Every call only enqueues work on `stream`
+ *   (a cudaStream_t) and returns.
+ * - Return value: NGC_OK or a negative ngc_status.  Invalid host-visible
+ *   arguments are refused before anything is launched.  Problems only visible
+ *   on the device (a budget larger than the list, a NaN logit, a corrupt kept
+ *   list, a full strip) are written to *dev_status (int32 in device memory,
+ *   first error wins, 0 = none; may be NULL) and the offending list / strip /
+ *   sequence is skipped.  Kernels never trap and every wait inside them is
+ *   bounded.
+ * - "Lists": a sequence has G eviction lists; G = 1 (one decision shared by all
+ *   layers and heads), L (one per layer, the paper's setting: Section 4.1,
+ *   "the same fraction (though not the same entries) in each of the L
+ *   layers"), or L*Hkv (one per layer and KV head).  List gi of sequence b is
+ *   row b*G + gi of every [B][G][...] array.
+ * - "Units": eviction acts on units of `block` consecutive tokens (Section 4.2,
+ *   block-level evictions); the last unit of a sequence may be short.
+ *
+ * Cache layout
+ * ------------
+ *   k, v    : [L][Hkv][R][d] elements; R rows per (layer, KV head) plane.
+ *   seq_off : int64 [B+1]; sequence b owns rows seq_off[b] .. seq_off[b+1] of
+ *             every plane (its capacity); seq_off[0] = 0, seq_off[B] = R.
+ *   lens    : int32 [B]; the first lens[b] rows of a strip are alive.
+ * A (layer, head, sequence) strip is therefore T x d contiguous rows, which
+ * decode streams linearly and compaction moves row by row.  Rows at or beyond
+ * lens[b] hold unspecified bytes.
+ */
+#ifndef NGC_H_
+#define NGC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* ngc_stream;   /* == cudaStream_t */
+
+typedef enum {
+  NGC_OK = 0,
+  NGC_ERR_INVALID_ARG = -1,   /* null pointer, negative size, inconsistent shape */
+  NGC_ERR_UNSUPPORTED = -2,   /* shape / dtype combination not built */
+  NGC_ERR_WORKSPACE = -3,     /* workspace missing or smaller than ngc_workspace_bytes() */
+  NGC_ERR_CUDA = -4           /* a CUDA call failed; code in ngc_last_cuda_error() */
+} ngc_status;
+
+/* values written to *dev_status */
+typedef enum {
+  NGC_DEV_OK = 0,
+  NGC_DEV_BAD_COUNTS = 1,     /* not 0 <= n_protect <= budget <= n <= n_max, or budget > k_max */
+  NGC_DEV_NAN_LOGIT = 2,      /* a candidate logit is NaN */
+  NGC_DEV_BAD_KEPT = 3,       /* kept list out of range, repeated or not ascending */
+  NGC_DEV_STRIP_FULL = 4,     /* append would exceed the sequence's row capacity */
+  NGC_DEV_LISTS_DISAGREE = 5, /* lists of one sequence keep different token counts */
+  NGC_DEV_TIMEOUT = 6         /* a bounded wait inside a kernel ran out */
+} ngc_dev_status;
+
+typedef enum { NGC_F32 = 0, NGC_BF16 = 1 } ngc_dtype;
+typedef enum { NGC_LISTS_SHARED = 0, NGC_LISTS_PER_LAYER = 1, NGC_LISTS_PER_LAYER_KVHEAD = 2 } ngc_lists;
+typedef enum { NGC_OP_SCORE = 0, NGC_OP_SAMPLE = 1, NGC_OP_LOGPROB = 2, NGC_OP_COMPACT = 3, NGC_OP_DECODE = 4 } ngc_op;
+
+/* Describes the cache; owns nothing.  `rows` and `max_len` are host copies the
+ * launch geometry needs: rows = seq_off[B]; max_len >= every lens[b] at the
+ * time of the call (a loose bound such as the largest capacity is fine; it
+ * only sizes grids and workspaces). */
+typedef struct {
+  void* k;
+  void* v;
+  const int64_t* seq_off;
+  int32_t* lens;
+  int64_t rows;
+  int32_t L, B, Hq, Hkv, d;   /* Hq % Hkv == 0; d in {64, 128} */
+  int32_t dtype;              /* ngc_dtype of k, v, queries and new rows */
+  int32_t max_len;
+} ngc_cache;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int ngc_version(void);
+/* Text for an ngc_status (host string, never NULL). */
+const char* ngc_strerror(int status);
+/* cudaError_t of the most recent NGC_ERR_CUDA on this host thread (0 = none). */
+int ngc_last_cuda_error(void);
+
+/* Bytes of workspace `op` needs for this cache / list shape (0 = none).  For
+ * NGC_OP_SAMPLE and NGC_OP_LOGPROB only c->B (sequences, times rounds for the
+ * log-prob) is read from the cache descriptor; pass G, n_max, k_max as in the
+ * call.  The workspace must be 256-byte aligned; its contents need not be
+ * preserved between calls, and calls sharing a workspace must be stream-ordered. */
+size_t ngc_workspace_bytes(int op, const ngc_cache* c, int G, int n_max, int k_max);
+
+/*
+ * Eviction scores -- Section 4.2 ("Parameterizing eviction actions" and
+ * "Coarsening the action space").  For every list: psi_t = mean, over the
+ * query heads feeding the list and the w most recent queries, of the softmax
+ * attention weight (scale 1/sqrt(d)) that query puts on alive key t; then
+ * s_j = mean of psi over the tokens of unit j.
+ *   q_recent [L][B][Hq][w][d], cache dtype.  Window query j sits at absolute
+ *            position lens[b]-w+j and sees keys at positions <= its own; when
+ *            lens[b] < w only the last lens[b] queries are used.
+ *   lists    which heads are averaged: SHARED = all layers and heads,
+ *            PER_LAYER = the Hq heads of the layer (the paper), PER_LAYER_KVHEAD
+ *            = the Hq/Hkv heads of one KV group.
+ *   logits   [B][G][n_max] fp32 out; units >= ceil(lens[b]/block) untouched.
+ *   log_transform  0: logit = s_j (the paper's literal reading); 1: logit = log s_j.
+ * Requires n_max >= ceil(max_len/block).  Reads K only.
+ */
+int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, int lists,
+                    int log_transform, float* logits, int n_max,
+                    void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
+
+/*
+ * Sampling the keep set -- Section 4.3 (Gumbel-top-k): perturbed key =
+ * logit + Gumbel noise; keep the budget largest.  The n_protect[b] leading
+ * units are always kept and take no part in the draw; budget[b] counts them.
+ * Noise: Philox4x32-10 with key = seed and counter = (i >> 2, list_base + b*G
+ * + gi, round low, round high); unit i takes output word i & 3; the word
+ * becomes an odd multiple of 2^-24 in (0,1) and then a Gumbel variate through a
+ * fixed sequence of correctly rounded fp32 operations, so that the draw does
+ * not depend on launch geometry, on the batch sharding or on the machine.
+ * Ties (equal fp32 keys): smaller index first.  greedy != 0 drops the noise
+ * (Section 5.1, evaluation uses deterministic top-k).
+ *   logits      [B][G][n_max] fp32
+ *   n, n_protect (may be NULL = 0), budget : int32 [B]
+ *   kept_order  [B][G][k_max] out: the budget-n_protect drawn units, largest key
+ *               first (the sequence sigma of Eq. (1)); -1 padded
+ *   kept_sorted [B][G][k_max] out: all kept units ascending; -1 padded
+ *   keep_mask   [B][G][n_max] out, 1 = kept (may be NULL)
+ * A list with bad counts or a NaN candidate logit is reported in *dev_status
+ * and gets all -1 / 0 outputs.
+ */
+int ngc_sample_evict(const float* logits, const int32_t* n, const int32_t* n_protect,
+                     const int32_t* budget, int B, int G, int n_max, int k_max,
+                     uint64_t seed, uint64_t round, uint32_t list_base, int greedy,
+                     int32_t* kept_order, int32_t* kept_sorted, uint8_t* keep_mask,
+                     void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
+
+/*
+ * Log-probability of the drawn sequence -- Eq. (1) of Section 4.3:
+ *   log p(sigma | s) = sum_j [ s_sigma_j - log sum_{t not in sigma_1..sigma_{j-1}} exp s_t ],
+ * over the non-protected units of each list, evaluated with the running
+ * remaining-mass scan the paper mentions right after the equation, in fp64.
+ * Rounds can be flattened into the leading dimension (the policy-gradient
+ * recompute of Section 4.4 evaluates all rounds of a rollout at once).
+ *   logits [n_batches][B][G][n_max] fp32; n, n_protect (NULL = 0), budget
+ *   int32 [n_batches][B]; kept_order [n_batches][B][G][k_max];
+ *   logp [n_batches][B][G] fp64 out (NaN for a list reported in *dev_status).
+ */
+int ngc_evict_logprob(const float* logits, const int32_t* n, const int32_t* n_protect,
+                      const int32_t* budget, const int32_t* kept_order,
+                      int n_batches, int B, int G, int n_max, int k_max, double* logp,
+                      void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
+
+/*
+ * Physical eviction -- Section 4.1 ("permanently evicts the rest").  In place:
+ * in every (layer, KV head, sequence) strip of K and V the tokens of the kept
+ * units move to the front in ascending original order, and lens[b] becomes
+ * the number of kept tokens.  Bit-exact row moves; rows beyond the new length
+ * are unspecified afterwards.
+ *   kept_sorted [B][G][k_max] ascending unit indices (as written by
+ *   ngc_sample_evict); budget int32 [B]; lists says how G maps to (layer, head).
+ * A strip whose list is corrupt is left untouched and reported.
+ */
+int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const int32_t* budget, int k_max,
+                   int lists, int block, int32_t* dev_status, ngc_stream stream);
+
+/*
+ * Decode attention over the surviving entries -- Section 4.1 (generation
+ * continues "conditioned on the surviving entries").  For layers
+ * [layer_begin, layer_end): if new_k/new_v are given, the new token's K/V row
+ * is first written at position lens[b] of each strip and is visible to its
+ * own query; then out = softmax(scale * q K^T) V over the alive rows, one
+ * pass, split along tokens.  lens[b] is incremented (once) by the call whose
+ * layer_end == L when new rows were given.
+ *   q      [L][B][Hq][d] cache dtype; new_k, new_v [L][B][Hkv][d] cache dtype or both NULL
+ *   out    [L][B][Hq][d] of out_dtype (NGC_F32, or NGC_BF16 for a bf16 cache);
+ *          only the layers of the range are written; an empty strip gives zeros.
+ * bf16 caches: fp32 scores, softmax and accumulation; the probabilities are
+ * rounded to bf16 for the P*V product.
+ */
+int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* new_k, const void* new_v,
+                           int layer_begin, int layer_end, float scale,
+                           void* out, int out_dtype,
+                           void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NGC_H_ */

@@ -1,0 +1,217 @@
+"""Thin Python binding of the C-ABI CUDA library (``include/ngc.h``).
+
+Argument marshalling only: torch tensors provide device memory and the current
+CUDA stream, every step of the path runs inside the library's kernels.  There
+is no CPU fallback: importing this module without the built library raises,
+and so does every call made without a CUDA device.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libngc_b200.so")
+
+F32, BF16 = 0, 1
+LISTS_SHARED, LISTS_PER_LAYER, LISTS_PER_LAYER_KVHEAD = 0, 1, 2
+OP_SCORE, OP_SAMPLE, OP_LOGPROB, OP_COMPACT, OP_DECODE = range(5)
+
+DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "strip full",
+              5: "lists disagree", 6: "timeout"}
+
+EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_score_evict",
+           "ngc_sample_evict", "ngc_evict_logprob", "ngc_compact_kv", "ngc_decode_attn_ragged"]
+
+
+class NgcError(RuntimeError):
+    pass
+
+
+class CacheDesc(C.Structure):
+    """Mirror of ``ngc_cache``."""
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("seq_off", C.c_void_p), ("lens", C.c_void_p),
+                ("rows", C.c_int64), ("L", C.c_int32), ("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
+                ("d", C.c_int32), ("dtype", C.c_int32), ("max_len", C.c_int32)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2604_18002_b200.build` "
+            "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, u32, u64, sz = C.c_void_p, C.c_int, C.c_uint32, C.c_uint64, C.c_size_t
+    lib.ngc_version.restype = i32
+    lib.ngc_strerror.restype = C.c_char_p
+    lib.ngc_strerror.argtypes = [i32]
+    lib.ngc_last_cuda_error.restype = i32
+    lib.ngc_workspace_bytes.restype = sz
+    lib.ngc_workspace_bytes.argtypes = [i32, C.POINTER(CacheDesc), i32, i32, i32]
+    lib.ngc_score_evict.restype = i32
+    lib.ngc_score_evict.argtypes = [C.POINTER(CacheDesc), vp, i32, i32, i32, i32, vp, i32, vp, sz, vp, vp]
+    lib.ngc_sample_evict.restype = i32
+    lib.ngc_sample_evict.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, u64, u64, u32, i32, vp, vp, vp, vp, sz, vp, vp]
+    lib.ngc_evict_logprob.restype = i32
+    lib.ngc_evict_logprob.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp, vp]
+    lib.ngc_compact_kv.restype = i32
+    lib.ngc_compact_kv.argtypes = [C.POINTER(CacheDesc), vp, vp, i32, i32, i32, vp, vp]
+    lib.ngc_decode_attn_ragged.restype = i32
+    lib.ngc_decode_attn_ragged.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, sz, vp, vp]
+    return lib
+
+
+lib = _load()
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        msg = lib.ngc_strerror(rc).decode()
+        if rc == -4:
+            msg += f" (cudaError {lib.ngc_last_cuda_error()})"
+        raise NgcError(f"{what}: {msg}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise NgcError("device tensors required: the library has no CPU path")
+    if not t.is_contiguous():
+        raise NgcError("contiguous tensors required")
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise NgcError(f"unsupported cache dtype {t.dtype}")
+
+
+def lists_G(lists: int, L: int, Hkv: int) -> int:
+    return 1 if lists == LISTS_SHARED else (L if lists == LISTS_PER_LAYER else L * Hkv)
+
+
+@dataclass
+class NgcCache:
+    """Device K/V cache plus the host-side numbers the launches need."""
+    k: torch.Tensor        # [L][Hkv][R][d]
+    v: torch.Tensor
+    seq_off: torch.Tensor  # int64 [B+1], device
+    lens: torch.Tensor     # int32 [B], device
+    Hq: int
+    max_len: int           # host bound on lens (any value >= max(lens) at call time)
+
+    def desc(self, extra_len: int = 0) -> CacheDesc:
+        L, Hkv, R, d = self.k.shape
+        return CacheDesc(_ptr(self.k), _ptr(self.v), _ptr(self.seq_off), _ptr(self.lens), R, L,
+                         self.lens.shape[0], self.Hq, Hkv, d, _dtype_code(self.k), self.max_len + extra_len)
+
+    @property
+    def L(self):
+        return self.k.shape[0]
+
+    @property
+    def B(self):
+        return self.lens.shape[0]
+
+    @property
+    def Hkv(self):
+        return self.k.shape[1]
+
+    @property
+    def d(self):
+        return self.k.shape[3]
+
+
+def version() -> int:
+    return lib.ngc_version()
+
+
+def workspace_bytes(op: int, cache: Optional[NgcCache] = None, G: int = 1, n_max: int = 0, k_max: int = 0,
+                    B: Optional[int] = None) -> int:
+    if cache is not None:
+        d = cache.desc(1)
+    else:
+        d = CacheDesc(None, None, None, None, 0, 1, B or 1, 1, 1, 128, BF16, 0)
+    return int(lib.ngc_workspace_bytes(op, C.byref(d), G, n_max, k_max))
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> Optional[torch.Tensor]:
+    if nbytes == 0:
+        return None
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
+def new_status(device="cuda") -> torch.Tensor:
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def ngc_score_evict(cache: NgcCache, q_recent: torch.Tensor, block: int, lists: int, logits: torch.Tensor,
+                    log_transform: int = 0, ws: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
+    """q_recent [L][B][Hq][w][d] -> logits [B][G][n_max] fp32 (in place)."""
+    w = q_recent.shape[3]
+    n_max = logits.shape[2]
+    d = cache.desc()
+    rc = lib.ngc_score_evict(C.byref(d), _ptr(q_recent), w, block, lists, log_transform, _ptr(logits), n_max,
+                             _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
+    _check(rc, "ngc_score_evict")
+
+
+def ngc_sample_evict(logits: torch.Tensor, n: torch.Tensor, n_protect: Optional[torch.Tensor], budget: torch.Tensor,
+                     seed: int, rnd: int, kept_order: torch.Tensor, kept_sorted: torch.Tensor,
+                     keep_mask: Optional[torch.Tensor] = None, greedy: int = 0, list_base: int = 0,
+                     ws: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
+    B, G, n_max = logits.shape
+    k_max = kept_order.shape[2]
+    rc = lib.ngc_sample_evict(_ptr(logits), _ptr(n), _ptr(n_protect), _ptr(budget), B, G, n_max, k_max,
+                              seed, rnd, list_base, greedy, _ptr(kept_order), _ptr(kept_sorted), _ptr(keep_mask),
+                              _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
+    _check(rc, "ngc_sample_evict")
+
+
+def ngc_evict_logprob(logits: torch.Tensor, n: torch.Tensor, n_protect: Optional[torch.Tensor], budget: torch.Tensor,
+                      kept_order: torch.Tensor, logp: torch.Tensor, status: Optional[torch.Tensor] = None):
+    """logits [NB][B][G][n_max] (or [B][G][n_max]); logp fp64 [NB][B][G]."""
+    if logits.dim() == 3:
+        NB = 1
+        B, G, n_max = logits.shape
+    else:
+        NB, B, G, n_max = logits.shape
+    k_max = kept_order.shape[-1]
+    rc = lib.ngc_evict_logprob(_ptr(logits), _ptr(n), _ptr(n_protect), _ptr(budget), _ptr(kept_order),
+                               NB, B, G, n_max, k_max, _ptr(logp), None, 0, _ptr(status), _stream())
+    _check(rc, "ngc_evict_logprob")
+
+
+def ngc_compact_kv(cache: NgcCache, kept_sorted: torch.Tensor, budget: torch.Tensor, lists: int, block: int = 1,
+                   status: Optional[torch.Tensor] = None):
+    d = cache.desc()
+    rc = lib.ngc_compact_kv(C.byref(d), _ptr(kept_sorted), _ptr(budget), kept_sorted.shape[2], lists, block,
+                            _ptr(status), _stream())
+    _check(rc, "ngc_compact_kv")
+
+
+def ngc_decode_attn_ragged(cache: NgcCache, q: torch.Tensor, out: torch.Tensor, new_k: Optional[torch.Tensor] = None,
+                           new_v: Optional[torch.Tensor] = None, layer_begin: int = 0, layer_end: Optional[int] = None,
+                           scale: Optional[float] = None, ws: Optional[torch.Tensor] = None,
+                           status: Optional[torch.Tensor] = None):
+    if layer_end is None:
+        layer_end = cache.L
+    if scale is None:
+        scale = 1.0 / (cache.d ** 0.5)
+    d = cache.desc(1 if new_k is not None else 0)
+    rc = lib.ngc_decode_attn_ragged(C.byref(d), _ptr(q), _ptr(new_k), _ptr(new_v), layer_begin, layer_end,
+                                    scale, _ptr(out), _dtype_code(out), _ptr(ws), 0 if ws is None else ws.numel(),
+                                    _ptr(status), _stream())
+    _check(rc, "ngc_decode_attn_ragged")

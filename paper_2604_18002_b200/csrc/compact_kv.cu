@@ -1,0 +1,172 @@
+// ngc_compact_kv: physical eviction (paper Section 4.1), in place.
+//
+// One CTA owns one (layer, KV head, sequence, K-or-V) strip and walks its
+// OUTPUT rows in ascending tiles.  Kept units are strictly ascending, so the
+// source of output token j is never in front of j: tile i reads rows >= i*T
+// only, tile i writes rows [i*T, (i+1)*T).  Hence loads may run ahead of stores
+// without ever seeing a moved row, as long as every load of tile i is done
+// before the first store of tile i (one __syncthreads per tile).  The leading
+// run of tokens that already sit in place is skipped.  HBM-bound: 16-byte
+// vector loads/stores, several CTAs per SM, next tile prefetched into
+// registers before the current one is stored.
+#include "ngc_common.cuh"
+
+namespace ngc {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kVecPerThread = 4;   // 16-byte vectors per thread per tile
+
+struct CompactParams {
+  uint4* k;
+  uint4* v;
+  const int64_t* seq_off;
+  const int32_t* lens;
+  const int32_t* kept_sorted;
+  const int32_t* budget;
+  int32_t* dev_status;
+  int64_t plane_vecs;   // R * row_vecs
+  int L, B, Hkv, G, lists, block, k_max;
+  int row_vecs;         // 16-byte vectors per row
+};
+
+// Validates one kept list with the whole CTA.  Returns (to every thread) the
+// number of kept tokens, or -1 if the list is corrupt.  *first_moved gets the
+// first output token whose source differs from its destination.
+__device__ int validate_list(const int32_t* kept, int K, int k_max, int len, int block, int* first_moved) {
+  __shared__ int s_bad, s_first;
+  if (threadIdx.x == 0) { s_bad = 0; s_first = 0x7fffffff; }
+  __syncthreads();
+  const int n_units = (len + block - 1) / block;
+  int bad = (K < 0 || K > k_max || K > n_units) ? 1 : 0;
+  int first = 0x7fffffff;
+  if (!bad) {
+    for (int j = threadIdx.x; j < K; j += blockDim.x) {
+      int u = kept[j];
+      int prev = j > 0 ? kept[j - 1] : -1;
+      if (u <= prev || u >= n_units) bad = 1;
+      if (u != j && j < first) first = j;
+    }
+  }
+  if (bad) atomicOr(&s_bad, 1);
+  if (first != 0x7fffffff) atomicMin(&s_first, first);
+  __syncthreads();
+  bad = s_bad;
+  first = s_first;
+  __syncthreads();
+  if (bad) return -1;
+  int tokens = K * block;
+  if (K > 0 && kept[K - 1] == n_units - 1) tokens -= n_units * block - len;   // short last unit
+  *first_moved = first == 0x7fffffff ? tokens : first * block;
+  return tokens;
+}
+
+__global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
+  int s = blockIdx.x;
+  const int kv = s & 1; s >>= 1;
+  const int b = s % p.B; s /= p.B;
+  const int h = s % p.Hkv;
+  const int l = s / p.Hkv;
+  const int gi = list_of(p.lists, l, h, p.Hkv);
+  const int len = p.lens[b];
+  const int K = p.budget[b];
+  const int32_t* kept = p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max;
+
+  int first_moved = 0;
+  const int tokens = validate_list(kept, K, p.k_max, len, p.block, &first_moved);
+  if (tokens < 0) {
+    if (threadIdx.x == 0) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
+    return;
+  }
+  uint4* strip = (kv ? p.v : p.k) + (int64_t)(l * p.Hkv + h) * p.plane_vecs + p.seq_off[b] * p.row_vecs;
+
+  const int rv = p.row_vecs;
+  const int tile_rows = kThreads * kVecPerThread / rv;
+  const int block = p.block;
+  uint4 cur[kVecPerThread], nxt[kVecPerThread];
+
+  auto load_tile = [&](int t0, uint4 (&r)[kVecPerThread]) {
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) {
+      int slot = u * kThreads + threadIdx.x;
+      int jt = t0 + slot / rv;
+      if (jt < tokens) {
+        int unit = jt / block;
+        int src = kept[unit] * block + (jt - unit * block);
+        r[u] = __ldcs(strip + (int64_t)src * rv + slot % rv);
+      }
+    }
+  };
+  auto store_tile = [&](int t0, const uint4 (&r)[kVecPerThread]) {
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) {
+      int slot = u * kThreads + threadIdx.x;
+      int jt = t0 + slot / rv;
+      if (jt < tokens) strip[(int64_t)jt * rv + slot % rv] = r[u];
+    }
+  };
+
+  int t0 = first_moved;
+  if (t0 >= tokens) return;
+  load_tile(t0, cur);
+  for (; t0 < tokens; t0 += tile_rows) {
+    if (t0 + tile_rows < tokens) load_tile(t0 + tile_rows, nxt);
+    __syncthreads();            // every load of this tile has completed
+    store_tile(t0, cur);
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) cur[u] = nxt[u];
+  }
+}
+
+// After all strips moved: lens[b] <- kept token count (one CTA per sequence,
+// every list of the sequence re-validated; they must agree).
+__global__ void __launch_bounds__(kThreads) compact_lens_kernel(CompactParams p) {
+  const int b = blockIdx.x;
+  const int len = p.lens[b];
+  const int K = p.budget[b];
+  int tokens0 = -1;
+  bool ok = true;
+  for (int gi = 0; gi < p.G; ++gi) {
+    int fm;
+    int t = validate_list(p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max, K, p.k_max, len, p.block, &fm);
+    if (t < 0) { ok = false; break; }            // already reported by the strip kernel
+    if (tokens0 < 0) tokens0 = t;
+    else if (t != tokens0) {
+      ok = false;
+      if (threadIdx.x == 0) set_dev_status(p.dev_status, NGC_DEV_LISTS_DISAGREE);
+      break;
+    }
+  }
+  if (ok && threadIdx.x == 0) const_cast<int32_t*>(p.lens)[b] = tokens0;
+}
+
+}  // namespace
+}  // namespace ngc
+
+extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const int32_t* budget, int k_max,
+                              int lists, int block, int32_t* dev_status, ngc_stream stream) {
+  using namespace ngc;
+  if (!valid_cache(c) || !kept_sorted || !budget || k_max <= 0 || block <= 0 || lists < 0 || lists > 2)
+    return NGC_ERR_INVALID_ARG;
+  const int row_bytes = c->d * elt_bytes(c->dtype);
+  CompactParams p;
+  p.k = (uint4*)c->k;
+  p.v = (uint4*)c->v;
+  p.seq_off = c->seq_off;
+  p.lens = c->lens;
+  p.kept_sorted = kept_sorted;
+  p.budget = budget;
+  p.dev_status = dev_status;
+  p.row_vecs = row_bytes / 16;
+  p.plane_vecs = c->rows * p.row_vecs;
+  p.L = c->L; p.B = c->B; p.Hkv = c->Hkv;
+  p.G = lists_G(lists, c->L, c->Hkv);
+  p.lists = lists; p.block = block; p.k_max = k_max;
+  const int64_t strips = (int64_t)c->L * c->Hkv * c->B * 2;
+  if (strips > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+  compact_kernel<<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
+  int rc = launch_status();
+  if (rc != NGC_OK) return rc;
+  compact_lens_kernel<<<c->B, kThreads, 0, (cudaStream_t)stream>>>(p);
+  return launch_status();
+}

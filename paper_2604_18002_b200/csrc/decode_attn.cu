@@ -1,0 +1,603 @@
+// ngc_decode_attn_ragged: decode attention over the surviving cache entries
+// (paper Section 4.1: generation continues conditioned on the pruned cache).
+//
+// Work item = (layer, sequence, KV head, token split).  Two device paths:
+//
+//  * bf16, d = 128, group size Hq/Hkv <= 16 (the GQA shapes): HBM-bound
+//    streaming kernel.  A producer warp feeds a ring of shared-memory stages
+//    with TMA tensor loads (64 tokens x 128 channels of K and of V per stage,
+//    128-byte swizzle, completion on mbarriers).  Four consumer warps each own
+//    16 tokens of a stage: S = Q K^T and O += P V run on the tensor cores
+//    (mma.sync m16n8k16, the group's query heads on the M axis, so the g heads
+//    that share a K/V row reuse it straight from shared memory), with a
+//    single-pass online softmax in fp32.  Per-warp partial states are merged
+//    through shared memory at the end of the item.
+//  * everything else (fp32 caches, d = 64, large groups): one query head per
+//    CTA, a warp per token row, fp32 FMA and warp-shuffle reductions.
+//
+// With n_split > 1 each item writes an unnormalised partial (m, l, o) and a
+// small combine kernel merges the splits.  The new token's K/V row is written
+// by a tiny kernel in front (same call, same stream); lens[] is bumped by a
+// kernel behind.  No kernel here ever waits on another CTA.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <mutex>
+
+#include "ngc_common.cuh"
+#include "ngc_plan.h"
+#include "ptx.cuh"
+
+namespace ngc {
+namespace {
+
+struct DecodeParams {
+  void* k;
+  void* v;
+  const int64_t* seq_off;
+  int32_t* lens;
+  const void* q;
+  const void* new_k;
+  const void* new_v;
+  void* out;
+  float* part_o;      // [items][n_split][d]
+  float2* part_ml;    // [items][n_split]  (m in log2 units, l)
+  int32_t* dev_status;
+  int64_t rows;
+  int L, B, Hq, Hkv, d, g;
+  int layer_begin, n_layers, n_split, append, out_bf16;
+  float scale_log2;   // scale * log2(e)
+};
+
+// Visible length of sequence b for this call; -1 if the appended row does not fit.
+__device__ __forceinline__ int visible_len(const DecodeParams& p, int b) {
+  const int len = p.lens[b];
+  if (!p.append) return len;
+  const int64_t cap = p.seq_off[b + 1] - p.seq_off[b];
+  return (len + 1 > cap) ? -1 : len + 1;
+}
+
+// ---------------------------------------------------------------- append
+
+__global__ void append_kernel(DecodeParams p, int row_vecs) {
+  int s = blockIdx.x;
+  const int h = s % p.Hkv; s /= p.Hkv;
+  const int b = s % p.B;
+  const int l = p.layer_begin + s / p.B;
+  const int len = p.lens[b];
+  const int64_t cap = p.seq_off[b + 1] - p.seq_off[b];
+  if (len + 1 > cap) {
+    if (threadIdx.x == 0) set_dev_status(p.dev_status, NGC_DEV_STRIP_FULL);
+    return;
+  }
+  const int t = threadIdx.x;
+  const int which = t >> 5, vec = t & 31;
+  if (vec >= row_vecs) return;
+  const uint4* src = (const uint4*)(which ? p.new_v : p.new_k) + (((int64_t)l * p.B + b) * p.Hkv + h) * row_vecs;
+  uint4* dst = (uint4*)(which ? p.v : p.k) + (((int64_t)(l * p.Hkv + h) * p.rows) + p.seq_off[b] + len) * row_vecs;
+  dst[vec] = src[vec];
+}
+
+__global__ void bump_lens_kernel(DecodeParams p) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= p.B) return;
+  const int len = p.lens[b];
+  const int64_t cap = p.seq_off[b + 1] - p.seq_off[b];
+  if (len + 1 <= cap) p.lens[b] = len + 1;
+}
+
+// ---------------------------------------------------------------- output helpers
+
+__device__ __forceinline__ void store_out(const DecodeParams& p, int64_t idx, float v) {
+  if (p.out_bf16) ((__nv_bfloat16*)p.out)[idx] = __float2bfloat16(v);
+  else ((float*)p.out)[idx] = v;
+}
+
+// ---------------------------------------------------------------- generic path
+
+template <typename T> struct RowLoad;
+template <> struct RowLoad<float> {
+  template <int VPL> static __device__ __forceinline__ void load(const float* row, int lane, float (&x)[VPL]) {
+    if constexpr (VPL == 2) {
+      const float2 t = ((const float2*)row)[lane];
+      x[0] = t.x; x[1] = t.y;
+    } else {
+      const float4 t = ((const float4*)row)[lane];
+      x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+    }
+  }
+};
+template <> struct RowLoad<__nv_bfloat16> {
+  template <int VPL> static __device__ __forceinline__ void load(const __nv_bfloat16* row, int lane, float (&x)[VPL]) {
+    if constexpr (VPL == 2) {
+      const __nv_bfloat162 t = ((const __nv_bfloat162*)row)[lane];
+      x[0] = __low2float(t); x[1] = __high2float(t);
+    } else {
+      const uint2 t = ((const uint2*)row)[lane];
+      const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+      const __nv_bfloat162 c = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+      x[0] = __low2float(a); x[1] = __high2float(a); x[2] = __low2float(c); x[3] = __high2float(c);
+    }
+  }
+};
+
+constexpr int kGenWarps = 4;
+constexpr int kGenChunk = 64;   // split granularity in tokens (same as the streaming path)
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kGenWarps * 32) decode_generic_kernel(DecodeParams p) {
+  constexpr int VPL = D / 32;
+  __shared__ float sm_m[kGenWarps], sm_l[kGenWarps];
+  __shared__ float sm_acc[kGenWarps][D];
+
+  int item = blockIdx.x;
+  const int split = item % p.n_split; item /= p.n_split;
+  const int hq = item % p.Hq;
+  const int b = (item / p.Hq) % p.B;
+  const int lr = item / (p.Hq * p.B);
+  const int l = p.layer_begin + lr;
+  const int h = hq / p.g;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  int len = visible_len(p, b);
+  if (len < 0) len = 0;
+  const int nt = (len + kGenChunk - 1) / kGenChunk;
+  const int tps = (nt + p.n_split - 1) / p.n_split;
+  const int t_begin = min(len, split * tps * kGenChunk);
+  const int t_end = min(len, (split + 1) * tps * kGenChunk);
+
+  const int64_t qo = (((int64_t)l * p.B + b) * p.Hq + hq) * D;
+  float qv[VPL];
+  RowLoad<T>::template load<VPL>((const T*)p.q + qo, lane, qv);
+  const T* kbase = (const T*)p.k + ((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b]) * D;
+  const T* vbase = (const T*)p.v + ((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b]) * D;
+
+  float m = -INFINITY, lsum = 0.f, acc[VPL];
+#pragma unroll
+  for (int i = 0; i < VPL; ++i) acc[i] = 0.f;
+  for (int t = t_begin + warp; t < t_end; t += kGenWarps) {
+    float kx[VPL], vx[VPL];
+    RowLoad<T>::template load<VPL>(kbase + (int64_t)t * D, lane, kx);
+    RowLoad<T>::template load<VPL>(vbase + (int64_t)t * D, lane, vx);
+    float dot = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) dot = fmaf(qv[i], kx[i], dot);
+    dot = warp_sum(dot);
+    const float z = dot * p.scale_log2;
+    const float m_new = fmaxf(m, z);
+    const float alpha = exp2f(m - m_new);
+    const float pz = exp2f(z - m_new);
+    lsum = lsum * alpha + pz;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) acc[i] = fmaf(pz, vx[i], acc[i] * alpha);
+    m = m_new;
+  }
+  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = lsum; }
+#pragma unroll
+  for (int i = 0; i < VPL; ++i) sm_acc[warp][lane * VPL + i] = acc[i];
+  __syncthreads();
+  if (tid < D) {
+    float mg = sm_m[0];
+#pragma unroll
+    for (int w = 1; w < kGenWarps; ++w) mg = fmaxf(mg, sm_m[w]);
+    float o = 0.f, ls = 0.f;
+#pragma unroll
+    for (int w = 0; w < kGenWarps; ++w) {
+      const float f = sm_m[w] == -INFINITY ? 0.f : exp2f(sm_m[w] - mg);
+      o = fmaf(sm_acc[w][tid], f, o);
+      ls = fmaf(sm_l[w], f, ls);
+    }
+    const int64_t it = ((int64_t)lr * p.B + b) * p.Hq + hq;
+    if (p.n_split == 1) {
+      store_out(p, qo + tid, ls > 0.f ? o / ls : 0.f);
+    } else {
+      p.part_o[(it * p.n_split + split) * D + tid] = o;
+      if (tid == 0) p.part_ml[it * p.n_split + split] = make_float2(mg, ls);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- split combine
+
+__global__ void combine_kernel(DecodeParams p) {
+  const int64_t it = blockIdx.x;               // (lr, b, hq)
+  const int c = threadIdx.x;                   // channel
+  const int lr = (int)(it / ((int64_t)p.B * p.Hq));
+  const int64_t rest = it - (int64_t)lr * p.B * p.Hq;
+  const int64_t qo = (((int64_t)(p.layer_begin + lr) * p.B) * p.Hq + rest) * p.d;
+  float mg = -INFINITY;
+  for (int s = 0; s < p.n_split; ++s) mg = fmaxf(mg, p.part_ml[it * p.n_split + s].x);
+  float o = 0.f, ls = 0.f;
+  for (int s = 0; s < p.n_split; ++s) {
+    const float2 ml = p.part_ml[it * p.n_split + s];
+    const float f = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mg);
+    o = fmaf(p.part_o[(it * p.n_split + s) * p.d + c], f, o);
+    ls = fmaf(ml.y, f, ls);
+  }
+  store_out(p, qo + c, ls > 0.f ? o / ls : 0.f);
+}
+
+// ---------------------------------------------------------------- streaming bf16 path
+
+constexpr int kTileT = 64;                    // tokens per stage
+constexpr int kConsumerWarps = 4;
+constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
+constexpr int kBoxBytes = kTileT * 128;       // one 64 x 64 bf16 box
+constexpr int kTileBytes = 2 * kBoxBytes;     // K (or V) tile: two boxes (channels 0-63, 64-127)
+constexpr int kStageBytes = 2 * kTileBytes;   // K + V
+constexpr int kStages = 3;
+constexpr int kORowStride = 132;              // floats; merge buffer row stride (bank spread)
+
+__global__ void __launch_bounds__(kStreamThreads, 2)
+decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, DecodeParams p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ uint64_t bar_full[kStages], bar_empty[kStages];
+  __shared__ float sm_m[kConsumerWarps][16], sm_l[kConsumerWarps][16];
+
+  uint8_t* stage_base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+
+  int item = blockIdx.x;
+  const int split = item % p.n_split; item /= p.n_split;
+  const int h = item % p.Hkv;
+  const int b = (item / p.Hkv) % p.B;
+  const int lr = item / (p.Hkv * p.B);
+  const int l = p.layer_begin + lr;
+  const int g = p.g;
+
+  int len = visible_len(p, b);
+  if (len < 0) len = 0;
+  const int nt = (len + kTileT - 1) / kTileT;
+  const int tps = (nt + p.n_split - 1) / p.n_split;
+  const int tile_lo = min(nt, split * tps);
+  const int tile_hi = min(nt, tile_lo + tps);
+  const int n_tiles = tile_hi - tile_lo;
+
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&bar_full[s], 1); ptx::mbar_init(&bar_empty[s], kConsumerWarps); }
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+
+  float o_acc[16][4];
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+#pragma unroll
+  for (int i = 0; i < 16; ++i) { o_acc[i][0] = 0.f; o_acc[i][1] = 0.f; o_acc[i][2] = 0.f; o_acc[i][3] = 0.f; }
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------ producer
+    if (lane == 0 && n_tiles > 0) {
+      ptx::prefetch_tensormap(&map_k);
+      ptx::prefetch_tensormap(&map_v);
+      const int plane = l * p.Hkv + h;
+      const int row0 = (int)p.seq_off[b];
+      for (int it = 0; it < n_tiles; ++it) {
+        const int s = it % kStages;
+        if (it >= kStages) {
+          if (!ptx::mbar_wait_bounded(&bar_empty[s], ((it / kStages) - 1) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
+        }
+        uint8_t* st = stage_base + s * kStageBytes;
+        ptx::mbar_expect_tx(&bar_full[s], kStageBytes);
+        const int y = row0 + (tile_lo + it) * kTileT;
+        ptx::tma_load_3d(st, &map_k, 0, y, plane, &bar_full[s]);
+        ptx::tma_load_3d(st + kBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
+        ptx::tma_load_3d(st + kTileBytes, &map_v, 0, y, plane, &bar_full[s]);
+        ptx::tma_load_3d(st + kTileBytes + kBoxBytes, &map_v, 64, y, plane, &bar_full[s]);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------ consumers
+    // Q fragments (A operand): rows = heads of the group (gid, gid+8), zero beyond g.
+    uint32_t qa[8][4];
+    {
+      const uint32_t* q0 = (const uint32_t*)((const __nv_bfloat16*)p.q + (((int64_t)l * p.B + b) * p.Hq + h * g + gid) * 128);
+      const uint32_t* q1 = q0 + 8 * 64;   // 8 heads further (128 bf16 = 64 words per head)
+      const bool v0 = gid < g, v1 = gid + 8 < g;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const int w0 = (16 * ks + 2 * tig) >> 1;
+        qa[ks][0] = v0 ? q0[w0] : 0u;
+        qa[ks][1] = v1 ? q1[w0] : 0u;
+        qa[ks][2] = v0 ? q0[w0 + 4] : 0u;
+        qa[ks][3] = v1 ? q1[w0 + 4] : 0u;
+      }
+    }
+    // lane-dependent parts of the swizzled shared-memory addresses
+    const uint32_t k_lane_off = (uint32_t)((16 * warp + (lane & 7)) * 128);
+    const uint32_t v_lane_off = (uint32_t)((16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * 128);
+    const uint32_t x7 = (uint32_t)(lane & 7);
+
+    for (int it = 0; it < n_tiles; ++it) {
+      const int s = it % kStages;
+      if (!ptx::mbar_wait_bounded(&bar_full[s], (it / kStages) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
+      uint8_t* st = stage_base + s * kStageBytes;
+      const uint32_t k_st = ptx::smem_u32(st);
+      const uint32_t v_st = k_st + kTileBytes;
+      const int tile_t0 = (tile_lo + it) * kTileT;
+      const int valid = len - tile_t0 - 16 * warp;      // live tokens in this warp's slice (may exceed 16)
+
+      if (valid > 0) {
+        if (valid < 16) {
+          // dead V rows may hold anything (NaN x 0 would poison the sum): zero them
+          for (int i = lane; i < 16 * 16; i += 32) {
+            const int r = i >> 4, c = i & 15;
+            if (r >= valid) {
+              uint8_t* rowp = st + kTileBytes + (c >> 3) * kBoxBytes + (16 * warp + r) * 128 + (c & 7) * 16;
+              *reinterpret_cast<uint4*>(rowp) = make_uint4(0, 0, 0, 0);
+            }
+          }
+          __syncwarp();
+        }
+        // ---- S = Q K^T for 16 tokens (two n-tiles of 8) ----
+        float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int n8 = 0; n8 < 2; ++n8) {
+            const uint32_t chunk = (uint32_t)(4 * (j & 1) + (lane >> 3));
+            const uint32_t addr = k_st + (j >> 1) * kBoxBytes + k_lane_off + n8 * (8 * 128) + ((chunk ^ x7) << 4);
+            uint32_t r0, r1, r2, r3;
+            ptx::ldmatrix_x4(addr, r0, r1, r2, r3);
+            ptx::mma_bf16_16816(sc[n8], qa[2 * j], r0, r1);
+            ptx::mma_bf16_16816(sc[n8], qa[2 * j + 1], r2, r3);
+          }
+        }
+        // ---- online softmax (log2 domain) ----
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int n8 = 0; n8 < 2; ++n8) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int tok = 8 * n8 + 2 * tig + (e & 1);
+            const float z = tok < valid ? sc[n8][e] * p.scale_log2 : -INFINITY;
+            sc[n8][e] = z;
+            mx[e >> 1] = fmaxf(mx[e >> 1], z);
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+        }
+        float m_new[2], alpha[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          m_new[r] = fmaxf(m_run[r], mx[r]);          // finite: token 0 of the slice is live
+          alpha[r] = ptx::ex2_approx(m_run[r] - m_new[r]);
+        }
+        const bool changed = (m_new[0] != m_run[0]) || (m_new[1] != m_run[1]);
+        if (__any_sync(0xffffffffu, changed)) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            o_acc[i][0] *= alpha[0]; o_acc[i][1] *= alpha[0];
+            o_acc[i][2] *= alpha[1]; o_acc[i][3] *= alpha[1];
+          }
+          l_run[0] *= alpha[0];
+          l_run[1] *= alpha[1];
+          m_run[0] = m_new[0];
+          m_run[1] = m_new[1];
+        }
+        uint32_t pa[4];
+        {
+          float pr[2][4];
+#pragma unroll
+          for (int n8 = 0; n8 < 2; ++n8)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              pr[n8][e] = ptx::ex2_approx(sc[n8][e] - m_run[e >> 1]);
+              l_run[e >> 1] += pr[n8][e];
+            }
+          pa[0] = ptx::pack_bf16x2(pr[0][0], pr[0][1]);
+          pa[1] = ptx::pack_bf16x2(pr[0][2], pr[0][3]);
+          pa[2] = ptx::pack_bf16x2(pr[1][0], pr[1][1]);
+          pa[3] = ptx::pack_bf16x2(pr[1][2], pr[1][3]);
+        }
+        // ---- O += P V (16 tokens x 128 channels) ----
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const uint32_t chunk = (uint32_t)(2 * (jj & 3) + (lane >> 4));
+          const uint32_t addr = v_st + (jj >> 2) * kBoxBytes + v_lane_off + ((chunk ^ x7) << 4);
+          uint32_t r0, r1, r2, r3;
+          ptx::ldmatrix_x4_trans(addr, r0, r1, r2, r3);
+          ptx::mma_bf16_16816(o_acc[2 * jj], pa, r0, r1);
+          ptx::mma_bf16_16816(o_acc[2 * jj + 1], pa, r2, r3);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&bar_empty[s]);
+    }
+    // quad-reduce the row sums and publish this warp's state
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+    }
+    if (tig == 0) {
+      sm_m[warp][gid] = m_run[0]; sm_m[warp][gid + 8] = m_run[1];
+      sm_l[warp][gid] = l_run[0]; sm_l[warp][gid + 8] = l_run[1];
+    }
+  }
+  __syncthreads();   // every stage has been consumed; the ring is free for the merge buffer
+
+  float* obuf = reinterpret_cast<float*>(stage_base);      // [warp][16][kORowStride]
+  if (warp < kConsumerWarps) {
+    float f[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int row = gid + 8 * r;
+      float mg = sm_m[0][row];
+#pragma unroll
+      for (int w = 1; w < kConsumerWarps; ++w) mg = fmaxf(mg, sm_m[w][row]);
+      f[r] = m_run[r] == -INFINITY ? 0.f : ptx::ex2_approx(m_run[r] - mg);
+    }
+    float* ob = obuf + warp * 16 * kORowStride;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      *reinterpret_cast<float2*>(ob + gid * kORowStride + 8 * i + 2 * tig) = make_float2(o_acc[i][0] * f[0], o_acc[i][1] * f[0]);
+      *reinterpret_cast<float2*>(ob + (gid + 8) * kORowStride + 8 * i + 2 * tig) = make_float2(o_acc[i][2] * f[1], o_acc[i][3] * f[1]);
+    }
+  }
+  __syncthreads();
+  if (tid < 128) {
+    const int c = tid;
+    for (int row = 0; row < g; ++row) {
+      float mg = sm_m[0][row];
+#pragma unroll
+      for (int w = 1; w < kConsumerWarps; ++w) mg = fmaxf(mg, sm_m[w][row]);
+      float o = 0.f, ls = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) {
+        o += obuf[(w * 16 + row) * kORowStride + c];
+        const float mw = sm_m[w][row];
+        ls += mw == -INFINITY ? 0.f : sm_l[w][row] * ptx::ex2_approx(mw - mg);
+      }
+      const int hq = h * g + row;
+      if (p.n_split == 1) {
+        store_out(p, (((int64_t)l * p.B + b) * p.Hq + hq) * 128 + c, ls > 0.f ? o / ls : 0.f);
+      } else {
+        const int64_t pit = (((int64_t)lr * p.B + b) * p.Hq + hq) * p.n_split + split;
+        p.part_o[pit * 128 + c] = o;
+        if (c == 0) p.part_ml[pit] = make_float2(mg, ls);
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)sym;
+  });
+  return fn;
+}
+
+// K or V as a 3-D bf16 tensor (channel, row in plane, plane); box = 64 channels x 64 rows.
+bool make_kv_map(CUtensorMap* map, void* base, int64_t rows, int planes) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)planes};
+  cuuint64_t strides[2] = {256, (cuuint64_t)rows * 256};
+  cuuint32_t box[3] = {64, (cuuint32_t)kTileT, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kTargetCtas = 148 * 2 * 2;   // two waves of two CTAs per SM
+
+}  // namespace
+
+int decode_n_split(const ngc_cache* c, int layers) {
+  const int64_t strips = (int64_t)layers * c->B * c->Hkv;
+  if (strips >= kTargetCtas) return 1;
+  int ns = (int)((kTargetCtas + strips - 1) / strips);
+  const int by_len = (c->max_len + 1 + 4 * kTileT - 1) / (4 * kTileT);   // at least 4 tiles per split
+  if (ns > by_len) ns = by_len;
+  if (ns > 64) ns = 64;
+  return ns < 1 ? 1 : ns;
+}
+
+size_t decode_workspace_bytes(const ngc_cache* c, int layers) {
+  size_t worst = 0;
+  for (int n = 1; n <= layers; ++n) {
+    const int ns = decode_n_split(c, n);
+    if (ns <= 1) continue;
+    const size_t items = (size_t)n * c->B * c->Hq * ns;
+    const size_t bytes = align256(items * c->d * 4) + align256(items * 8);
+    if (bytes > worst) worst = bytes;
+  }
+  return worst;
+}
+
+}  // namespace ngc
+
+extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* new_k, const void* new_v,
+                                      int layer_begin, int layer_end, float scale,
+                                      void* out, int out_dtype,
+                                      void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream_) {
+  using namespace ngc;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!valid_cache(c) || !q || !out || layer_begin < 0 || layer_end > c->L || layer_begin >= layer_end)
+    return NGC_ERR_INVALID_ARG;
+  if ((new_k == nullptr) != (new_v == nullptr)) return NGC_ERR_INVALID_ARG;
+  if (out_dtype != NGC_F32 && !(out_dtype == NGC_BF16 && c->dtype == NGC_BF16)) return NGC_ERR_INVALID_ARG;
+  if (c->rows == 0) return NGC_OK;
+
+  DecodeParams p;
+  p.k = c->k; p.v = c->v; p.seq_off = c->seq_off; p.lens = c->lens;
+  p.q = q; p.new_k = new_k; p.new_v = new_v; p.out = out;
+  p.dev_status = dev_status; p.rows = c->rows;
+  p.L = c->L; p.B = c->B; p.Hq = c->Hq; p.Hkv = c->Hkv; p.d = c->d; p.g = c->Hq / c->Hkv;
+  p.layer_begin = layer_begin; p.n_layers = layer_end - layer_begin;
+  p.append = new_k != nullptr; p.out_bf16 = out_dtype == NGC_BF16;
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.n_split = decode_n_split(c, p.n_layers);
+  p.part_o = nullptr; p.part_ml = nullptr;
+  if (p.n_split > 1) {
+    const size_t items = (size_t)p.n_layers * c->B * c->Hq * p.n_split;
+    const size_t need = align256(items * c->d * 4) + align256(items * 8);
+    if (!ws || ws_bytes < need || ((uintptr_t)ws & 255)) return NGC_ERR_WORKSPACE;
+    p.part_o = (float*)ws;
+    p.part_ml = (float2*)((char*)ws + align256(items * c->d * 4));
+  }
+
+  const int row_vecs = c->d * elt_bytes(c->dtype) / 16;
+  if (p.append) {
+    append_kernel<<<(unsigned)(p.n_layers * c->B * c->Hkv), 64, 0, stream>>>(p, row_vecs);
+    int rc = launch_status();
+    if (rc != NGC_OK) return rc;
+  }
+
+  const bool stream_path = c->dtype == NGC_BF16 && c->d == 128 && p.g <= 16 && c->rows < 0x7fffffffLL &&
+                           (((uintptr_t)c->k | (uintptr_t)c->v) & 15) == 0;
+  if (stream_path) {
+    CUtensorMap map_k, map_v;
+    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv) || !make_kv_map(&map_v, c->v, c->rows, c->L * c->Hkv))
+      return NGC_ERR_UNSUPPORTED;
+    const int64_t items = (int64_t)p.n_layers * c->B * c->Hkv * p.n_split;
+    if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+    const int smem = kStages * kStageBytes + 1024;
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, [&] {
+      attr_err = cudaFuncSetAttribute(decode_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    });
+    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    decode_stream_kernel<<<(unsigned)items, kStreamThreads, smem, stream>>>(map_k, map_v, p);
+  } else {
+    const int64_t items = (int64_t)p.n_layers * c->B * c->Hq * p.n_split;
+    if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+    const unsigned grid = (unsigned)items;
+    if (c->dtype == NGC_F32 && c->d == 64) decode_generic_kernel<float, 64><<<grid, kGenWarps * 32, 0, stream>>>(p);
+    else if (c->dtype == NGC_F32) decode_generic_kernel<float, 128><<<grid, kGenWarps * 32, 0, stream>>>(p);
+    else if (c->d == 64) decode_generic_kernel<__nv_bfloat16, 64><<<grid, kGenWarps * 32, 0, stream>>>(p);
+    else decode_generic_kernel<__nv_bfloat16, 128><<<grid, kGenWarps * 32, 0, stream>>>(p);
+  }
+  int rc = launch_status();
+  if (rc != NGC_OK) return rc;
+  if (p.n_split > 1) {
+    combine_kernel<<<(unsigned)(p.n_layers * c->B * c->Hq), c->d, 0, stream>>>(p);
+    rc = launch_status();
+    if (rc != NGC_OK) return rc;
+  }
+  if (p.append && layer_end == c->L) {
+    bump_lens_kernel<<<(c->B + 255) / 256, 256, 0, stream>>>(p);
+    rc = launch_status();
+  }
+  return rc;
+}

@@ -1,0 +1,156 @@
+// ngc_evict_logprob: Eq. (1) of the paper (Section 4.3), fp64.
+//
+// One CTA per list.  With e_t = exp(s_t - M) (M = largest candidate logit) the
+// partition function of step j is the mass still present:
+//   rem_j = sum_{t never drawn} e_t + sum_{i >= j} e_sigma_i ,
+// so all K of them come from one scan over sigma taken from the tail, by
+// additions only (the remaining-mass bookkeeping the paper mentions after
+// Eq. (1), arranged so that nothing is subtracted).  Reductions and the scan
+// use a fixed tree order: results are reproducible run to run.
+#include "ngc_common.cuh"
+
+namespace ngc {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+
+struct LogprobParams {
+  const float* logits;
+  const int32_t* n;
+  const int32_t* n_protect;
+  const int32_t* budget;
+  const int32_t* kept_order;
+  double* logp;
+  int32_t* dev_status;
+  int G, n_max, k_max;
+};
+
+__device__ double block_sum(double v, double* s_red) {
+  v = warp_sum(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double t = 0.0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) t += s_red[w];
+  return t;
+}
+
+__global__ void __launch_bounds__(kThreads) logprob_kernel(LogprobParams p) {
+  extern __shared__ uint32_t bitmap[];
+  __shared__ double s_red[kWarps];
+  __shared__ float s_redf[kWarps];
+  __shared__ int s_bad;
+
+  const int64_t li = blockIdx.x;
+  const int64_t outer = li / p.G;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = p.n[outer];
+  const int P = p.n_protect ? p.n_protect[outer] : 0;
+  const int K = p.budget[outer];
+  const int Kp = K - P;
+  const float* s = p.logits + li * p.n_max;
+  const int32_t* sigma = p.kept_order + li * p.k_max;
+  const double kNaN = __longlong_as_double(0x7ff8000000000000LL);
+
+  if (!(P >= 0 && P <= K && K <= n && n <= p.n_max && Kp <= p.k_max)) {
+    if (tid == 0) { set_dev_status(p.dev_status, NGC_DEV_BAD_COUNTS); p.logp[li] = kNaN; }
+    return;
+  }
+  // ---- mark the drawn units; refuse repeats and out-of-range entries ----
+  if (tid == 0) s_bad = 0;
+  for (int w = tid; w < (n + 31) / 32; w += kThreads) bitmap[w] = 0u;
+  __syncthreads();
+  int bad = 0;
+  for (int j = tid; j < Kp; j += kThreads) {
+    const int t = sigma[j];
+    if (t < P || t >= n) bad = 1;
+    else if (atomicOr(&bitmap[t >> 5], 1u << (t & 31)) & (1u << (t & 31))) bad = 1;
+  }
+  if (bad) atomicOr(&s_bad, 1);
+  __syncthreads();
+  if (s_bad) {
+    if (tid == 0) { set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); p.logp[li] = kNaN; }
+    return;
+  }
+  if (Kp == 0) {
+    if (tid == 0) p.logp[li] = 0.0;
+    return;
+  }
+  // ---- M = max candidate logit ----
+  float mx = -INFINITY;
+  int nan_seen = 0;
+  for (int t = P + tid; t < n; t += kThreads) {
+    const float v = s[t];
+    if (v != v) nan_seen = 1;
+    mx = fmaxf(mx, v);
+  }
+  mx = warp_max(mx);
+  if (lane == 0) s_redf[warp] = mx;
+  if (nan_seen) atomicOr(&s_bad, 1);
+  __syncthreads();
+  mx = s_redf[0];
+#pragma unroll
+  for (int w = 1; w < kWarps; ++w) mx = fmaxf(mx, s_redf[w]);
+  if (s_bad) {
+    if (tid == 0) { set_dev_status(p.dev_status, NGC_DEV_NAN_LOGIT); p.logp[li] = kNaN; }
+    return;
+  }
+  const double M = (double)mx;
+  // ---- mass of the candidates that are never drawn ----
+  double u = 0.0;
+  for (int t = P + tid; t < n; t += kThreads)
+    if (!((bitmap[t >> 5] >> (t & 31)) & 1u)) u += exp((double)s[t] - M);
+  double carry = block_sum(u, s_red);
+  // ---- scan sigma from the tail: rem_j = carry + e_sigma_j + ... ----
+  double acc = 0.0;
+  for (int base = 0; base < Kp; base += kThreads) {
+    const int j = Kp - 1 - (base + tid);
+    double sj = 0.0, e = 0.0;
+    if (j >= 0) { sj = (double)s[sigma[j]] - M; e = exp(sj); }
+    double incl = e;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    __syncthreads();
+    if (lane == 31) s_red[warp] = incl;
+    __syncthreads();
+    double off = 0.0, tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      if (w < warp) off += s_red[w];
+      tot += s_red[w];
+    }
+    if (j >= 0) acc += sj - log(carry + off + incl);
+    carry += tot;
+  }
+  const double total = block_sum(acc, s_red);
+  if (tid == 0) p.logp[li] = total;
+}
+
+}  // namespace
+}  // namespace ngc
+
+extern "C" int ngc_evict_logprob(const float* logits, const int32_t* n, const int32_t* n_protect,
+                                 const int32_t* budget, const int32_t* kept_order,
+                                 int n_batches, int B, int G, int n_max, int k_max, double* logp,
+                                 void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  using namespace ngc;
+  (void)ws; (void)ws_bytes;
+  if (!logits || !n || !budget || !kept_order || !logp || n_batches <= 0 || B <= 0 || G <= 0 || n_max <= 0 || k_max <= 0)
+    return NGC_ERR_INVALID_ARG;
+  const int64_t lists = (int64_t)n_batches * B * G;
+  if (lists > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)((n_max + 31) / 32) * 4;
+  if (smem > 200 * 1024) return NGC_ERR_UNSUPPORTED;
+  if (smem > 48 * 1024)
+    NGC_CUDA_TRY(cudaFuncSetAttribute(logprob_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  LogprobParams p;
+  p.logits = logits; p.n = n; p.n_protect = n_protect; p.budget = budget; p.kept_order = kept_order;
+  p.logp = logp; p.dev_status = dev_status; p.G = G; p.n_max = n_max; p.k_max = k_max;
+  logprob_kernel<<<(unsigned)lists, kThreads, smem, (cudaStream_t)stream>>>(p);
+  return launch_status();
+}

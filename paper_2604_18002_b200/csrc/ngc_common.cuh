@@ -1,0 +1,71 @@
+// Shared host/device helpers of the NGC CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ngc.h"
+
+namespace ngc {
+
+// Last cudaError_t seen by a failing call on this host thread.
+extern thread_local int g_last_cuda_error;
+
+inline int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return NGC_ERR_CUDA;
+}
+
+#define NGC_CUDA_TRY(expr)                              \
+  do {                                                  \
+    cudaError_t _e = (expr);                            \
+    if (_e != cudaSuccess) return ::ngc::cuda_fail(_e); \
+  } while (0)
+
+// Check the launch that was just enqueued.
+inline int launch_status() {
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? NGC_OK : cuda_fail(e);
+}
+
+__host__ __device__ inline int lists_G(int lists, int L, int Hkv) {
+  return lists == NGC_LISTS_SHARED ? 1 : (lists == NGC_LISTS_PER_LAYER ? L : L * Hkv);
+}
+__host__ __device__ inline int list_of(int lists, int l, int h, int Hkv) {
+  return lists == NGC_LISTS_SHARED ? 0 : (lists == NGC_LISTS_PER_LAYER ? l : l * Hkv + h);
+}
+
+inline int elt_bytes(int dtype) { return dtype == NGC_F32 ? 4 : 2; }
+
+inline bool valid_cache(const ngc_cache* c) {
+  return c && c->k && c->v && c->seq_off && c->lens && c->L > 0 && c->B > 0 && c->Hq > 0 && c->Hkv > 0 &&
+         c->Hq % c->Hkv == 0 && (c->d == 64 || c->d == 128) && c->rows >= 0 && c->max_len >= 0 &&
+         (c->dtype == NGC_F32 || c->dtype == NGC_BF16);
+}
+
+inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+#ifdef __CUDACC__
+// First error wins.
+__device__ __forceinline__ void set_dev_status(int32_t* st, int code) {
+  if (st) atomicCAS(st, 0, code);
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+#endif
+
+}  // namespace ngc

@@ -1,0 +1,276 @@
+// ngc_sample_evict: Gumbel-top-k draw of the keep set (paper Section 4.3).
+//
+// One CTA per list.  Every candidate unit gets a 64-bit sort key: the
+// order-preserving integer image of its perturbed fp32 key in the high word
+// and the bit-inverted index in the low word, so that one descending integer
+// sort realises "larger key first, equal keys -> smaller index first".  The
+// keys live in shared memory (lists up to kSampleSmemMaxUnits candidates) or in
+// the caller's workspace (longer lists) and are ordered by a bitonic network;
+// the kept prefix is then marked in a bitmap whose prefix popcounts place the
+// ascending kept list.  Integer work throughout; results do not depend on the
+// launch shape.
+//
+// This translation unit must be compiled WITHOUT fast-math: the Gumbel
+// transform is a fixed sequence of correctly rounded fp32 operations.
+#include "ngc_common.cuh"
+#include "ngc_plan.h"
+
+namespace ngc {
+namespace {
+
+// ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3") ----
+__device__ __forceinline__ uint4 philox4x32_10(uint4 ctr, uint2 key) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, ctr.x), lo0 = 0xD2511F53u * ctr.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, ctr.z), lo1 = 0xCD9E8D57u * ctr.z;
+    ctr = make_uint4(hi1 ^ ctr.y ^ key.x, lo1, hi0 ^ ctr.w ^ key.y, lo0);
+    key.x += 0x9E3779B9u;
+    key.y += 0xBB67AE85u;
+  }
+  return ctr;
+}
+
+// Natural logarithm of a positive normal float by a fixed recipe: range
+// reduction to m in [sqrt(1/2), sqrt(2)), then log m = 2 atanh((m-1)/(m+1))
+// with a degree-4 polynomial in z^2.  Only IEEE round-to-nearest add, mul,
+// div and fma, so every machine produces the same bits.
+__device__ __forceinline__ float det_log(float x) {
+  const uint32_t bits = __float_as_uint(x);
+  int e = (int)(bits >> 23) - 127;
+  float m = __uint_as_float((bits & 0x007FFFFFu) | 0x3F800000u);
+  if (m >= 1.41421354f) { m = __fmul_rn(m, 0.5f); e += 1; }
+  const float z = __fdiv_rn(__fsub_rn(m, 1.0f), __fadd_rn(m, 1.0f));
+  const float w = __fmul_rn(z, z);
+  float p = 2.0f / 9.0f;
+  p = __fmaf_rn(p, w, 2.0f / 7.0f);
+  p = __fmaf_rn(p, w, 2.0f / 5.0f);
+  p = __fmaf_rn(p, w, 2.0f / 3.0f);
+  p = __fmaf_rn(p, w, 2.0f);
+  const float r = __fmul_rn(z, p);
+  return __fmaf_rn((float)e, 0.693147180559945f, r);
+}
+
+__device__ __forceinline__ float gumbel_from_word(uint32_t x) {
+  const float u = __fmul_rn((float)(2u * (x >> 9) + 1u), 5.9604644775390625e-08f);   // odd multiple of 2^-24
+  return -det_log(-det_log(u));
+}
+
+// Order-preserving map float -> uint32 (larger float, larger integer; -0 == +0 upstream).
+__device__ __forceinline__ uint32_t float_image(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+struct SampleParams {
+  const float* logits;
+  const int32_t* n;
+  const int32_t* n_protect;
+  const int32_t* budget;
+  int32_t* kept_order;
+  int32_t* kept_sorted;
+  uint8_t* keep_mask;
+  unsigned long long* ws_keys;   // [lists][pad_max] when sorting in global memory
+  int32_t* dev_status;
+  uint64_t seed, round;
+  uint32_t list_base;
+  int B, G, n_max, k_max, greedy;
+  int pad_max;                   // power of two >= n_max
+};
+
+template <bool kSmemKeys>
+__global__ void sample_kernel(SampleParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ int s_flag;
+  __shared__ int s_warp_tot[32];
+  __shared__ int s_carry;
+
+  const int li = blockIdx.x;
+  const int b = li / p.G;
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  const int n = p.n[b];
+  const int P = p.n_protect ? p.n_protect[b] : 0;
+  const int K = p.budget[b];
+  const float* s = p.logits + (int64_t)li * p.n_max;
+  int32_t* ko = p.kept_order + (int64_t)li * p.k_max;
+  int32_t* ks = p.kept_sorted + (int64_t)li * p.k_max;
+  uint8_t* km = p.keep_mask ? p.keep_mask + (int64_t)li * p.n_max : nullptr;
+
+  unsigned long long* keys;
+  uint32_t* bitmap;
+  if (kSmemKeys) {
+    keys = reinterpret_cast<unsigned long long*>(smem_raw);
+    bitmap = reinterpret_cast<uint32_t*>(smem_raw + (size_t)p.pad_max * 8);
+  } else {
+    keys = p.ws_keys + (int64_t)li * p.pad_max;
+    bitmap = reinterpret_cast<uint32_t*>(smem_raw);
+  }
+
+  if (tid == 0) s_flag = 0;
+  __syncthreads();
+  const bool counts_ok = P >= 0 && P <= K && K <= n && n <= p.n_max && K <= p.k_max;
+  const int n_cand = counts_ok ? n - P : 0;
+  const int Kp = counts_ok ? K - P : 0;
+  int pad = 1;
+  while (pad < n_cand) pad <<= 1;
+
+  // ---- perturbed keys: one Philox call serves units 4q .. 4q+3 ----
+  if (counts_ok) {
+    const uint2 key = make_uint2((uint32_t)p.seed, (uint32_t)(p.seed >> 32));
+    const uint32_t list_id = p.list_base + (uint32_t)li;
+    int nan_seen = 0;
+    for (int q = (P >> 2) + tid; q <= ((n - 1) >> 2) && n > 0; q += nthr) {
+      uint32_t w[4] = {0, 0, 0, 0};
+      if (!p.greedy) {
+        const uint4 r = philox4x32_10(make_uint4((uint32_t)q, list_id, (uint32_t)p.round, (uint32_t)(p.round >> 32)), key);
+        w[0] = r.x; w[1] = r.y; w[2] = r.z; w[3] = r.w;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int i = 4 * q + j;
+        if (i >= P && i < n) {
+          const float si = s[i];
+          if (si != si) nan_seen = 1;
+          float kf = p.greedy ? si : __fadd_rn(si, gumbel_from_word(w[j]));
+          kf = __fadd_rn(kf, 0.0f);                       // -0 -> +0
+          keys[i - P] = ((unsigned long long)float_image(kf) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
+        }
+      }
+    }
+    for (int i = n_cand + tid; i < pad; i += nthr) keys[i] = 0ull;   // below every real key
+    if (nan_seen) atomicOr(&s_flag, 1);
+  }
+  __syncthreads();
+  const bool ok = counts_ok && s_flag == 0;
+  if (!ok) {
+    if (tid == 0) set_dev_status(p.dev_status, counts_ok ? NGC_DEV_NAN_LOGIT : NGC_DEV_BAD_COUNTS);
+    for (int j = tid; j < p.k_max; j += nthr) { ko[j] = -1; ks[j] = -1; }
+    if (km) for (int i = tid; i < p.n_max; i += nthr) km[i] = 0;
+    return;
+  }
+
+  // ---- bitonic sort, descending ----
+  for (int k = 2; k <= pad; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int t = tid; t < (pad >> 1); t += nthr) {
+        const int i = 2 * t - (t & (j - 1));
+        const int l = i + j;
+        const unsigned long long x = keys[i], y = keys[l];
+        const bool desc = (i & k) == 0;
+        if ((x < y) == desc) { keys[i] = y; keys[l] = x; }
+      }
+      __syncthreads();
+    }
+  }
+
+  // ---- sigma: the drawn units in descending key order; bitmap of kept units ----
+  const int n_words = (n + 31) >> 5;
+  for (int wd = tid; wd < n_words; wd += nthr) {
+    // protected prefix [0, P)
+    const int lo = wd << 5;
+    uint32_t m = 0;
+    if (P >= lo + 32) m = 0xFFFFFFFFu;
+    else if (P > lo) m = (1u << (P - lo)) - 1u;
+    bitmap[wd] = m;
+  }
+  __syncthreads();
+  for (int j = tid; j < p.k_max; j += nthr) {
+    int idx = -1;
+    if (j < Kp) {
+      idx = (int)(0xFFFFFFFFu - (uint32_t)(keys[j] & 0xFFFFFFFFull));
+      atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
+    }
+    ko[j] = idx;
+  }
+  __syncthreads();
+
+  // ---- ascending kept list from the prefix popcounts of the bitmap ----
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  const int lane = tid & 31, warp = tid >> 5, n_warps = nthr >> 5;
+  for (int base = 0; base < n_words; base += nthr) {
+    const int wd = base + tid;
+    const uint32_t m = wd < n_words ? bitmap[wd] : 0u;
+    const int cnt = __popc(m);
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) s_warp_tot[warp] = incl;
+    __syncthreads();
+    int warp_off = 0;
+    for (int w2 = 0; w2 < warp; ++w2) warp_off += s_warp_tot[w2];
+    int pos = s_carry + warp_off + incl - cnt;
+    uint32_t mm = m;
+    while (mm) {
+      const int bit = __ffs(mm) - 1;
+      mm &= mm - 1;
+      ks[pos++] = (wd << 5) + bit;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int tot = 0;
+      for (int w2 = 0; w2 < n_warps; ++w2) tot += s_warp_tot[w2];
+      s_carry += tot;
+    }
+    __syncthreads();
+  }
+  for (int j = K + tid; j < p.k_max; j += nthr) ks[j] = -1;
+  if (km) {
+    for (int i = tid; i < p.n_max; i += nthr)
+      km[i] = (i < n && ((bitmap[i >> 5] >> (i & 31)) & 1u)) ? 1 : 0;
+  }
+}
+
+inline int pow2_at_least(int x) {
+  int p = 1;
+  while (p < x) p <<= 1;
+  return p;
+}
+
+}  // namespace
+
+size_t sample_workspace_bytes(int B, int G, int n_max) {
+  if (n_max <= kSampleSmemMaxUnits) return 0;
+  return align256((size_t)B * G * pow2_at_least(n_max) * 8);
+}
+
+}  // namespace ngc
+
+extern "C" int ngc_sample_evict(const float* logits, const int32_t* n, const int32_t* n_protect,
+                                const int32_t* budget, int B, int G, int n_max, int k_max,
+                                uint64_t seed, uint64_t round, uint32_t list_base, int greedy,
+                                int32_t* kept_order, int32_t* kept_sorted, uint8_t* keep_mask,
+                                void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  using namespace ngc;
+  if (!logits || !n || !budget || !kept_order || !kept_sorted || B <= 0 || G <= 0 || n_max <= 0 || k_max <= 0)
+    return NGC_ERR_INVALID_ARG;
+  if ((int64_t)B * G > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+  SampleParams p;
+  p.logits = logits; p.n = n; p.n_protect = n_protect; p.budget = budget;
+  p.kept_order = kept_order; p.kept_sorted = kept_sorted; p.keep_mask = keep_mask;
+  p.dev_status = dev_status; p.seed = seed; p.round = round; p.list_base = list_base;
+  p.B = B; p.G = G; p.n_max = n_max; p.k_max = k_max; p.greedy = greedy;
+  p.pad_max = pow2_at_least(n_max);
+  p.ws_keys = nullptr;
+  const size_t bitmap_bytes = (size_t)((n_max + 31) / 32) * 4;
+  int threads = p.pad_max >= 2048 ? 1024 : (p.pad_max >= 512 ? 256 : 64);
+  const unsigned grid = (unsigned)(B * G);
+  if (n_max <= kSampleSmemMaxUnits) {
+    const size_t smem = (size_t)p.pad_max * 8 + bitmap_bytes;
+    if (smem > 48 * 1024)
+      NGC_CUDA_TRY(cudaFuncSetAttribute(sample_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    sample_kernel<true><<<grid, threads, smem, (cudaStream_t)stream>>>(p);
+  } else {
+    const size_t need = sample_workspace_bytes(B, G, n_max);
+    if (!ws || ws_bytes < need) return NGC_ERR_WORKSPACE;
+    if (bitmap_bytes > 200 * 1024) return NGC_ERR_UNSUPPORTED;
+    p.ws_keys = (unsigned long long*)ws;
+    if (bitmap_bytes > 48 * 1024)
+      NGC_CUDA_TRY(cudaFuncSetAttribute(sample_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bitmap_bytes));
+    sample_kernel<false><<<grid, threads, bitmap_bytes, (cudaStream_t)stream>>>(p);
+  }
+  return launch_status();
+}
