@@ -1,0 +1,382 @@
+"""Benchmark of the NGC hot path on B200.
+
+One "step" = one pass of the whole hot path over one batch of synthetic
+rollouts: an eviction round (score -> Gumbel-top-k sample -> log-prob ->
+in-place compaction) followed by the workload's decode steps (append + ragged
+attention over the surviving cache).  The workload is the 1.5B-shaped GQA
+rollout step at B = 64: 28 layers, 12 query / 2 KV heads, d = 128, bf16 K/V,
+4096 cached tokens evicted to 2048, then 256 decode steps.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ngc|reference]
+
+Prints ONE JSON line (rank 0).  `value` is tokens/s with all inputs resident in
+HBM; `e2e` is the same step driven from pinned host buffers through the public
+host entry (copies inside the timed region); `roofline` is the decode kernel's
+achieved HBM bandwidth; `cpu_baseline` is the CPU oracle timed on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2604_18002_b200 import synth
+
+CFG = dict(synth.CONFIGS[2])
+WORKLOAD = "config2: 1.5B-shaped GQA rollout step (L28, 12q/2kv, d128, bf16, B64, 4096->2048 tokens, 256 decode steps)"
+METRIC = "evict+compact+decode tokens/sec at B=64"
+W_RECENT = 5
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            j = json.load(f)
+        return float(j["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.idx), "-lms", "50"], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def stop(self, t_begin=None, t_end=None):
+        """Summary of the samples that arrived inside [t_begin, t_end] (the timed region)."""
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, ln in self.lines:
+            if t_begin is not None and not (t_begin <= ts <= t_end):
+                continue
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x: float, world, device):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def algorithmic_decode_bytes(cfg, visible_tokens_total):
+    """K and V rows every decode launch must read: per (sequence, visible token) L*Hkv*2*d*2 bytes."""
+    per_token = cfg["L"] * cfg["Hkv"] * 2 * cfg["d"] * 2
+    return per_token * visible_tokens_total
+
+
+# ------------------------------------------------------------------------------------ CUDA arm
+
+def run_ngc(args):
+    from paper_2604_18002_b200 import binding as ngc
+    from paper_2604_18002_b200.rollout import HostStep, NgcRollout
+
+    rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    cfg = CFG
+    L, B, Hq, Hkv, d, T, K, steps = cfg["L"], cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["d"], cfg["T"], cfg["budget"], cfg["steps"]
+    if args.decode_steps:
+        steps = args.decode_steps
+    if args.batch:
+        B = args.batch
+    dtype = torch.bfloat16
+    # every rank owns a full batch of B rollouts (weak scaling); Philox streams use global list ids
+    ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=T, n_max=T, k_max=K, lists=cfg["lists"], device=dev,
+                    list_base=rank * B, w=W_RECENT)
+    seed = cfg["data_seed"] + 1000 * rank
+    src = synth.make_cache(L, B, Hq, Hkv, d, dtype, [T] * B, capacity=T, seed=seed, outlier_channels=cfg["outliers"], device=dev)
+    ro.cache.k.copy_(src.k)
+    ro.cache.v.copy_(src.v)
+    del src
+    lens0 = torch.full((B,), T, dtype=torch.int32, device=dev)
+    logits = synth.make_logits(B, 1, T, seed=seed + 7, std=cfg["logit_std"], device=dev)
+    n_t = lens0.clone()
+    k_t = torch.full((B,), K, dtype=torch.int32, device=dev)
+    q = synth.make_queries(L, B, Hq, d, dtype, seed=seed + 11, steps=steps, device=dev)
+    nk, nv = synth.make_new_kv(L, B, Hkv, d, dtype, seed=seed + 13, steps=steps, device=dev)
+    q_recent = synth.normal((L, B, Hq, W_RECENT, d), seed + 17, dtype, device=dev)
+    out = torch.empty((steps, L, B, Hq, d), dtype=torch.float32, device=dev)
+    noise_seed = cfg["noise_seed"]
+
+    ev_pairs = []
+
+    def one_step(step_idx, time_decode=False):
+        ro.cache.lens.copy_(lens0, non_blocking=True)
+        ro.eviction_round(n_t, None, k_t, noise_seed, step_idx, q_recent=q_recent, logits=logits)
+        for s in range(steps):
+            if time_decode:
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e0.record()
+                ro.decode_step(q[s], out[s], nk[s], nv[s])
+                e1.record()
+                ev_pairs.append((e0, e1))
+            else:
+                ro.decode_step(q[s], out[s], nk[s], nv[s])
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()          # nvidia-smi takes a while to come up: start it before the warm-up
+    for w in range(args.warmup):
+        one_step(w)
+    torch.cuda.synchronize()
+    ro.check_status()
+
+    launches0 = ro.launches
+    barrier(world)
+    torch.cuda.synchronize()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    wall0 = time.perf_counter()
+    t0.record()
+    for k in range(args.steps):
+        one_step(args.warmup + k, time_decode=True)
+    t1.record()
+    torch.cuda.synchronize()
+    wall1 = time.perf_counter()
+    barrier(world)
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
+    ms_total = max_over_ranks(t0.elapsed_time(t1), world, dev)
+    ro.check_status()
+    launches = ro.launches - launches0
+    ms_per_step = ms_total / args.steps
+    tokens = B * steps * world
+    value = tokens / (ms_per_step * 1e-3)
+
+    # roofline of the dominant kernel (decode): algorithmic K/V bytes per launch / mean launch time
+    dec_ms = [a.elapsed_time(b) for a, b in ev_pairs]
+    mean_dec_ms = float(np.mean(dec_ms))
+    visible_total = sum(B * (K + s + 1) for s in range(steps)) / steps      # per launch, averaged over the step
+    bytes_per_launch = algorithmic_decode_bytes(cfg, visible_total)
+    peak, peak_kind = peaks()
+    achieved = bytes_per_launch / (mean_dec_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (per ngc_decode_attn_ragged call: append + attention + lens bump)",
+                "achieved": round(achieved, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "traffic": args.traffic, "bytes_per_launch": int(bytes_per_launch),
+                "ms_per_launch": round(mean_dec_ms, 4), "decode_share_of_step": round(sum(dec_ms) / ms_total, 4)}
+
+    result = {"metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+              "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
+              "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+              "config": {"workload": WORKLOAD, "decode_steps": steps, "batch_per_gpu": B, "parallelism": f"batch-shard x{world}, no collective",
+                         "l2": "inputs larger than L2 (7.5 GB cache streamed per decode step)", "score_in_step": True,
+                         "logits": "synthetic N(0, var 2), shared list"},
+              "gpu_launches": int(launches), "roofline": roofline}
+    if clocks is not None:
+        result["clocks"] = clocks
+
+    # ---- end to end from pinned host buffers (all ranks take part, rank 0 reports) ----
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        hs = HostStep(ro, steps)
+        pin = dict(pin_memory=True)
+        h_k = torch.empty(ro.cache.k.shape, dtype=dtype, **pin).copy_(ro.cache.k)
+        h_v = torch.empty(ro.cache.v.shape, dtype=dtype, **pin).copy_(ro.cache.v)
+        h_lens = torch.empty(B, dtype=torch.int32, **pin).copy_(lens0)
+        h_logits = torch.empty(logits.shape, dtype=torch.float32, **pin).copy_(logits)
+        h_q = torch.empty(q.shape, dtype=dtype, **pin).copy_(q)
+        h_nk = torch.empty(nk.shape, dtype=dtype, **pin).copy_(nk)
+        h_nv = torch.empty(nv.shape, dtype=dtype, **pin).copy_(nv)
+        h_qr = torch.empty(q_recent.shape, dtype=dtype, **pin).copy_(q_recent)
+        h_out = torch.empty(out.shape, dtype=torch.float32, **pin)
+        h_ko = torch.empty(ro.kept_order.shape, dtype=torch.int32, **pin)
+        h_lp = torch.empty(ro.logp.shape, dtype=torch.float64, **pin)
+        torch.cuda.synchronize()
+
+        def host_step(i):
+            return hs.run(h_k, h_v, h_lens, h_logits, h_q, h_nk, h_nv, h_out, h_ko, h_lp, n_t, None, k_t, noise_seed, i,
+                          h_q_recent=h_qr, d_q_recent=q_recent)
+        host_step(0)
+        torch.cuda.synchronize()
+        barrier(world)
+        c0 = time.perf_counter()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(e2e_steps):
+            h2d, d2h = host_step(100 + i)
+        e1.record()
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - c0
+        barrier(world)
+        e2e_ms = max_over_ranks(max(e0.elapsed_time(e1), wall * 1e3), world, dev) / e2e_steps
+        ro.check_status()
+        result["e2e"] = {"value": round(tokens / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
+                         "d2h_bytes_per_step": int(d2h), "ms_per_step": round(e2e_ms, 3), "steps": e2e_steps,
+                         "api": "paper_2604_18002_b200.rollout.HostStep.run (pinned host buffers, copies overlapped with compute)"}
+        del h_k, h_v, h_q, h_out
+
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1 only) ----
+    if rank == 0 and world == 1 and not args.no_cpu:
+        result["cpu_baseline"] = cpu_baseline_sample(args.cpu_seqs, args.cpu_decode_steps)
+    if rank == 0:
+        print(json.dumps(result), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------ CPU oracle arm
+
+def oracle_step(cache_np, logits, q, nk, nv, qr, K, rnd, decode_steps, seed):
+    """One step of the workload through the CPU oracle, as it stands."""
+    import oracle
+    k, v, so, lens = cache_np
+    B = lens.shape[0]
+    budget = np.full(B, K, np.int32)
+    oracle.score_evict(k, so, lens, qr, 1, 0)
+    ko, ks, _, st = oracle.sample_evict(logits, lens, None, budget, K, seed=seed, rnd=rnd)
+    oracle.evict_logprob(logits, lens, None, budget, ko)
+    kc, vc, nl, rc = oracle.compact_kv(k, v, so, lens, ks, budget, 0)
+    lens2 = nl.copy()
+    for s in range(decode_steps):
+        oracle.decode_attn(kc, vc, so, lens2, q[s], nk[s], nv[s])
+
+
+def make_cpu_sample(n_seqs, decode_steps):
+    cfg = CFG
+    L, Hq, Hkv, d, T = cfg["L"], cfg["Hq"], cfg["Hkv"], cfg["d"], cfg["T"]
+    c = synth.make_cache(L, n_seqs, Hq, Hkv, d, torch.bfloat16, [T] * n_seqs, capacity=T, seed=0, outlier_channels=cfg["outliers"])
+    logits = synth.make_logits(n_seqs, 1, T, seed=7, std=cfg["logit_std"]).numpy()
+    q = synth.to_numpy(synth.make_queries(L, n_seqs, Hq, d, torch.bfloat16, seed=11, steps=decode_steps))
+    nk, nv = synth.make_new_kv(L, n_seqs, Hkv, d, torch.bfloat16, seed=13, steps=decode_steps)
+    qr = synth.to_numpy(synth.normal((L, n_seqs, Hq, W_RECENT, d), 17, torch.bfloat16))
+    cache_np = (synth.to_numpy(c.k), synth.to_numpy(c.v), c.seq_off.numpy(), c.lens.numpy())
+    return cache_np, logits, q, synth.to_numpy(nk), synth.to_numpy(nv), qr
+
+
+def cpu_baseline_sample(n_seqs, decode_steps):
+    import oracle
+    data = make_cpu_sample(n_seqs, decode_steps)
+    t0 = time.perf_counter()
+    oracle_step(*data, CFG["budget"], 0, decode_steps, CFG["noise_seed"])
+    dt = time.perf_counter() - t0
+    return {"value": round(n_seqs * decode_steps / dt, 2), "unit": "tokens/s", "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"{n_seqs} of {CFG['B']} sequences, one eviction round (score+sample+logprob+compact) + {decode_steps} of "
+                      f"{CFG['steps']} decode steps, {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    n_seqs, dsteps = args.cpu_seqs, args.cpu_decode_steps
+    data = make_cpu_sample(n_seqs, dsteps)
+    for w in range(args.warmup):
+        oracle_step(*data, CFG["budget"], w, dsteps, CFG["noise_seed"])
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        oracle_step(*data, CFG["budget"], args.warmup + k, dsteps, CFG["noise_seed"])
+    dt = (time.perf_counter() - t0) / args.steps
+    value = n_seqs * dsteps / dt
+    sample = (f"each step: {n_seqs} of {CFG['B']} sequences, one eviction round + {dsteps} of {CFG['steps']} decode steps "
+              f"({dt:.1f} s per step)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 2), "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 1), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": round(value, 2), "unit": "tokens/s", "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 2), "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ngc", choices=["ngc", "reference"])
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's 256 decode steps (profiling only)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's B = 64 (profiling only)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-seqs", type=int, default=4)
+    ap.add_argument("--cpu-decode-steps", type=int, default=48)
+    ap.add_argument("--traffic", type=float, default=None, help="dram bytes per decode launch from an ncu capture (profiles/)")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ngc" and not (args.decode_steps or args.batch):
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the CPU oracle")
+        run_ngc(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -104,6 +104,11 @@ int ngc_last_cuda_error(void);
  * preserved between calls, and calls sharing a workspace must be stream-ordered. */
 size_t ngc_workspace_bytes(int op, const ngc_cache* c, int G, int n_max, int k_max);
 
+/* Number of token-range splits ngc_decode_attn_ragged uses for a call over
+ * `layers` layers of this cache (1 = every strip is handled by one CTA and no
+ * combine kernel runs).  Host-only planning query. */
+int ngc_decode_splits(const ngc_cache* c, int layers);
+
 /*
  * Eviction scores -- Section 4.2 ("Parameterizing eviction actions" and
  * "Coarsening the action space").  For every list: psi_t = mean, over the

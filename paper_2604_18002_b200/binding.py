@@ -24,7 +24,7 @@ OP_SCORE, OP_SAMPLE, OP_LOGPROB, OP_COMPACT, OP_DECODE = range(5)
 DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "strip full",
               5: "lists disagree", 6: "timeout"}
 
-EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_score_evict",
+EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
            "ngc_sample_evict", "ngc_evict_logprob", "ngc_compact_kv", "ngc_decode_attn_ragged"]
 
 
@@ -52,6 +52,8 @@ def _load():
     lib.ngc_last_cuda_error.restype = i32
     lib.ngc_workspace_bytes.restype = sz
     lib.ngc_workspace_bytes.argtypes = [i32, C.POINTER(CacheDesc), i32, i32, i32]
+    lib.ngc_decode_splits.restype = i32
+    lib.ngc_decode_splits.argtypes = [C.POINTER(CacheDesc), i32]
     lib.ngc_score_evict.restype = i32
     lib.ngc_score_evict.argtypes = [C.POINTER(CacheDesc), vp, i32, i32, i32, i32, vp, i32, vp, sz, vp, vp]
     lib.ngc_sample_evict.restype = i32
@@ -145,6 +147,11 @@ def workspace_bytes(op: int, cache: Optional[NgcCache] = None, G: int = 1, n_max
     else:
         d = CacheDesc(None, None, None, None, 0, 1, B or 1, 1, 1, 128, BF16, 0)
     return int(lib.ngc_workspace_bytes(op, C.byref(d), G, n_max, k_max))
+
+
+def decode_splits(cache: NgcCache, layers: Optional[int] = None, append: bool = True) -> int:
+    d = cache.desc(1 if append else 0)
+    return int(lib.ngc_decode_splits(C.byref(d), cache.L if layers is None else layers))
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> Optional[torch.Tensor]:

@@ -23,6 +23,11 @@ const char* ngc_strerror(int status) {
 
 int ngc_last_cuda_error(void) { return ngc::g_last_cuda_error; }
 
+int ngc_decode_splits(const ngc_cache* c, int layers) {
+  if (!ngc::valid_cache(c) || layers <= 0) return 0;
+  return ngc::decode_n_split(c, layers);
+}
+
 size_t ngc_workspace_bytes(int op, const ngc_cache* c, int G, int n_max, int k_max) {
   switch (op) {
     case NGC_OP_SCORE: return c ? ngc::score_workspace_bytes(c, G, n_max) : 0;
