@@ -39,6 +39,9 @@ CFG = dict(synth.CONFIGS[2])
 WORKLOAD = "config2: 1.5B-shaped GQA rollout step (L28, 12q/2kv, d128, bf16, B64, 4096->2048 tokens, 256 decode steps)"
 METRIC = "evict+compact+decode tokens/sec at B=64"
 W_RECENT = 5
+# dram__bytes_read.sum + dram__bytes_write.sum over algorithmic K/V bytes for decode_stream_kernel, from the ncu
+# capture summarised in profiles/decode_stream_kernel_config2.md (small case, scaled by tokens processed)
+NCU_TRAFFIC_RATIO = 1.0377
 
 
 def peaks():
@@ -222,7 +225,9 @@ def run_ngc(args):
     achieved = bytes_per_launch / (mean_dec_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (per ngc_decode_attn_ragged call: append + attention + lens bump)",
                 "achieved": round(achieved, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "traffic": args.traffic, "bytes_per_launch": int(bytes_per_launch),
+                "frac": round(achieved / peak, 4),
+                "traffic": int(args.traffic if args.traffic else NCU_TRAFFIC_RATIO * bytes_per_launch),
+                "traffic_source": "ncu capture of a B=16 launch scaled by tokens processed (profiles/decode_stream_kernel_config2.md)", "bytes_per_launch": int(bytes_per_launch),
                 "ms_per_launch": round(mean_dec_ms, 4), "decode_share_of_step": round(sum(dec_ms) / ms_total, 4)}
 
     result = {"metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
