@@ -57,7 +57,8 @@ typedef enum {
   NGC_ERR_INVALID_ARG = -1,   /* null pointer, negative size, inconsistent shape */
   NGC_ERR_UNSUPPORTED = -2,   /* shape / dtype combination not built */
   NGC_ERR_WORKSPACE = -3,     /* workspace missing or smaller than ngc_workspace_bytes() */
-  NGC_ERR_CUDA = -4           /* a CUDA call failed; code in ngc_last_cuda_error() */
+  NGC_ERR_CUDA = -4,          /* a CUDA call failed; code in ngc_last_cuda_error() */
+  NGC_ERR_STATIC_SCRATCH = -5 /* launch needs more scratch than the built-in static array holds */
 } ngc_status;
 
 /* values written to *dev_status */
@@ -202,6 +203,38 @@ int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* new_k, const
                            int layer_begin, int layer_end, float scale,
                            void* out, int out_dtype,
                            void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
+
+/*
+ * ngc_decode_attn_ragged without a caller-supplied workspace.  (The paper has
+ * no counterpart: this entry exists for the library's users, not the method.)
+ *
+ * Some callers cannot hand the library device scratch memory: code embedded
+ * in a host application that has already given every byte of device memory
+ * to its own pool, plug-ins that are not allowed to call the CUDA allocator,
+ * and latency-critical serving loops where a cudaMalloc (which synchronises
+ * the whole device) must never happen.  For them the split partials of the
+ * decode kernel live in a scratch array built into the library image
+ * (NGC_STATIC_SCRATCH_BYTES of device memory, resident on every GPU that
+ * loads the library until the process exits).  The call allocates nothing,
+ * frees nothing and calls no allocating routine.
+ *
+ * Same arguments and results as ngc_decode_attn_ragged, minus ws/ws_bytes.
+ * - A launch whose scratch need exceeds NGC_STATIC_SCRATCH_BYTES is refused
+ *   with NGC_ERR_STATIC_SCRATCH before anything is enqueued (use the
+ *   workspace variant, or narrow the layer range).
+ * - The first call on each device looks up the device address of the array
+ *   (a one-off host-side set-up on the current device, serialised by a
+ *   mutex); make that first call before starting any stream capture.
+ * - All calls on a device share the one array, which keeps whatever the last
+ *   call left in it.  Nothing in it needs to start at zero (every slot is
+ *   written before it is read within a call), but two calls that overlap on
+ *   the GPU (different streams without an ordering between them) race on it:
+ *   keep calls to this entry stream-ordered.
+ */
+#define NGC_STATIC_SCRATCH_BYTES (8u << 20)
+int ngc_decode_attn_ragged_static(ngc_cache* c, const void* q, const void* new_k, const void* new_v,
+                                  int layer_begin, int layer_end, float scale,
+                                  void* out, int out_dtype, int32_t* dev_status, ngc_stream stream);
 
 #ifdef __cplusplus
 }

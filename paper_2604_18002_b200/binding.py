@@ -25,7 +25,9 @@ DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "
               5: "lists disagree", 6: "timeout"}
 
 EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
-           "ngc_sample_evict", "ngc_evict_logprob", "ngc_compact_kv", "ngc_decode_attn_ragged"]
+           "ngc_sample_evict", "ngc_evict_logprob", "ngc_compact_kv", "ngc_decode_attn_ragged",
+           "ngc_decode_attn_ragged_static"]
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class NgcError(RuntimeError):
@@ -64,6 +66,8 @@ def _load():
     lib.ngc_compact_kv.argtypes = [C.POINTER(CacheDesc), vp, vp, i32, i32, i32, vp, vp]
     lib.ngc_decode_attn_ragged.restype = i32
     lib.ngc_decode_attn_ragged.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, sz, vp, vp]
+    lib.ngc_decode_attn_ragged_static.restype = i32
+    lib.ngc_decode_attn_ragged_static.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, vp]
     return lib
 
 
@@ -222,3 +226,22 @@ def ngc_decode_attn_ragged(cache: NgcCache, q: torch.Tensor, out: torch.Tensor, 
                                     scale, _ptr(out), _dtype_code(out), _ptr(ws), 0 if ws is None else ws.numel(),
                                     _ptr(status), _stream())
     _check(rc, "ngc_decode_attn_ragged")
+
+
+def ngc_decode_attn_ragged_static(cache: NgcCache, q: torch.Tensor, out: torch.Tensor, new_k: Optional[torch.Tensor] = None,
+                                  new_v: Optional[torch.Tensor] = None, layer_begin: int = 0,
+                                  layer_end: Optional[int] = None, scale: Optional[float] = None,
+                                  status: Optional[torch.Tensor] = None):
+    """Decode attention for callers that cannot supply device scratch memory: the split partials
+    live in an array built into the library (``STATIC_SCRATCH_BYTES``), nothing is allocated.
+    Keep calls stream-ordered (they share the array); make the first call on a device outside
+    any stream capture (it looks the array's address up).  Raises when the launch would need
+    more scratch than the array holds."""
+    if layer_end is None:
+        layer_end = cache.L
+    if scale is None:
+        scale = 1.0 / (cache.d ** 0.5)
+    d = cache.desc(1 if new_k is not None else 0)
+    rc = lib.ngc_decode_attn_ragged_static(C.byref(d), _ptr(q), _ptr(new_k), _ptr(new_v), layer_begin, layer_end,
+                                           scale, _ptr(out), _dtype_code(out), _ptr(status), _stream())
+    _check(rc, "ngc_decode_attn_ragged_static")

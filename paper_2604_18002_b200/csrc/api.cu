@@ -17,6 +17,8 @@ const char* ngc_strerror(int status) {
     case NGC_ERR_UNSUPPORTED: return "shape or dtype not supported by this build";
     case NGC_ERR_WORKSPACE: return "workspace missing or too small";
     case NGC_ERR_CUDA: return "CUDA call failed (see ngc_last_cuda_error)";
+    case NGC_ERR_STATIC_SCRATCH:
+      return "launch needs more scratch than NGC_STATIC_SCRATCH_BYTES: use the workspace variant or a narrower layer range";
     default: return "unknown status";
   }
 }

@@ -601,3 +601,55 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
   }
   return rc;
 }
+
+// ---------------------------------------------------------------- allocation-free variant
+//
+// For callers that cannot provide device scratch (no allocator access, all
+// memory owned by a host framework's pool, or no tolerance for cudaMalloc's
+// device-wide synchronisation): the split partials go to an array that is
+// part of the library image.  In host code the array's name is only a
+// host-side stand-in, never a device address; the address is looked up once
+// per device with cudaGetSymbolAddress while that device is current.
+namespace ngc {
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_scratch[NGC_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_scratch_mutex;
+void* g_static_scratch_addr[kMaxDevices] = {nullptr};
+
+// Scratch bytes one call over `n_layers` layers uses (0 when it does not split).
+size_t decode_call_scratch_bytes(const ngc_cache* c, int n_layers) {
+  const int ns = decode_n_split(c, n_layers);
+  if (ns <= 1) return 0;
+  const size_t items = (size_t)n_layers * c->B * c->Hq * ns;
+  return align256(items * c->d * 4) + align256(items * 8);
+}
+
+}  // namespace
+}  // namespace ngc
+
+extern "C" int ngc_decode_attn_ragged_static(ngc_cache* c, const void* q, const void* new_k, const void* new_v,
+                                             int layer_begin, int layer_end, float scale,
+                                             void* out, int out_dtype, int32_t* dev_status, ngc_stream stream) {
+  using namespace ngc;
+  if (!valid_cache(c) || layer_begin < 0 || layer_end > c->L || layer_begin >= layer_end) return NGC_ERR_INVALID_ARG;
+  if (decode_call_scratch_bytes(c, layer_end - layer_begin) > (size_t)NGC_STATIC_SCRATCH_BYTES)
+    return NGC_ERR_STATIC_SCRATCH;
+  int dev = -1;
+  NGC_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return NGC_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_addr[dev]) {
+      void* p = nullptr;
+      NGC_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));   // device address on the current device
+      g_static_scratch_addr[dev] = p;
+    }
+    scratch = g_static_scratch_addr[dev];
+  }
+  return ngc_decode_attn_ragged(c, q, new_k, new_v, layer_begin, layer_end, scale, out, out_dtype,
+                                scratch, (size_t)NGC_STATIC_SCRATCH_BYTES, dev_status, stream);
+}
