@@ -154,12 +154,10 @@ def run_ngc(args):
         B = args.batch
     dtype = torch.bfloat16
     # every rank owns a full batch of B rollouts (weak scaling); Philox streams use global list ids
-    ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=T, n_max=T, k_max=K, lists=cfg["lists"], device=dev,
-                    list_base=rank * B, w=W_RECENT)
     seed = cfg["data_seed"] + 1000 * rank
     src = synth.make_cache(L, B, Hq, Hkv, d, dtype, [T] * B, capacity=T, seed=seed, outlier_channels=cfg["outliers"], device=dev)
-    ro.cache.k.copy_(src.k)
-    ro.cache.v.copy_(src.v)
+    ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=T, n_max=T, k_max=K, lists=cfg["lists"], device=dev,
+                    list_base=rank * B, w=W_RECENT, kv=(src.k, src.v))
     del src
     lens0 = torch.full((B,), T, dtype=torch.int32, device=dev)
     logits = synth.make_logits(B, 1, T, seed=seed + 7, std=cfg["logit_std"], device=dev)

@@ -19,7 +19,9 @@ from . import binding as ngc
 
 class NgcRollout:
     def __init__(self, L, B, Hq, Hkv, d, dtype, capacity, n_max, k_max, lists=ngc.LISTS_SHARED, block=1,
-                 w=5, device="cuda", list_base=0, with_score=True):
+                 w=5, device="cuda", list_base=0, with_score=True, kv=None):
+        """``kv``: optional (k, v) device tensors of shape [L][Hkv][sum(capacity)][d] to adopt
+        instead of allocating fresh ones."""
         self.L, self.B, self.Hq, self.Hkv, self.d = L, B, Hq, Hkv, d
         self.dtype, self.lists, self.block, self.w = dtype, lists, block, w
         self.device = device
@@ -29,9 +31,12 @@ class NgcRollout:
         seq_off = torch.zeros(B + 1, dtype=torch.int64)
         seq_off[1:] = torch.cumsum(cap, 0)
         R = int(seq_off[-1])
-        self.cache = ngc.NgcCache(
-            torch.empty((L, Hkv, R, d), dtype=dtype, device=device), torch.empty((L, Hkv, R, d), dtype=dtype, device=device),
-            seq_off.to(device), torch.zeros(B, dtype=torch.int32, device=device), Hq, int(cap.max()))
+        if kv is None:
+            kv = (torch.empty((L, Hkv, R, d), dtype=dtype, device=device),
+                  torch.empty((L, Hkv, R, d), dtype=dtype, device=device))
+        assert tuple(kv[0].shape) == (L, Hkv, R, d) and tuple(kv[1].shape) == (L, Hkv, R, d)
+        self.cache = ngc.NgcCache(kv[0], kv[1], seq_off.to(device), torch.zeros(B, dtype=torch.int32, device=device),
+                                  Hq, int(cap.max()))
         self.n_max, self.k_max = n_max, k_max
         self.logits = torch.empty((B, self.G, n_max), dtype=torch.float32, device=device)
         self.score_logits = torch.empty_like(self.logits) if with_score else None
