@@ -24,6 +24,7 @@
 
 #include <mutex>
 
+#include "kv_map.cuh"
 #include "ngc_common.cuh"
 #include "ngc_plan.h"
 #include "ptx.cuh"
@@ -469,35 +470,6 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 
 // ---------------------------------------------------------------- host side
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)sym;
-  });
-  return fn;
-}
-
-// K or V as a 3-D bf16 tensor (channel, row in plane, plane); box = 64 channels x 64 rows.
-bool make_kv_map(CUtensorMap* map, void* base, int64_t rows, int planes) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return false;
-  cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)planes};
-  cuuint64_t strides[2] = {256, (cuuint64_t)rows * 256};
-  cuuint32_t box[3] = {64, (cuuint32_t)kTileT, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 constexpr int kTargetCtas = 148 * 2 * 2;   // two waves of two CTAs per SM
 
 }  // namespace
@@ -567,7 +539,7 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
                            (((uintptr_t)c->k | (uintptr_t)c->v) & 15) == 0;
   if (stream_path) {
     CUtensorMap map_k, map_v;
-    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv) || !make_kv_map(&map_v, c->v, c->rows, c->L * c->Hkv))
+    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, kTileT) || !make_kv_map(&map_v, c->v, c->rows, c->L * c->Hkv, kTileT))
       return NGC_ERR_UNSUPPORTED;
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hkv * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;

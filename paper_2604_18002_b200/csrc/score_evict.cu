@@ -3,19 +3,29 @@
 // psi_t = mean over (query head, recent query) rows of softmax(q K^T / sqrt(d))_t,
 // s_j = mean of psi over the tokens of unit j.  The softmax of a row spans the
 // whole strip, so the work is split into three launches:
-//   1. per (strip, 256-token chunk): the row-wise max and sum of exponentials
-//      of the chunk's scores (a thread owns one token, the rows' queries sit in
-//      shared memory as fp32);
-//   2. same geometry: the chunk statistics of a row are merged, the scores are
-//      recomputed (K comes from L2 where it fits) and each token's probability
-//      summed over the rows of the strip is written out;
+//   1. per (strip, token range): the row-wise max and sum of exponentials of the
+//      range's scores;
+//   2. same geometry: the range statistics of a row are merged, the scores are
+//      recomputed and each token's probability summed over the rows of the
+//      strip is written out;
 //   3. per list: the strips feeding the list are added in a fixed order, the
 //      block mean is taken and the logit written.
 // No atomics on floating-point data: the result is reproducible run to run.
+//
+// Two device paths for launches 1 and 2:
+//  * bf16, d = 128, at most 40 rows per strip (group size x window): the strip
+//    is streamed once per launch through a TMA + mbarrier ring (64 tokens x 128
+//    channels per stage, 128-byte swizzle) and S = K Q^T runs on the tensor
+//    cores (mma.sync m16n8k16: 16 tokens on M, the strip's rows on N, their
+//    query fragments held in registers), so the launch stays HBM-bound.
+//  * everything else: a thread owns one token, the rows' queries sit in shared
+//    memory as fp32, plain FMA.
 #include <cuda_bf16.h>
 
+#include "kv_map.cuh"
 #include "ngc_common.cuh"
 #include "ngc_plan.h"
+#include "ptx.cuh"
 
 namespace ngc {
 namespace {
@@ -35,6 +45,7 @@ struct ScoreParams {
   int64_t rows_R;
   int L, B, Hq, Hkv, g, w, n_rows;   // n_rows = g * w rows per strip
   int n_chunks, block, lists, G, n_max, log_transform;
+  int n_split;       // token ranges per strip (streaming path)
   float inv_sqrt_d;
 };
 
@@ -174,6 +185,238 @@ __global__ void __launch_bounds__(kChunk) score_kernel(ScoreParams p) {
   if (PASS == 2 && active) p.psi[(int64_t)(l * p.Hkv + h) * p.rows_R + p.seq_off[b] + t] = mass;
 }
 
+// ---------------------------------------------------------------- streaming bf16 path
+
+constexpr int kSTileT = 64;                       // tokens per stage
+constexpr int kSConsumerWarps = 4;
+constexpr int kSThreads = (kSConsumerWarps + 1) * 32;
+constexpr int kSBoxBytes = kSTileT * 128;         // 64 tokens x 64 channels of bf16
+constexpr int kSStageBytes = 2 * kSBoxBytes;      // channels 0-63 and 64-127
+constexpr int kSStages = 4;
+constexpr int kSMaxRows = 40;                     // rows (columns of S) a strip may have on this path
+
+// (m, s) <- merge of two (max, sum of 2^(z - max)) pairs; either side may be empty (m = -inf).
+__device__ __forceinline__ void merge_ms(float& m, float& s, float mo, float so) {
+  const float mn = fmaxf(m, mo);
+  if (mn == -INFINITY) { s = 0.f; return; }
+  s = s * ptx::ex2_approx(m - mn) + so * ptx::ex2_approx(mo - mn);
+  m = mn;
+}
+
+// NT = number of 8-column tiles of S (ceil(rows / 8)).  PASS 1 writes the range
+// statistics, PASS 2 the per-token probability mass.  Scores are kept in the
+// log2 domain: z = (q.k) * scale * log2(e).
+template <int NT, int PASS>
+__global__ void __launch_bounds__(kSThreads, 2)
+score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, float scale_log2, int32_t* dev_status) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ uint64_t bar_full[kSStages], bar_empty[kSStages];
+  __shared__ float2 sm_ms[kSConsumerWarps][kSMaxRows];
+  __shared__ float sm_M[kSMaxRows], sm_inv[kSMaxRows];
+
+  uint8_t* stage_base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+
+  const int split = blockIdx.x % p.n_split;
+  const int strip = blockIdx.x / p.n_split;
+  const int h = strip % p.Hkv;
+  const int b = (strip / p.Hkv) % p.B;
+  const int l = strip / (p.Hkv * p.B);
+  const int T_b = p.lens[b];
+  const int n_rows = p.n_rows;
+  const int w_eff = min(p.w, T_b);
+
+  const int nt = (T_b + kSTileT - 1) / kSTileT;
+  const int tps = (nt + p.n_split - 1) / p.n_split;
+  const int tile_lo = min(nt, split * tps);
+  const int tile_hi = min(nt, tile_lo + tps);
+  const int n_tiles = tile_hi - tile_lo;
+
+  float2* st = p.stats + (int64_t)strip * p.n_split * kSMaxRows;
+
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < kSStages; ++s) { ptx::mbar_init(&bar_full[s], 1); ptx::mbar_init(&bar_empty[s], kSConsumerWarps); }
+    ptx::fence_barrier_init();
+  }
+  if (PASS == 2 && tid < kSMaxRows) {
+    float m = -INFINITY, sum = 0.f;
+    for (int c = 0; c < p.n_split; ++c) {
+      const float2 v = st[c * kSMaxRows + tid];
+      merge_ms(m, sum, v.x, v.y);
+    }
+    const bool live = tid < n_rows && sum > 0.f;
+    sm_M[tid] = live ? m : 0.f;
+    sm_inv[tid] = live ? 1.f / sum : 0.f;
+  }
+  __syncthreads();
+
+  if (warp == kSConsumerWarps) {
+    // ------------------------------------------------ producer
+    if (lane == 0 && n_tiles > 0) {
+      ptx::prefetch_tensormap(&map_k);
+      const int plane = l * p.Hkv + h;
+      const int row0 = (int)p.seq_off[b];
+      for (int it = 0; it < n_tiles; ++it) {
+        const int s = it % kSStages;
+        if (it >= kSStages) {
+          if (!ptx::mbar_wait_bounded(&bar_empty[s], ((it / kSStages) - 1) & 1)) set_dev_status(dev_status, NGC_DEV_TIMEOUT);
+        }
+        uint8_t* sp = stage_base + s * kSStageBytes;
+        ptx::mbar_expect_tx(&bar_full[s], kSStageBytes);
+        const int y = row0 + (tile_lo + it) * kSTileT;
+        ptx::tma_load_3d(sp, &map_k, 0, y, plane, &bar_full[s]);
+        ptx::tma_load_3d(sp + kSBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------ consumers
+    // B operand: Q^T, column n of an 8-wide tile = row 8*tile + n of the strip
+    // (row r = head-in-group r / w, window slot r % w); zero beyond n_rows.
+    uint32_t qb[NT][8][2];
+    int lim[NT][2];          // last visible token of the thread's columns (-1: column unused)
+#pragma unroll
+    for (int t8 = 0; t8 < NT; ++t8) {
+      const int r = 8 * t8 + gid;
+      const bool live = r < n_rows;
+      const int hl = live ? r / p.w : 0, j = live ? r - hl * p.w : 0;
+      const uint32_t* qrow = (const uint32_t*)((const __nv_bfloat16*)p.q_recent +
+                                               ((((int64_t)l * p.B + b) * p.Hq + h * p.g + hl) * p.w + j) * 128);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        qb[t8][ks][0] = live ? qrow[8 * ks + tig] : 0u;
+        qb[t8][ks][1] = live ? qrow[8 * ks + tig + 4] : 0u;
+      }
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int c = 8 * t8 + 2 * tig + e;
+        const int jc = c % p.w;
+        // window slot j sits at absolute position T_b - w + j; slots before the sequence start do not exist
+        lim[t8][e] = (c < n_rows && jc >= p.w - w_eff) ? T_b - p.w + jc : -1;
+      }
+    }
+    float m_run[NT][2], s_run[NT][2];      // PASS 1: running max (raw dot products) and sum
+    float negM[NT][2], inv[NT][2];         // PASS 2: -M (log2 domain) and 1 / row sum
+#pragma unroll
+    for (int t8 = 0; t8 < NT; ++t8)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        m_run[t8][e] = -INFINITY; s_run[t8][e] = 0.f;
+        if (PASS == 2) {
+          const int c = 8 * t8 + 2 * tig + e;
+          negM[t8][e] = -sm_M[c];
+          inv[t8][e] = sm_inv[c];
+        } else {
+          negM[t8][e] = 0.f; inv[t8][e] = 0.f;
+        }
+      }
+    const uint32_t a_lane_off = (uint32_t)((16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * 128);
+    const uint32_t x7 = (uint32_t)(lane & 7);
+    float* psi_strip = p.psi + (int64_t)(l * p.Hkv + h) * p.rows_R + p.seq_off[b];
+
+    for (int it = 0; it < n_tiles; ++it) {
+      const int s = it % kSStages;
+      if (!ptx::mbar_wait_bounded(&bar_full[s], (it / kSStages) & 1)) set_dev_status(dev_status, NGC_DEV_TIMEOUT);
+      const uint32_t k_st = ptx::smem_u32(stage_base + s * kSStageBytes);
+      const int t_base = (tile_lo + it) * kSTileT + 16 * warp;
+
+      if (t_base < T_b) {
+        float acc[NT][4];
+#pragma unroll
+        for (int t8 = 0; t8 < NT; ++t8) { acc[t8][0] = 0.f; acc[t8][1] = 0.f; acc[t8][2] = 0.f; acc[t8][3] = 0.f; }
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t chunk = (uint32_t)(2 * (ks & 3) + (lane >> 4));
+          const uint32_t addr = k_st + (ks >> 2) * kSBoxBytes + a_lane_off + ((chunk ^ x7) << 4);
+          uint32_t a[4];
+          ptx::ldmatrix_x4(addr, a[0], a[1], a[2], a[3]);
+#pragma unroll
+          for (int t8 = 0; t8 < NT; ++t8) ptx::mma_bf16_16816(acc[t8], a, qb[t8][ks][0], qb[t8][ks][1]);
+        }
+        const int t0 = t_base + gid, t1 = t0 + 8;
+        // tokens of this slice that some row cannot see: the window itself and the tail beyond T_b
+        const bool masked = t_base + 16 > T_b - p.w;
+        if (PASS == 1) {
+#pragma unroll
+          for (int t8 = 0; t8 < NT; ++t8)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              float a0 = acc[t8][e], a1 = acc[t8][e + 2];
+              if (masked) {
+                a0 = t0 <= lim[t8][e] ? a0 : -INFINITY;
+                a1 = t1 <= lim[t8][e] ? a1 : -INFINITY;
+              }
+              const float mx = fmaxf(fmaxf(m_run[t8][e], a0), a1);
+              const float ms = masked && mx == -INFINITY ? 0.f : mx;
+              const float neg = -ms * scale_log2;
+              const float e_old = ptx::ex2_approx(fmaf(m_run[t8][e], scale_log2, neg));
+              const float e0 = ptx::ex2_approx(fmaf(a0, scale_log2, neg));
+              const float e1 = ptx::ex2_approx(fmaf(a1, scale_log2, neg));
+              s_run[t8][e] = fmaf(s_run[t8][e], e_old, e0 + e1);
+              m_run[t8][e] = mx;
+            }
+        } else {
+          float p0 = 0.f, p1 = 0.f;
+#pragma unroll
+          for (int t8 = 0; t8 < NT; ++t8)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              float e0 = ptx::ex2_approx(fmaf(acc[t8][e], scale_log2, negM[t8][e]));
+              float e1 = ptx::ex2_approx(fmaf(acc[t8][e + 2], scale_log2, negM[t8][e]));
+              if (masked) {
+                e0 = t0 <= lim[t8][e] ? e0 : 0.f;
+                e1 = t1 <= lim[t8][e] ? e1 : 0.f;
+              }
+              p0 = fmaf(e0, inv[t8][e], p0);
+              p1 = fmaf(e1, inv[t8][e], p1);
+            }
+          p0 += __shfl_xor_sync(0xffffffffu, p0, 1);
+          p0 += __shfl_xor_sync(0xffffffffu, p0, 2);
+          p1 += __shfl_xor_sync(0xffffffffu, p1, 1);
+          p1 += __shfl_xor_sync(0xffffffffu, p1, 2);
+          if (tig == 0) {
+            if (t0 < T_b) psi_strip[t0] = p0;
+            if (t1 < T_b) psi_strip[t1] = p1;
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&bar_empty[s]);
+    }
+    if (PASS == 1) {
+      // columns are spread over the quad (tig), tokens over gid: merge over gid, then over warps
+#pragma unroll
+      for (int t8 = 0; t8 < NT; ++t8)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          float m = m_run[t8][e] * scale_log2, sum = s_run[t8][e];     // -inf stays -inf (scale > 0)
+#pragma unroll
+          for (int o = 4; o < 32; o <<= 1) {
+            const float mo = __shfl_xor_sync(0xffffffffu, m, o);
+            const float so = __shfl_xor_sync(0xffffffffu, sum, o);
+            merge_ms(m, sum, mo, so);
+          }
+          if (gid == 0) sm_ms[warp][8 * t8 + 2 * tig + e] = make_float2(m, sum);
+        }
+    }
+  }
+  if (PASS == 1) {
+    __syncthreads();
+    if (tid < kSMaxRows) {
+      float m = -INFINITY, sum = 0.f;
+      if (tid < 8 * NT) {
+#pragma unroll
+        for (int w2 = 0; w2 < kSConsumerWarps; ++w2) merge_ms(m, sum, sm_ms[w2][tid].x, sm_ms[w2][tid].y);
+      }
+      st[split * kSMaxRows + tid] = make_float2(m, sum);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- list reduction
+
 __global__ void __launch_bounds__(256) score_finish_kernel(ScoreParams p) {
   const int li = blockIdx.x;                    // b * G + gi
   const int b = li / p.G, gi = li - b * p.G;
@@ -199,9 +442,46 @@ __global__ void __launch_bounds__(256) score_finish_kernel(ScoreParams p) {
   p.logits[(int64_t)li * p.n_max + u] = p.log_transform ? logf(s) : s;
 }
 
+constexpr int kScoreTargetCtas = 148 * 2 * 2;   // two waves of two CTAs per SM
+
+bool score_stream_shape(const ngc_cache* c, int w) {
+  return c->dtype == NGC_BF16 && c->d == 128 && (c->Hq / c->Hkv) * w <= kSMaxRows && c->rows < 0x7fffffffLL;
+}
+
+// Token ranges per strip on the streaming path: enough CTAs to fill the GPU, at least 4 tiles each.
+int score_n_split(const ngc_cache* c) {
+  const int64_t strips = (int64_t)c->L * c->B * c->Hkv;
+  if (strips >= kScoreTargetCtas) return 1;
+  int ns = (int)((kScoreTargetCtas + strips - 1) / strips);
+  const int by_len = (c->max_len + 4 * kSTileT - 1) / (4 * kSTileT);
+  if (ns > by_len) ns = by_len;
+  if (ns > 64) ns = 64;
+  return ns < 1 ? 1 : ns;
+}
+
 size_t stats_bytes(const ngc_cache* c) {
   const int n_chunks = (c->max_len + kChunk - 1) / kChunk;
-  return align256((size_t)c->L * c->Hkv * c->B * (n_chunks > 0 ? n_chunks : 1) * (c->Hq / c->Hkv) * 16 /*w <= 16*/ * 8);
+  const size_t strips = (size_t)c->L * c->Hkv * c->B;
+  const size_t generic = strips * (n_chunks > 0 ? n_chunks : 1) * (c->Hq / c->Hkv) * 16 /*w <= 16*/ * 8;
+  const size_t stream = strips * score_n_split(c) * kSMaxRows * 8;
+  return align256(generic > stream ? generic : stream);
+}
+
+template <int NT>
+int launch_score_stream(const CUtensorMap& map_k, const ScoreParams& p, float scale_log2, int32_t* dev_status,
+                        unsigned grid, cudaStream_t stream) {
+  const int smem = kSStages * kSStageBytes + 1024;
+  static std::once_flag attr_once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(attr_once, [&] {
+    attr_err = cudaFuncSetAttribute(score_stream_kernel<NT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (attr_err == cudaSuccess)
+      attr_err = cudaFuncSetAttribute(score_stream_kernel<NT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  });
+  if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+  score_stream_kernel<NT, 1><<<grid, kSThreads, smem, stream>>>(map_k, p, scale_log2, dev_status);
+  score_stream_kernel<NT, 2><<<grid, kSThreads, smem, stream>>>(map_k, p, scale_log2, dev_status);
+  return launch_status();
 }
 
 }  // namespace
@@ -217,7 +497,6 @@ extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, 
                                int log_transform, float* logits, int n_max,
                                void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream_) {
   using namespace ngc;
-  (void)dev_status;
   cudaStream_t stream = (cudaStream_t)stream_;
   if (!valid_cache(c) || !q_recent || !logits || w <= 0 || w > 16 || block <= 0 || lists < 0 || lists > 2 || n_max <= 0)
     return NGC_ERR_INVALID_ARG;
@@ -239,10 +518,28 @@ extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, 
   p.log_transform = log_transform;
   p.inv_sqrt_d = 1.0f / sqrtf((float)c->d);
 
-  const int64_t ctas = (int64_t)c->L * c->B * c->Hkv * p.n_chunks;
-  if (ctas > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
-  const size_t smem = (size_t)p.n_rows * c->d * 4;
-  const unsigned grid = (unsigned)ctas;
+  p.n_split = 1;
+  int rc;
+  if (score_stream_shape(c, w) && ((uintptr_t)c->k & 15) == 0 && ((uintptr_t)q_recent & 3) == 0) {
+    p.n_split = score_n_split(c);
+    const int64_t ctas = (int64_t)c->L * c->B * c->Hkv * p.n_split;
+    if (ctas > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+    CUtensorMap map_k;
+    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, kSTileT)) return NGC_ERR_UNSUPPORTED;
+    const float scale_log2 = p.inv_sqrt_d * 1.4426950408889634f;
+    const unsigned grid = (unsigned)ctas;
+    switch ((p.n_rows + 7) / 8) {
+      case 1: rc = launch_score_stream<1>(map_k, p, scale_log2, dev_status, grid, stream); break;
+      case 2: rc = launch_score_stream<2>(map_k, p, scale_log2, dev_status, grid, stream); break;
+      case 3: rc = launch_score_stream<3>(map_k, p, scale_log2, dev_status, grid, stream); break;
+      case 4: rc = launch_score_stream<4>(map_k, p, scale_log2, dev_status, grid, stream); break;
+      default: rc = launch_score_stream<5>(map_k, p, scale_log2, dev_status, grid, stream); break;
+    }
+  } else {
+    const int64_t ctas = (int64_t)c->L * c->B * c->Hkv * p.n_chunks;
+    if (ctas > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)p.n_rows * c->d * 4;
+    const unsigned grid = (unsigned)ctas;
 
 #define NGC_SCORE_LAUNCH(T, D)                                                                                   \
   do {                                                                                                           \
@@ -254,12 +551,13 @@ extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, 
     score_kernel<T, D, 2><<<grid, kChunk, smem, stream>>>(p);                                                    \
   } while (0)
 
-  if (c->dtype == NGC_F32 && c->d == 64) NGC_SCORE_LAUNCH(float, 64);
-  else if (c->dtype == NGC_F32) NGC_SCORE_LAUNCH(float, 128);
-  else if (c->d == 64) NGC_SCORE_LAUNCH(__nv_bfloat16, 64);
-  else NGC_SCORE_LAUNCH(__nv_bfloat16, 128);
+    if (c->dtype == NGC_F32 && c->d == 64) NGC_SCORE_LAUNCH(float, 64);
+    else if (c->dtype == NGC_F32) NGC_SCORE_LAUNCH(float, 128);
+    else if (c->d == 64) NGC_SCORE_LAUNCH(__nv_bfloat16, 64);
+    else NGC_SCORE_LAUNCH(__nv_bfloat16, 128);
 #undef NGC_SCORE_LAUNCH
-  int rc = launch_status();
+    rc = launch_status();
+  }
   if (rc != NGC_OK) return rc;
   const int n_units_max = (c->max_len + block - 1) / block;
   dim3 fgrid(c->B * p.G, (n_units_max + 255) / 256);

@@ -360,3 +360,34 @@ def test_score_matches_oracle(dtype, d, Hq, Hkv, lists, block):
     torch.cuda.synchronize()
     got_log = logits.cpu().numpy().astype(np.float64)
     assert np.allclose(got_log[live], np.log(got[live]), atol=1e-5)
+
+
+@pytest.mark.parametrize("Hq,Hkv,w,lens", [(12, 2, 1, [1, 63, 64, 2000]), (12, 2, 3, [2, 65, 128, 1500]), (28, 4, 5, [4, 5, 6, 3000]),
+                                            (8, 1, 5, [700, 64, 1, 129]), (16, 2, 7, [900, 10, 3, 300]), (4, 4, 6, [5, 6, 7, 2100])])
+def test_score_window_sizes_and_ragged_lengths(Hq, Hkv, w, lens):
+    """bf16, d = 128: the tensor-core path (rows per strip <= 40) and the plain path (more rows), windows
+    shorter and longer than the sequence, lengths on and off the 64-token tile boundary, several
+    token ranges per strip."""
+    L, B, d, dtype = 2, 4, 128, torch.bfloat16
+    cap = max(lens) + 3
+    c = synth.make_cache(L, B, Hq, Hkv, d, dtype, lens, capacity=cap, seed=77, outlier_channels=4)
+    qr = synth.normal((L, B, Hq, w, d), 78, dtype)
+    b = ngc()
+    for lists in (1, 2):
+        ref = oracle.score_evict(synth.to_numpy(c.k), c.seq_off.numpy(), c.lens.numpy(), synth.to_numpy(qr), 1, lists, n_max=cap)
+        dc = to_device_cache(c, cap)
+        G = oracle.lists_G(lists, L, Hkv)
+        logits = torch.full((B, G, cap), -5.0, dtype=torch.float32, device="cuda")
+        ws = b.alloc_workspace(b.workspace_bytes(b.OP_SCORE, dc, G, cap))
+        st = b.new_status()
+        b.ngc_score_evict(dc, qr.cuda(), 1, lists, logits, ws=ws, status=st)
+        torch.cuda.synchronize()
+        assert status_value(st) == 0
+        got = logits.cpu().numpy().astype(np.float64)
+        live = ~np.isnan(ref)
+        assert np.all(got[~live] == -5.0)
+        for bb in range(B):
+            for g in range(G):
+                m = live[bb, g]
+                assert np.max(np.abs(got[bb, g][m] - ref[bb, g][m])) <= 2e-2 * ref[bb, g][m].max()
+                assert abs(got[bb, g][m].sum() - 1.0) <= 1e-3          # psi is a mean of probability rows
