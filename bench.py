@@ -174,16 +174,15 @@ def run_ngc(args):
     def one_step(step_idx, time_decode=False):
         ro.cache.lens.copy_(lens0, non_blocking=True)
         ro.eviction_round(n_t, None, k_t, noise_seed, step_idx, q_recent=q_recent, logits=logits)
+        if time_decode:       # one event pair around the step's decode calls (none between them)
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
         for s in range(steps):
-            if time_decode:
-                e0 = torch.cuda.Event(enable_timing=True)
-                e1 = torch.cuda.Event(enable_timing=True)
-                e0.record()
-                ro.decode_step(q[s], out[s], nk[s], nv[s])
-                e1.record()
-                ev_pairs.append((e0, e1))
-            else:
-                ro.decode_step(q[s], out[s], nk[s], nv[s])
+            ro.decode_step(q[s], out[s], nk[s], nv[s])
+        if time_decode:
+            e1.record()
+            ev_pairs.append((e0, e1))
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -215,13 +214,13 @@ def run_ngc(args):
     value = tokens / (ms_per_step * 1e-3)
 
     # roofline of the dominant kernel (decode): algorithmic K/V bytes per launch / mean launch time
-    dec_ms = [a.elapsed_time(b) for a, b in ev_pairs]
-    mean_dec_ms = float(np.mean(dec_ms))
+    dec_ms = [a.elapsed_time(b) for a, b in ev_pairs]          # per step: all decode calls of the step
+    mean_dec_ms = float(np.sum(dec_ms)) / (len(dec_ms) * steps)   # average duration of one decode call
     visible_total = sum(B * (K + s + 1) for s in range(steps)) / steps      # per launch, averaged over the step
     bytes_per_launch = algorithmic_decode_bytes(cfg, visible_total)
     peak, peak_kind = peaks()
     achieved = bytes_per_launch / (mean_dec_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (per ngc_decode_attn_ragged call: append + attention + lens bump)",
+    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (time per ngc_decode_attn_ragged call: attention with fused append + lens bump, launch gaps included)",
                 "achieved": round(achieved, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": round(achieved / peak, 4),
                 "traffic": int(args.traffic if args.traffic else NCU_TRAFFIC_RATIO * bytes_per_launch),

@@ -16,9 +16,14 @@
 //    CTA, a warp per token row, fp32 FMA and warp-shuffle reductions.
 //
 // With n_split > 1 each item writes an unnormalised partial (m, l, o) and a
-// small combine kernel merges the splits.  The new token's K/V row is written
-// by a tiny kernel in front (same call, same stream); lens[] is bumped by a
-// kernel behind.  No kernel here ever waits on another CTA.
+// small combine kernel merges the splits.  The new token's K/V row is handled
+// inside the attention kernel: the CTA whose token range ends the strip takes
+// the row from the caller's buffer (patching it into its shared-memory tile on
+// the streaming path) and stores it into the cache for later steps, so no CTA
+// ever reads that cache row during the call.  lens[] is bumped by a one-CTA
+// kernel behind.  The kernels of a call, and consecutive calls on a stream,
+// are chained by programmatic dependent launch, so each one's prologue
+// overlaps its predecessor's tail.  No kernel here ever waits on another CTA.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -58,28 +63,11 @@ __device__ __forceinline__ int visible_len(const DecodeParams& p, int b) {
   return (len + 1 > cap) ? -1 : len + 1;
 }
 
-// ---------------------------------------------------------------- append
-
-__global__ void append_kernel(DecodeParams p, int row_vecs) {
-  int s = blockIdx.x;
-  const int h = s % p.Hkv; s /= p.Hkv;
-  const int b = s % p.B;
-  const int l = p.layer_begin + s / p.B;
-  const int len = p.lens[b];
-  const int64_t cap = p.seq_off[b + 1] - p.seq_off[b];
-  if (len + 1 > cap) {
-    if (threadIdx.x == 0) set_dev_status(p.dev_status, NGC_DEV_STRIP_FULL);
-    return;
-  }
-  const int t = threadIdx.x;
-  const int which = t >> 5, vec = t & 31;
-  if (vec >= row_vecs) return;
-  const uint4* src = (const uint4*)(which ? p.new_v : p.new_k) + (((int64_t)l * p.B + b) * p.Hkv + h) * row_vecs;
-  uint4* dst = (uint4*)(which ? p.v : p.k) + (((int64_t)(l * p.Hkv + h) * p.rows) + p.seq_off[b] + len) * row_vecs;
-  dst[vec] = src[vec];
-}
+// ---------------------------------------------------------------- lens bump
 
 __global__ void bump_lens_kernel(DecodeParams p) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();          // every CTA of the attention (and combine) kernel has read lens
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= p.B) return;
   const int len = p.lens[b];
@@ -140,8 +128,14 @@ __global__ void __launch_bounds__(kGenWarps * 32) decode_generic_kernel(DecodePa
   const int h = hq / p.g;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+  ptx::grid_dep_wait();
+  ptx::grid_dep_launch();
   int len = visible_len(p, b);
-  if (len < 0) len = 0;
+  if (len < 0) {
+    if (tid == 0) set_dev_status(p.dev_status, NGC_DEV_STRIP_FULL);
+    len = 0;
+  }
+  const int t_new = (p.append && len > 0) ? len - 1 : -1;      // position of the appended row
   const int nt = (len + kGenChunk - 1) / kGenChunk;
   const int tps = (nt + p.n_split - 1) / p.n_split;
   const int t_begin = min(len, split * tps * kGenChunk);
@@ -150,16 +144,19 @@ __global__ void __launch_bounds__(kGenWarps * 32) decode_generic_kernel(DecodePa
   const int64_t qo = (((int64_t)l * p.B + b) * p.Hq + hq) * D;
   float qv[VPL];
   RowLoad<T>::template load<VPL>((const T*)p.q + qo, lane, qv);
-  const T* kbase = (const T*)p.k + ((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b]) * D;
-  const T* vbase = (const T*)p.v + ((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b]) * D;
+  T* kbase = (T*)p.k + ((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b]) * D;
+  T* vbase = (T*)p.v + ((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b]) * D;
+  const T* knew = (const T*)p.new_k + (((int64_t)l * p.B + b) * p.Hkv + h) * D;
+  const T* vnew = (const T*)p.new_v + (((int64_t)l * p.B + b) * p.Hkv + h) * D;
 
   float m = -INFINITY, lsum = 0.f, acc[VPL];
 #pragma unroll
   for (int i = 0; i < VPL; ++i) acc[i] = 0.f;
   for (int t = t_begin + warp; t < t_end; t += kGenWarps) {
     float kx[VPL], vx[VPL];
-    RowLoad<T>::template load<VPL>(kbase + (int64_t)t * D, lane, kx);
-    RowLoad<T>::template load<VPL>(vbase + (int64_t)t * D, lane, vx);
+    // the appended row is taken from the caller's buffer: its cache row is written during this launch
+    RowLoad<T>::template load<VPL>(t == t_new ? knew : kbase + (int64_t)t * D, lane, kx);
+    RowLoad<T>::template load<VPL>(t == t_new ? vnew : vbase + (int64_t)t * D, lane, vx);
     float dot = 0.f;
 #pragma unroll
     for (int i = 0; i < VPL; ++i) dot = fmaf(qv[i], kx[i], dot);
@@ -172,6 +169,13 @@ __global__ void __launch_bounds__(kGenWarps * 32) decode_generic_kernel(DecodePa
 #pragma unroll
     for (int i = 0; i < VPL; ++i) acc[i] = fmaf(pz, vx[i], acc[i] * alpha);
     m = m_new;
+  }
+  // one CTA per KV head stores the appended row for the following steps
+  if (t_new >= t_begin && t_new < t_end && hq == h * p.g && warp < 2) {
+    const T* src = warp ? vnew : knew;
+    T* dst = (warp ? vbase : kbase) + (int64_t)t_new * D;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) dst[lane * VPL + i] = src[lane * VPL + i];
   }
   if (lane == 0) { sm_m[warp] = m; sm_l[warp] = lsum; }
 #pragma unroll
@@ -201,6 +205,8 @@ __global__ void __launch_bounds__(kGenWarps * 32) decode_generic_kernel(DecodePa
 // ---------------------------------------------------------------- split combine
 
 __global__ void combine_kernel(DecodeParams p) {
+  ptx::grid_dep_wait();
+  ptx::grid_dep_launch();
   const int64_t it = blockIdx.x;               // (lr, b, hq)
   const int c = threadIdx.x;                   // channel
   const int lr = (int)(it / ((int64_t)p.B * p.Hq));
@@ -247,19 +253,27 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
   const int l = p.layer_begin + lr;
   const int g = p.g;
 
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&bar_full[s], 1); ptx::mbar_init(&bar_empty[s], kConsumerWarps); }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&map_k);
+    ptx::prefetch_tensormap(&map_v);
+  }
+  ptx::grid_dep_wait();           // lens and the cache rows of earlier calls are final from here on
+  ptx::grid_dep_launch();
+
   int len = visible_len(p, b);
-  if (len < 0) len = 0;
+  if (len < 0) {
+    if (tid == 0) set_dev_status(p.dev_status, NGC_DEV_STRIP_FULL);
+    len = 0;
+  }
+  const int t_new = (p.append && len > 0) ? len - 1 : -1;      // position of the appended row
   const int nt = (len + kTileT - 1) / kTileT;
   const int tps = (nt + p.n_split - 1) / p.n_split;
   const int tile_lo = min(nt, split * tps);
   const int tile_hi = min(nt, tile_lo + tps);
   const int n_tiles = tile_hi - tile_lo;
-
-  if (tid == 0) {
-#pragma unroll
-    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&bar_full[s], 1); ptx::mbar_init(&bar_empty[s], kConsumerWarps); }
-    ptx::fence_barrier_init();
-  }
   __syncthreads();
 
   float o_acc[16][4];
@@ -271,8 +285,6 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
   if (warp == kConsumerWarps) {
     // ------------------------------------------------ producer
     if (lane == 0 && n_tiles > 0) {
-      ptx::prefetch_tensormap(&map_k);
-      ptx::prefetch_tensormap(&map_v);
       const int plane = l * p.Hkv + h;
       const int row0 = (int)p.seq_off[b];
       for (int it = 0; it < n_tiles; ++it) {
@@ -321,6 +333,18 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
       const int tile_t0 = (tile_lo + it) * kTileT;
       const int valid = len - tile_t0 - 16 * warp;      // live tokens in this warp's slice (may exceed 16)
 
+      if (t_new >= tile_t0 + 16 * warp && t_new < tile_t0 + 16 * warp + 16) {
+        // The appended row lives in this warp's slice: take it from the caller's buffer (the tile
+        // holds whatever the cache row held before) and store it into the cache for later steps.
+        // Lanes 0-15 move the sixteen 16-byte pieces of the K row, lanes 16-31 those of the V row.
+        const int isv = lane >> 4, c = lane & 15, r = t_new - tile_t0;
+        const uint4 piece = ((const uint4*)(isv ? p.new_v : p.new_k))[(((int64_t)l * p.B + b) * p.Hkv + h) * 16 + c];
+        uint8_t* dst = st + isv * kTileBytes + (c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(dst) = piece;
+        ((uint4*)(isv ? p.v : p.k))[((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b] + t_new) * 16 + c] = piece;
+        ptx::fence_proxy_async();      // the stage is refilled by TMA later: order this generic write before it
+        __syncwarp();
+      }
       if (valid > 0) {
         if (valid < 16) {
           // dead V rows may hold anything (NaN x 0 would poison the sum): zero them
@@ -507,6 +531,8 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
   if (!valid_cache(c) || !q || !out || layer_begin < 0 || layer_end > c->L || layer_begin >= layer_end)
     return NGC_ERR_INVALID_ARG;
   if ((new_k == nullptr) != (new_v == nullptr)) return NGC_ERR_INVALID_ARG;
+  if ((((uintptr_t)q | (uintptr_t)new_k | (uintptr_t)new_v | (uintptr_t)out | (uintptr_t)c->k | (uintptr_t)c->v) & 15) != 0)
+    return NGC_ERR_INVALID_ARG;      // rows are moved as 16-byte vectors
   if (out_dtype != NGC_F32 && !(out_dtype == NGC_BF16 && c->dtype == NGC_BF16)) return NGC_ERR_INVALID_ARG;
   if (c->rows == 0) return NGC_OK;
 
@@ -528,15 +554,7 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
     p.part_ml = (float2*)((char*)ws + align256(items * c->d * 4));
   }
 
-  const int row_vecs = c->d * elt_bytes(c->dtype) / 16;
-  if (p.append) {
-    append_kernel<<<(unsigned)(p.n_layers * c->B * c->Hkv), 64, 0, stream>>>(p, row_vecs);
-    int rc = launch_status();
-    if (rc != NGC_OK) return rc;
-  }
-
-  const bool stream_path = c->dtype == NGC_BF16 && c->d == 128 && p.g <= 16 && c->rows < 0x7fffffffLL &&
-                           (((uintptr_t)c->k | (uintptr_t)c->v) & 15) == 0;
+  const bool stream_path = c->dtype == NGC_BF16 && c->d == 128 && p.g <= 16 && c->rows < 0x7fffffffLL;
   if (stream_path) {
     CUtensorMap map_k, map_v;
     if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, kTileT) || !make_kv_map(&map_v, c->v, c->rows, c->L * c->Hkv, kTileT))
@@ -550,28 +568,22 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
       attr_err = cudaFuncSetAttribute(decode_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
-    decode_stream_kernel<<<(unsigned)items, kStreamThreads, smem, stream>>>(map_k, map_v, p);
+    NGC_CUDA_TRY(launch_pdl(decode_stream_kernel, dim3((unsigned)items), dim3(kStreamThreads), smem, stream, map_k, map_v, p));
   } else {
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hq * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
     const unsigned grid = (unsigned)items;
-    if (c->dtype == NGC_F32 && c->d == 64) decode_generic_kernel<float, 64><<<grid, kGenWarps * 32, 0, stream>>>(p);
-    else if (c->dtype == NGC_F32) decode_generic_kernel<float, 128><<<grid, kGenWarps * 32, 0, stream>>>(p);
-    else if (c->d == 64) decode_generic_kernel<__nv_bfloat16, 64><<<grid, kGenWarps * 32, 0, stream>>>(p);
-    else decode_generic_kernel<__nv_bfloat16, 128><<<grid, kGenWarps * 32, 0, stream>>>(p);
+    const dim3 blk(kGenWarps * 32);
+    if (c->dtype == NGC_F32 && c->d == 64) NGC_CUDA_TRY(launch_pdl(decode_generic_kernel<float, 64>, dim3(grid), blk, 0, stream, p));
+    else if (c->dtype == NGC_F32) NGC_CUDA_TRY(launch_pdl(decode_generic_kernel<float, 128>, dim3(grid), blk, 0, stream, p));
+    else if (c->d == 64) NGC_CUDA_TRY(launch_pdl(decode_generic_kernel<__nv_bfloat16, 64>, dim3(grid), blk, 0, stream, p));
+    else NGC_CUDA_TRY(launch_pdl(decode_generic_kernel<__nv_bfloat16, 128>, dim3(grid), blk, 0, stream, p));
   }
-  int rc = launch_status();
-  if (rc != NGC_OK) return rc;
-  if (p.n_split > 1) {
-    combine_kernel<<<(unsigned)(p.n_layers * c->B * c->Hq), c->d, 0, stream>>>(p);
-    rc = launch_status();
-    if (rc != NGC_OK) return rc;
-  }
-  if (p.append && layer_end == c->L) {
-    bump_lens_kernel<<<(c->B + 255) / 256, 256, 0, stream>>>(p);
-    rc = launch_status();
-  }
-  return rc;
+  if (p.n_split > 1)
+    NGC_CUDA_TRY(launch_pdl(combine_kernel, dim3((unsigned)(p.n_layers * c->B * c->Hq)), dim3(c->d), 0, stream, p));
+  if (p.append && layer_end == c->L)
+    NGC_CUDA_TRY(launch_pdl(bump_lens_kernel, dim3((c->B + 255) / 256), dim3(256), 0, stream, p));
+  return NGC_OK;
 }
 
 // ---------------------------------------------------------------- allocation-free variant

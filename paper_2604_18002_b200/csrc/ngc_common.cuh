@@ -46,6 +46,25 @@ inline bool valid_cache(const ngc_cache* c) {
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 #ifdef __CUDACC__
+// Launch with programmatic stream serialisation: the kernel may begin while
+// the previous kernel of the stream drains, and waits for it on the device
+// (ptx::grid_dep_wait) before touching dependent memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // First error wins.
 __device__ __forceinline__ void set_dev_status(int32_t* st, int code) {
   if (st) atomicCAS(st, 0, code);

@@ -72,7 +72,7 @@ class NgcRollout:
                     new_v: Optional[torch.Tensor] = None):
         ngc.ngc_decode_attn_ragged(self.cache, q, out, new_k, new_v, ws=self.ws_decode, status=self.status)
         split = ngc.decode_splits(self.cache, append=new_k is not None) > 1
-        self.launches += 1 + (2 if new_k is not None else 0) + (1 if split else 0)
+        self.launches += 1 + (1 if new_k is not None else 0) + (1 if split else 0)
 
     def check_status(self):
         code = int(self.status.item())
