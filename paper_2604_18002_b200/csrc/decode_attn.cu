@@ -324,6 +324,14 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     const uint32_t v_lane_off = (uint32_t)((16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * 128);
     const uint32_t x7 = (uint32_t)(lane & 7);
 
+    // The appended row sits in the strip's last tile.  The warp whose slice holds it fetches the row
+    // from the caller's buffer now, long before the tile arrives: lanes 0-15 take the sixteen
+    // 16-byte pieces of the K row, lanes 16-31 those of the V row.
+    const bool own_new = t_new >= 0 && tile_hi == nt && n_tiles > 0 && ((t_new % kTileT) >> 4) == warp;
+    uint4 piece = make_uint4(0, 0, 0, 0);
+    if (own_new)
+      piece = ((const uint4*)((lane >> 4) ? p.new_v : p.new_k))[(((int64_t)l * p.B + b) * p.Hkv + h) * 16 + (lane & 15)];
+
     for (int it = 0; it < n_tiles; ++it) {
       const int s = it % kStages;
       if (!ptx::mbar_wait_bounded(&bar_full[s], (it / kStages) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
@@ -333,12 +341,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
       const int tile_t0 = (tile_lo + it) * kTileT;
       const int valid = len - tile_t0 - 16 * warp;      // live tokens in this warp's slice (may exceed 16)
 
-      if (t_new >= tile_t0 + 16 * warp && t_new < tile_t0 + 16 * warp + 16) {
+      if (own_new && it == n_tiles - 1) {
         // The appended row lives in this warp's slice: take it from the caller's buffer (the tile
         // holds whatever the cache row held before) and store it into the cache for later steps.
-        // Lanes 0-15 move the sixteen 16-byte pieces of the K row, lanes 16-31 those of the V row.
         const int isv = lane >> 4, c = lane & 15, r = t_new - tile_t0;
-        const uint4 piece = ((const uint4*)(isv ? p.new_v : p.new_k))[(((int64_t)l * p.B + b) * p.Hkv + h) * 16 + c];
         uint8_t* dst = st + isv * kTileBytes + (c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
         *reinterpret_cast<uint4*>(dst) = piece;
         ((uint4*)(isv ? p.v : p.k))[((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b] + t_new) * 16 + c] = piece;
