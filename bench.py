@@ -37,6 +37,13 @@ from paper_2604_18002_b200 import synth
 
 CFG = dict(synth.CONFIGS[2])
 WORKLOAD = "config2: 1.5B-shaped GQA rollout step (L28, 12q/2kv, d128, bf16, B64, 4096->2048 tokens, 256 decode steps)"
+# the other workloads (--config 3|4|5) are measurement aids; the default line is always config 2
+OTHER_WORKLOADS = {
+    3: "config3: 7B-shaped ragged batch (L28, 28q/4kv, d128, bf16, B256, lengths 1024..8192 -> ceil(len/3), 128 decode steps)",
+    4: "config4: per-(layer, KV head) eviction (L28, 12q/2kv, d128, bf16, B128, 16384 -> 8192 tokens, 7168 lists, 64 decode steps)",
+    5: "config5: rollout loop (L28, 12q/2kv, d128, bf16, B64, 256 prompt + 8192 generated, a round every 512 tokens 768 -> 256, "
+       "per-layer lists) + log-prob recompute of all 16 rounds",
+}
 METRIC = "evict+compact+decode tokens/sec at B=64"
 W_RECENT = 5
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic K/V bytes for decode_stream_kernel, from the ncu
@@ -288,6 +295,159 @@ def run_ngc(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------ other workloads (measurement aid)
+
+def run_other(args):
+    """Configs 3, 4 and 5 on one GPU: the same hot path, timed per phase.  Decode inputs come from a ring of
+    `ring` distinct steps (the full set would not fit beside the 60+ GB caches); outputs of a step overwrite the ring slot."""
+    from paper_2604_18002_b200 import binding as ngc
+    from paper_2604_18002_b200.rollout import NgcRollout
+
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    cid = args.config
+    cfg = synth.CONFIGS[cid]
+    L, B, Hq, Hkv, d, steps = cfg["L"], args.batch or cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["d"], args.decode_steps or cfg["steps"]
+    dtype = torch.bfloat16
+    lists = cfg["lists"]
+    if cid == 5:
+        prompt, cadence, K = cfg["T"], cfg["cadence"], cfg["budget"]
+        rounds = max(1, steps // cadence)
+        steps = rounds * cadence
+        lens = torch.full((B,), prompt, dtype=torch.int32)
+        budget = torch.full((B,), K, dtype=torch.int32)
+        cap = torch.full((B,), prompt + cadence, dtype=torch.int64)
+        n_evict = torch.full((B,), prompt + cadence, dtype=torch.int32)
+    else:
+        if isinstance(cfg["T"], tuple):
+            lens = synth.ragged_lens(B, cfg["T"][0], cfg["T"][1], cfg["len_seed"])
+        else:
+            lens = torch.full((B,), cfg["T"], dtype=torch.int32)
+        budget = torch.ceil(lens.double() / 3).to(torch.int32) if cfg["budget"] == "third" else torch.full((B,), cfg["budget"], dtype=torch.int32)
+        cap = torch.maximum(lens.long(), budget.long() + steps)
+        n_evict = lens
+    n_max, k_max = int(n_evict.max()), int(budget.max())
+    src = synth.make_cache(L, B, Hq, Hkv, d, dtype, lens, capacity=cap, seed=cfg["data_seed"], outlier_channels=cfg["outliers"], device=dev)
+    ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=cap, n_max=n_max, k_max=k_max, lists=lists, device=dev, w=W_RECENT, kv=(src.k, src.v))
+    del src
+    G = ro.G
+    lens0 = lens.to(dev)
+    logits = synth.make_logits(B, G, n_max, seed=cfg["data_seed"] + 7, std=cfg["logit_std"], device=dev)
+    n_t, k_t = n_evict.to(dev), budget.to(dev)
+    ring = min(steps, args.ring)
+    q = synth.make_queries(L, B, Hq, d, dtype, seed=11, steps=ring, device=dev)
+    nk, nv = synth.make_new_kv(L, B, Hkv, d, dtype, seed=13, steps=ring, device=dev)
+    q_recent = synth.normal((L, B, Hq, W_RECENT, d), 17, dtype, device=dev)
+    out = torch.empty((ring, L, B, Hq, d), dtype=torch.float32, device=dev)
+    row_bytes = L * Hkv * 2 * d * 2
+    names = ["score", "sample", "logprob", "compact", "decode", "recompute"]
+    acc = {n: [] for n in names}
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def eviction(rnd, t):
+        e = [ev() for _ in range(5)]
+        e[0].record()
+        ngc.ngc_score_evict(ro.cache, q_recent, ro.block, lists, ro.score_logits, ws=ro.ws_score, status=ro.status)
+        e[1].record()
+        ngc.ngc_sample_evict(logits, n_t, None, k_t, cfg["noise_seed"], rnd, ro.kept_order, ro.kept_sorted, None, ws=ro.ws_sample, status=ro.status)
+        e[2].record()
+        ngc.ngc_evict_logprob(logits, n_t, None, k_t, ro.kept_order, ro.logp, status=ro.status)
+        e[3].record()
+        ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, lists, 1, status=ro.status)
+        e[4].record()
+        ro.launches += 7          # score 3, sample 1, log-prob 1, compaction 2
+        t.append(e)
+
+    def decode(n, t):
+        e0, e1 = ev(), ev()
+        e0.record()
+        for s in range(n):
+            ro.decode_step(q[s % ring], out[s % ring], nk[s % ring], nv[s % ring])
+        e1.record()
+        t.append((e0, e1))
+
+    if cid == 5:
+        all_logits = logits.unsqueeze(0).expand(rounds, B, G, n_max).contiguous()
+        all_ko = torch.zeros((rounds, B, G, k_max), dtype=torch.int32, device=dev)
+        all_lp = torch.empty((rounds, B, G), dtype=torch.float64, device=dev)
+        n_all, k_all = n_t.unsqueeze(0).expand(rounds, B).contiguous(), k_t.unsqueeze(0).expand(rounds, B).contiguous()
+
+    def one_step(i, rec):
+        ro.cache.lens.copy_(lens0, non_blocking=True)
+        ev_t, dec_t, rc = [], [], None
+        if cid == 5:
+            for r in range(rounds):
+                decode(cadence, dec_t)
+                eviction(i * rounds + r, ev_t)
+                all_ko[r].copy_(ro.kept_order, non_blocking=True)
+            rc = (ev(), ev())
+            rc[0].record()
+            ngc.ngc_evict_logprob(all_logits, n_all, None, k_all, all_ko, all_lp, status=ro.status)
+            rc[1].record()
+            ro.launches += 1
+        else:
+            eviction(i, ev_t)
+            decode(steps, dec_t)
+        rec.append((ev_t, dec_t, rc))
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    for w in range(args.warmup):
+        one_step(w, [])
+    torch.cuda.synchronize()
+    ro.check_status()
+    rec = []
+    launches0 = ro.launches
+    t0, t1 = ev(), ev()
+    wall0 = time.perf_counter()
+    t0.record()
+    for k in range(args.steps):
+        one_step(args.warmup + k, rec)
+    t1.record()
+    torch.cuda.synchronize()
+    wall1 = time.perf_counter()
+    clocks = sampler.stop(wall0, wall1)
+    ro.check_status()
+    ms_per_step = t0.elapsed_time(t1) / args.steps
+    for ev_t, dec_t, rc in rec:
+        for e in ev_t:
+            for i, n in enumerate(names[:4]):
+                acc[n].append(e[i].elapsed_time(e[i + 1]))
+        acc["decode"].append(sum(a.elapsed_time(b) for a, b in dec_t))
+        if rc:
+            acc["recompute"].append(rc[0].elapsed_time(rc[1]))
+    tokens = B * steps
+    # algorithmic K/V bytes: every visible token of every decode launch; every kept row read + written by compaction
+    kept = float(budget.sum())
+    if cid == 5:
+        vis = B * rounds * sum(prompt + s + 1 for s in range(cadence))
+        score_bytes = float(n_evict.sum()) * row_bytes / 2
+    else:
+        vis = sum(kept + B * (s + 1) for s in range(steps))
+        score_bytes = float(lens.sum()) * row_bytes / 2
+    compact_bytes = 2 * kept * row_bytes
+    dec_ms = float(np.mean(acc["decode"]))
+    peak, peak_kind = peaks()
+    med = {n: round(float(np.median(v)), 4) for n, v in acc.items() if v}
+    dec_gbs = vis * row_bytes / (dec_ms * 1e-3) / 1e9
+    cmp_gbs = compact_bytes / (med["compact"] * 1e-3) / 1e9
+    result = {"metric": "evict+compact+decode tokens/sec", "value": round(tokens / (ms_per_step * 1e-3), 1), "unit": "tokens/s", "n_gpus": 1,
+              "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "dtype": "bf16", "data": "synthetic",
+              "config": {"workload": OTHER_WORKLOADS[cid], "batch": B, "decode_steps": steps, "input_ring": ring},
+              "per_call_ms": med,
+              "roofline": {"bound": "hbm", "kernel": "decode_stream_kernel (all decode calls of a step, launch gaps included)",
+                           "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                           "frac": round(dec_gbs / peak, 4), "decode_ms_per_step": round(dec_ms, 3), "decode_calls": steps, "traffic": None},
+              "compact": {"bytes": int(compact_bytes), "GB/s": round(cmp_gbs, 1), "frac_of_peak": round(cmp_gbs / peak, 4),
+                          "note": "algorithmic bytes = every kept row read once and written once (rows already in place are skipped by the kernel)"},
+              "score": {"bytes": int(score_bytes), "GB/s": round(score_bytes / (med["score"] * 1e-3) / 1e9, 1),
+                        "note": "algorithmic bytes = K read once; the kernel streams K twice"},
+              "gpu_launches": int(ro.launches - launches0), "clocks": clocks}
+    print(json.dumps(result), flush=True)
+
+
 # ------------------------------------------------------------------------------------ CPU oracle arm
 
 def oracle_step(cache_np, logits, q, nk, nv, qr, K, rnd, decode_steps, seed):
@@ -368,6 +528,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seqs", type=int, default=4)
     ap.add_argument("--cpu-decode-steps", type=int, default=48)
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5],
+                    help="2 = the benchmark workload (default); 3, 4, 5 = the other workloads, one GPU, per-phase timing only")
+    ap.add_argument("--ring", type=int, default=8, help="distinct decode-input steps kept on the device for --config 3|4|5")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per decode launch from an ncu capture (profiles/)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ngc" and not (args.decode_steps or args.batch):
@@ -377,7 +540,10 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the CPU oracle")
-        run_ngc(args)
+        if args.config != 2:
+            run_other(args)
+        else:
+            run_ngc(args)
 
 
 if __name__ == "__main__":
