@@ -118,26 +118,48 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
   }
 }
 
-// After all strips moved: lens[b] <- kept token count (one CTA per sequence,
-// every list of the sequence re-validated; they must agree).
-__global__ void __launch_bounds__(kThreads) compact_lens_kernel(CompactParams p) {
+// Warp-level check of one kept list (coalesced reads, neighbours through shuffles).
+// Returns to every lane the number of kept tokens, or -1 if the list is corrupt.
+__device__ int validate_list_warp(const int32_t* kept, int K, int k_max, int len, int block) {
+  const int lane = threadIdx.x & 31;
+  const int n_units = (len + block - 1) / block;
+  if (K < 0 || K > k_max || K > n_units) return -1;
+  bool bad = false;
+  for (int j0 = 0; j0 < K; j0 += 32) {
+    const int j = j0 + lane;
+    const int u = j < K ? kept[j] : 0x7fffffff;
+    int prev = __shfl_up_sync(0xffffffffu, u, 1);
+    if (lane == 0) prev = j0 > 0 ? kept[j0 - 1] : -1;
+    if (j < K && (u <= prev || u >= n_units)) bad = true;
+  }
+  if (__any_sync(0xffffffffu, bad)) return -1;
+  int tokens = K * block;
+  if (K > 0 && kept[K - 1] == n_units - 1) tokens -= n_units * block - len;   // short last unit
+  return tokens;
+}
+
+// After all strips moved: lens[b] <- kept token count (one CTA per sequence, a warp per list;
+// every list of the sequence is re-validated and they must agree).
+__global__ void compact_lens_kernel(CompactParams p) {
+  __shared__ int s_bad, s_min, s_max;
   const int b = blockIdx.x;
   const int len = p.lens[b];
   const int K = p.budget[b];
-  int tokens0 = -1;
-  bool ok = true;
-  for (int gi = 0; gi < p.G; ++gi) {
-    int fm;
-    int t = validate_list(p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max, K, p.k_max, len, p.block, &fm);
-    if (t < 0) { ok = false; break; }            // already reported by the strip kernel
-    if (tokens0 < 0) tokens0 = t;
-    else if (t != tokens0) {
-      ok = false;
-      if (threadIdx.x == 0) set_dev_status(p.dev_status, NGC_DEV_LISTS_DISAGREE);
-      break;
+  if (threadIdx.x == 0) { s_bad = 0; s_min = 0x7fffffff; s_max = -1; }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  for (int gi = warp; gi < p.G; gi += n_warps) {
+    const int t = validate_list_warp(p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max, K, p.k_max, len, p.block);
+    if ((threadIdx.x & 31) == 0) {
+      if (t < 0) atomicOr(&s_bad, 1);            // already reported by the strip kernel
+      else { atomicMin(&s_min, t); atomicMax(&s_max, t); }
     }
   }
-  if (ok && threadIdx.x == 0) const_cast<int32_t*>(p.lens)[b] = tokens0;
+  __syncthreads();
+  if (threadIdx.x == 0 && !s_bad) {
+    if (s_min != s_max) set_dev_status(p.dev_status, NGC_DEV_LISTS_DISAGREE);
+    else const_cast<int32_t*>(p.lens)[b] = s_min;
+  }
 }
 
 }  // namespace
@@ -167,6 +189,6 @@ extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const in
   compact_kernel<<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
   int rc = launch_status();
   if (rc != NGC_OK) return rc;
-  compact_lens_kernel<<<c->B, kThreads, 0, (cudaStream_t)stream>>>(p);
+  compact_lens_kernel<<<c->B, p.G > 4 ? 1024 : 128, 0, (cudaStream_t)stream>>>(p);
   return launch_status();
 }

@@ -1,12 +1,19 @@
 // ngc_sample_evict: Gumbel-top-k draw of the keep set (paper Section 4.3).
 //
-// One CTA per list.  Every candidate unit gets a 64-bit sort key: the
-// order-preserving integer image of its perturbed fp32 key in the high word
-// and the bit-inverted index in the low word, so that one descending integer
-// sort realises "larger key first, equal keys -> smaller index first".  The
-// keys live in shared memory (lists up to kSampleSmemMaxUnits candidates) or in
-// the caller's workspace (longer lists) and are ordered by a bitonic network;
-// the kept prefix is then marked in a bitmap whose prefix popcounts place the
+// One CTA per list.  The order "larger perturbed key first, equal keys ->
+// smaller index first" is realised on integers: the order-preserving 32-bit
+// image of the fp32 key, sorted descending by a STABLE sort of the candidates
+// taken in index order.
+//  * Lists of up to kSampleSmemMaxUnits candidates: least-significant-digit
+//    radix sort in shared memory, four passes of 8 bits.  Each warp owns a
+//    contiguous segment of the list; per pass it counts its digits (lanes with
+//    equal digits found with one ballot per digit bit, counted with popc), a
+//    CTA-wide prefix scan over (digit, warp) turns the counts into output
+//    offsets, and the warp walks its segment again scattering 16-bit candidate
+//    indices to their ranks.  No atomics.
+//  * Longer lists: 64-bit composite keys (image, inverted index) ordered by a
+//    bitonic network in the caller's workspace.
+// The kept prefix is then marked in a bitmap whose prefix popcounts place the
 // ascending kept list.  Integer work throughout; results do not depend on the
 // launch shape.
 //
@@ -62,6 +69,19 @@ __device__ __forceinline__ uint32_t float_image(float f) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+// Lanes of the warp that are live and hold the same 8-bit digit as the caller: one ballot per
+// digit bit (match.any costs one round per distinct value, about thirty here).
+__device__ __forceinline__ uint32_t same_digit_lanes(uint32_t d, bool live) {
+  uint32_t peers = __ballot_sync(0xffffffffu, live);
+#pragma unroll
+  for (int bit = 0; bit < 8; ++bit) {
+    const bool one = (d >> bit) & 1u;
+    const uint32_t bal = __ballot_sync(0xffffffffu, one);
+    peers &= one ? bal : ~bal;
+  }
+  return peers;
+}
+
 struct SampleParams {
   const float* logits;
   const int32_t* n;
@@ -78,7 +98,9 @@ struct SampleParams {
   int pad_max;                   // power of two >= n_max
 };
 
-template <bool kSmemKeys>
+// kRadix: shared-memory radix sort (n_max <= kSampleSmemMaxUnits); otherwise bitonic sort of
+// 64-bit keys in the workspace.
+template <bool kRadix>
 __global__ void sample_kernel(SampleParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int s_flag;
@@ -88,6 +110,7 @@ __global__ void sample_kernel(SampleParams p) {
   const int li = blockIdx.x;
   const int b = li / p.G;
   const int tid = threadIdx.x, nthr = blockDim.x;
+  const int lane = tid & 31, warp = tid >> 5, n_warps = nthr >> 5;
   const int n = p.n[b];
   const int P = p.n_protect ? p.n_protect[b] : 0;
   const int K = p.budget[b];
@@ -96,11 +119,20 @@ __global__ void sample_kernel(SampleParams p) {
   int32_t* ks = p.kept_sorted + (int64_t)li * p.k_max;
   uint8_t* km = p.keep_mask ? p.keep_mask + (int64_t)li * p.n_max : nullptr;
 
-  unsigned long long* keys;
+  // shared-memory layout
+  uint32_t* img = nullptr;             // [n_max] key images (radix)
+  uint16_t* idx_a = nullptr;           // [n_max] candidate order, ping
+  uint16_t* idx_b = nullptr;           // [n_max] pong
+  uint16_t* hist = nullptr;            // [256][n_warps] digit counts, then output offsets
+  unsigned long long* keys = nullptr;  // composite keys (bitonic)
   uint32_t* bitmap;
-  if (kSmemKeys) {
-    keys = reinterpret_cast<unsigned long long*>(smem_raw);
-    bitmap = reinterpret_cast<uint32_t*>(smem_raw + (size_t)p.pad_max * 8);
+  if (kRadix) {
+    const int n_al = (p.n_max + 7) & ~7;
+    img = reinterpret_cast<uint32_t*>(smem_raw);
+    idx_a = reinterpret_cast<uint16_t*>(smem_raw + (size_t)n_al * 4);
+    idx_b = idx_a + n_al;
+    hist = idx_b + n_al;
+    bitmap = reinterpret_cast<uint32_t*>(hist + 256 * n_warps);
   } else {
     keys = p.ws_keys + (int64_t)li * p.pad_max;
     bitmap = reinterpret_cast<uint32_t*>(smem_raw);
@@ -133,11 +165,17 @@ __global__ void sample_kernel(SampleParams p) {
           if (si != si) nan_seen = 1;
           float kf = p.greedy ? si : __fadd_rn(si, gumbel_from_word(w[j]));
           kf = __fadd_rn(kf, 0.0f);                       // -0 -> +0
-          keys[i - P] = ((unsigned long long)float_image(kf) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
+          if (kRadix) {
+            img[i - P] = float_image(kf);
+            idx_a[i - P] = (uint16_t)(i - P);
+          } else {
+            keys[i - P] = ((unsigned long long)float_image(kf) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
+          }
         }
       }
     }
-    for (int i = n_cand + tid; i < pad; i += nthr) keys[i] = 0ull;   // below every real key
+    if (!kRadix)
+      for (int i = n_cand + tid; i < pad; i += nthr) keys[i] = 0ull;   // below every real key
     if (nan_seen) atomicOr(&s_flag, 1);
   }
   __syncthreads();
@@ -149,17 +187,76 @@ __global__ void sample_kernel(SampleParams p) {
     return;
   }
 
-  // ---- bitonic sort, descending ----
-  for (int k = 2; k <= pad; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int t = tid; t < (pad >> 1); t += nthr) {
-        const int i = 2 * t - (t & (j - 1));
-        const int l = i + j;
-        const unsigned long long x = keys[i], y = keys[l];
-        const bool desc = (i & k) == 0;
-        if ((x < y) == desc) { keys[i] = y; keys[l] = x; }
+  if (kRadix) {
+    // ---- stable LSD radix sort of the candidate order, descending image ----
+    // warp w owns candidates [w*seg, (w+1)*seg), seg a multiple of 32
+    const int seg = (((n_cand + n_warps - 1) / n_warps) + 31) & ~31;
+    const int seg_lo = min(n_cand, warp * seg), seg_hi = min(n_cand, seg_lo + seg);
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint16_t* src = idx_a;
+    uint16_t* dst = idx_b;
+    for (int shift = 0; shift < 32 && Kp > 0; shift += 8) {
+      for (int i = tid; i < 256 * n_warps; i += nthr) hist[i] = 0;
+      __syncthreads();
+      // count: the lowest lane of each group of equal digits adds the group's size
+      for (int i0 = seg_lo; i0 < seg_hi; i0 += 32) {
+        const int i = i0 + lane;
+        const bool live = i < seg_hi;
+        const uint32_t d = live ? 255u - ((img[src[i]] >> shift) & 255u) : 0u;
+        const uint32_t peers = same_digit_lanes(d, live);
+        if (live && (peers & lt_mask) == 0) hist[d * n_warps + warp] += (uint16_t)__popc(peers);
+        __syncwarp();
       }
       __syncthreads();
+      // exclusive scan over (digit, warp): 8 consecutive entries per thread
+      {
+        uint16_t* hp = hist + 8 * tid;
+        int c[8], sum = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { c[e] = hp[e]; sum += c[e]; }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_warp_tot[warp] = incl;
+        __syncthreads();
+        int run = incl - sum;
+        for (int w2 = 0; w2 < warp; ++w2) run += s_warp_tot[w2];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { hp[e] = (uint16_t)run; run += c[e]; }
+      }
+      __syncthreads();
+      // scatter: rank = offset of (digit, warp) + position inside the group
+      for (int i0 = seg_lo; i0 < seg_hi; i0 += 32) {
+        const int i = i0 + lane;
+        const bool live = i < seg_hi;
+        const uint16_t cand = live ? src[i] : (uint16_t)0;
+        const uint32_t d = live ? 255u - ((img[cand] >> shift) & 255u) : 0u;
+        const uint32_t peers = same_digit_lanes(d, live);
+        if (live) dst[hist[d * n_warps + warp] + __popc(peers & lt_mask)] = cand;
+        __syncwarp();
+        if (live && (peers & lt_mask) == 0) hist[d * n_warps + warp] += (uint16_t)__popc(peers);
+        __syncwarp();
+      }
+      __syncthreads();
+      uint16_t* t = src; src = dst; dst = t;
+    }
+    idx_a = src;        // the sorted order
+  } else {
+    // ---- bitonic sort, descending ----
+    for (int k = 2; k <= pad; k <<= 1) {
+      for (int j = k >> 1; j > 0; j >>= 1) {
+        for (int t = tid; t < (pad >> 1); t += nthr) {
+          const int i = 2 * t - (t & (j - 1));
+          const int l = i + j;
+          const unsigned long long x = keys[i], y = keys[l];
+          const bool desc = (i & k) == 0;
+          if ((x < y) == desc) { keys[i] = y; keys[l] = x; }
+        }
+        __syncthreads();
+      }
     }
   }
 
@@ -177,7 +274,7 @@ __global__ void sample_kernel(SampleParams p) {
   for (int j = tid; j < p.k_max; j += nthr) {
     int idx = -1;
     if (j < Kp) {
-      idx = (int)(0xFFFFFFFFu - (uint32_t)(keys[j] & 0xFFFFFFFFull));
+      idx = kRadix ? P + (int)idx_a[j] : (int)(0xFFFFFFFFu - (uint32_t)(keys[j] & 0xFFFFFFFFull));
       atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
     }
     ko[j] = idx;
@@ -187,7 +284,6 @@ __global__ void sample_kernel(SampleParams p) {
   // ---- ascending kept list from the prefix popcounts of the bitmap ----
   if (tid == 0) s_carry = 0;
   __syncthreads();
-  const int lane = tid & 31, warp = tid >> 5, n_warps = nthr >> 5;
   for (int base = 0; base < n_words; base += nthr) {
     const int wd = base + tid;
     const uint32_t m = wd < n_words ? bitmap[wd] : 0u;
@@ -259,7 +355,8 @@ extern "C" int ngc_sample_evict(const float* logits, const int32_t* n, const int
   int threads = p.pad_max >= 2048 ? 1024 : (p.pad_max >= 512 ? 256 : 64);
   const unsigned grid = (unsigned)(B * G);
   if (n_max <= kSampleSmemMaxUnits) {
-    const size_t smem = (size_t)p.pad_max * 8 + bitmap_bytes;
+    const size_t n_al = (size_t)((n_max + 7) & ~7);
+    const size_t smem = n_al * 4 + 2 * n_al * 2 + (size_t)256 * (threads / 32) * 2 + bitmap_bytes;
     if (smem > 48 * 1024)
       NGC_CUDA_TRY(cudaFuncSetAttribute(sample_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     sample_kernel<true><<<grid, threads, smem, (cudaStream_t)stream>>>(p);
