@@ -7,8 +7,11 @@
 // without ever seeing a moved row, as long as every load of tile i is done
 // before the first store of tile i (one __syncthreads per tile).  The leading
 // run of tokens that already sit in place is skipped.  HBM-bound: 16-byte
-// vector loads/stores, several CTAs per SM, next tile prefetched into
-// registers before the current one is stored.
+// vector loads/stores, four CTAs per SM, next tile prefetched into registers
+// before the current one is stored.  (Measured alternatives that were slower
+// on B200: per-row bulk async copies, 256 bytes each, are limited by the copy
+// engine's request rate; a cp.async gather into a shared-memory ring with one
+// bulk store per 16 KB tile loses to this kernel the deeper its ring is.)
 #include "ngc_common.cuh"
 
 namespace ngc {
@@ -41,11 +44,23 @@ __device__ int validate_list(const int32_t* kept, int K, int k_max, int len, int
   int bad = (K < 0 || K > k_max || K > n_units) ? 1 : 0;
   int first = 0x7fffffff;
   if (!bad) {
-    for (int j = threadIdx.x; j < K; j += blockDim.x) {
-      int u = kept[j];
-      int prev = j > 0 ? kept[j - 1] : -1;
-      if (u <= prev || u >= n_units) bad = 1;
-      if (u != j && j < first) first = j;
+    // eight independent loads per thread in flight: the list may come from HBM
+    for (int j0 = threadIdx.x; j0 < K; j0 += 8 * blockDim.x) {
+      int u[8], prev[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int j = j0 + e * blockDim.x;
+        u[e] = j < K ? kept[j] : 0;
+        prev[e] = (j > 0 && j < K) ? kept[j - 1] : -1;
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int j = j0 + e * blockDim.x;
+        if (j < K) {
+          if (u[e] <= prev[e] || u[e] >= n_units) bad = 1;
+          if (u[e] != j && j < first) first = j;
+        }
+      }
     }
   }
   if (bad) atomicOr(&s_bad, 1);
@@ -125,12 +140,22 @@ __device__ int validate_list_warp(const int32_t* kept, int K, int k_max, int len
   const int n_units = (len + block - 1) / block;
   if (K < 0 || K > k_max || K > n_units) return -1;
   bool bad = false;
-  for (int j0 = 0; j0 < K; j0 += 32) {
-    const int j = j0 + lane;
-    const int u = j < K ? kept[j] : 0x7fffffff;
-    int prev = __shfl_up_sync(0xffffffffu, u, 1);
-    if (lane == 0) prev = j0 > 0 ? kept[j0 - 1] : -1;
-    if (j < K && (u <= prev || u >= n_units)) bad = true;
+  for (int jb = 0; jb < K; jb += 128) {          // four independent loads per lane in flight
+    int u[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int j = jb + 32 * e + lane;
+      u[e] = j < K ? kept[j] : 0x7fffffff;
+    }
+    int edge = (lane < 4 && jb + 32 * lane > 0 && jb + 32 * lane < K) ? kept[jb + 32 * lane - 1] : -1;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int j = jb + 32 * e + lane;
+      int prev = __shfl_up_sync(0xffffffffu, u[e], 1);
+      const int first_prev = __shfl_sync(0xffffffffu, edge, e);
+      if (lane == 0) prev = first_prev;
+      if (j < K && (u[e] <= prev || u[e] >= n_units)) bad = true;
+    }
   }
   if (__any_sync(0xffffffffu, bad)) return -1;
   int tokens = K * block;
