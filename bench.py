@@ -43,12 +43,16 @@ OTHER_WORKLOADS = {
     4: "config4: per-(layer, KV head) eviction (L28, 12q/2kv, d128, bf16, B128, 16384 -> 8192 tokens, 7168 lists, 64 decode steps)",
     5: "config5: rollout loop (L28, 12q/2kv, d128, bf16, B64, 256 prompt + 8192 generated, a round every 512 tokens 768 -> 256, "
        "per-layer lists) + log-prob recompute of all 16 rounds",
+    6: "config6: the paper's Countdown setting (L28, 12q/2kv, d128, bf16, B512 = 32 prompts x 16 rollouts, 256 prompt + 1024 generated, "
+       "a round every 256 tokens 512 -> 256, units of 32 tokens, per-layer lists scored from K with 5 recent queries)",
+    7: "config7: the paper's math setting (L28, 12q/2kv, d128, bf16, B2048 = 256 prompts x 8 rollouts, 352 prompt + 1056 generated, "
+       "a round every 352 tokens 704 -> 352, units of 32 tokens, per-layer lists scored from K with 5 recent queries)",
 }
 METRIC = "evict+compact+decode tokens/sec at B=64"
 W_RECENT = 5
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic K/V bytes for decode_stream_kernel, from the ncu
 # capture summarised in profiles/decode_stream_kernel_config2.md (small case, scaled by tokens processed)
-NCU_TRAFFIC_RATIO = 1.0377
+NCU_TRAFFIC_RATIO = 1.0387
 
 
 def peaks():
@@ -310,14 +314,17 @@ def run_other(args):
     L, B, Hq, Hkv, d, steps = cfg["L"], args.batch or cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["d"], args.decode_steps or cfg["steps"]
     dtype = torch.bfloat16
     lists = cfg["lists"]
-    if cid == 5:
+    loop = cid >= 5                      # grow-then-evict loop (rounds) instead of one round + decode
+    block = cfg.get("block", 1)
+    from_score = cid >= 6               # the draw uses the scores of the real K, not synthetic logits
+    if loop:
         prompt, cadence, K = cfg["T"], cfg["cadence"], cfg["budget"]
         rounds = max(1, steps // cadence)
         steps = rounds * cadence
         lens = torch.full((B,), prompt, dtype=torch.int32)
-        budget = torch.full((B,), K, dtype=torch.int32)
+        budget = torch.full((B,), K, dtype=torch.int32)              # in units
         cap = torch.full((B,), prompt + cadence, dtype=torch.int64)
-        n_evict = torch.full((B,), prompt + cadence, dtype=torch.int32)
+        n_evict = torch.full((B,), (prompt + cadence) // block, dtype=torch.int32)
     else:
         if isinstance(cfg["T"], tuple):
             lens = synth.ragged_lens(B, cfg["T"][0], cfg["T"][1], cfg["len_seed"])
@@ -328,11 +335,12 @@ def run_other(args):
         n_evict = lens
     n_max, k_max = int(n_evict.max()), int(budget.max())
     src = synth.make_cache(L, B, Hq, Hkv, d, dtype, lens, capacity=cap, seed=cfg["data_seed"], outlier_channels=cfg["outliers"], device=dev)
-    ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=cap, n_max=n_max, k_max=k_max, lists=lists, device=dev, w=W_RECENT, kv=(src.k, src.v))
+    ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=cap, n_max=n_max, k_max=k_max, lists=lists, block=block, device=dev, w=W_RECENT,
+                    kv=(src.k, src.v))
     del src
     G = ro.G
     lens0 = lens.to(dev)
-    logits = synth.make_logits(B, G, n_max, seed=cfg["data_seed"] + 7, std=cfg["logit_std"], device=dev)
+    logits = ro.score_logits if from_score else synth.make_logits(B, G, n_max, seed=cfg["data_seed"] + 7, std=cfg["logit_std"], device=dev)
     n_t, k_t = n_evict.to(dev), budget.to(dev)
     ring = min(steps, args.ring)
     q = synth.make_queries(L, B, Hq, d, dtype, seed=11, steps=ring, device=dev)
@@ -355,7 +363,7 @@ def run_other(args):
         e[2].record()
         ngc.ngc_evict_logprob(logits, n_t, None, k_t, ro.kept_order, ro.logp, status=ro.status)
         e[3].record()
-        ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, lists, 1, status=ro.status)
+        ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, lists, block, status=ro.status)
         e[4].record()
         ro.launches += 7          # score 3, sample 1, log-prob 1, compaction 2
         t.append(e)
@@ -368,7 +376,7 @@ def run_other(args):
         e1.record()
         t.append((e0, e1))
 
-    if cid == 5:
+    if loop:
         all_logits = logits.unsqueeze(0).expand(rounds, B, G, n_max).contiguous()
         all_ko = torch.zeros((rounds, B, G, k_max), dtype=torch.int32, device=dev)
         all_lp = torch.empty((rounds, B, G), dtype=torch.float64, device=dev)
@@ -377,11 +385,13 @@ def run_other(args):
     def one_step(i, rec):
         ro.cache.lens.copy_(lens0, non_blocking=True)
         ev_t, dec_t, rc = [], [], None
-        if cid == 5:
+        if loop:
             for r in range(rounds):
                 decode(cadence, dec_t)
                 eviction(i * rounds + r, ev_t)
                 all_ko[r].copy_(ro.kept_order, non_blocking=True)
+                if from_score:
+                    all_logits[r].copy_(logits, non_blocking=True)
             rc = (ev(), ev())
             rc[0].record()
             ngc.ngc_evict_logprob(all_logits, n_all, None, k_all, all_ko, all_lp, status=ro.status)
@@ -421,9 +431,10 @@ def run_other(args):
     tokens = B * steps
     # algorithmic K/V bytes: every visible token of every decode launch; every kept row read + written by compaction
     kept = float(budget.sum())
-    if cid == 5:
+    if loop:
+        kept *= block
         vis = B * rounds * sum(prompt + s + 1 for s in range(cadence))
-        score_bytes = float(n_evict.sum()) * row_bytes / 2
+        score_bytes = float(n_evict.sum()) * block * row_bytes / 2
     else:
         vis = sum(kept + B * (s + 1) for s in range(steps))
         score_bytes = float(lens.sum()) * row_bytes / 2
@@ -528,8 +539,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seqs", type=int, default=4)
     ap.add_argument("--cpu-decode-steps", type=int, default=48)
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5],
-                    help="2 = the benchmark workload (default); 3, 4, 5 = the other workloads, one GPU, per-phase timing only")
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5, 6, 7],
+                    help="2 = the benchmark workload (default); 3..7 = the other workloads, one GPU, per-phase timing only")
     ap.add_argument("--ring", type=int, default=8, help="distinct decode-input steps kept on the device for --config 3|4|5")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per decode launch from an ncu capture (profiles/)")
     args = ap.parse_args()

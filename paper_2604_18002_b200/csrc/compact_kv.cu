@@ -76,7 +76,12 @@ __device__ int validate_list(const int32_t* kept, int K, int k_max, int len, int
   return tokens;
 }
 
+// RV = 16-byte vectors per row (8, 16 or 32: rows of 128, 256 or 512 bytes); compile-time so that
+// the row / column split of a thread's vectors costs shifts, not divisions.
+template <int RV>
 __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
+  constexpr int kRowsPerPass = kThreads / RV;                 // rows the CTA covers with one vector per thread
+  constexpr int kTileRows = kRowsPerPass * kVecPerThread;
   int s = blockIdx.x;
   const int kv = s & 1; s >>= 1;
   const int b = s % p.B; s /= p.B;
@@ -93,39 +98,40 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
     if (threadIdx.x == 0) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
     return;
   }
-  uint4* strip = (kv ? p.v : p.k) + (int64_t)(l * p.Hkv + h) * p.plane_vecs + p.seq_off[b] * p.row_vecs;
-
-  const int rv = p.row_vecs;
-  const int tile_rows = kThreads * kVecPerThread / rv;
+  const int my_row = threadIdx.x / RV, my_col = threadIdx.x % RV;
+  uint4* strip = (kv ? p.v : p.k) + (int64_t)(l * p.Hkv + h) * p.plane_vecs + p.seq_off[b] * RV + my_col;
   const int block = p.block;
   uint4 cur[kVecPerThread], nxt[kVecPerThread];
 
   auto load_tile = [&](int t0, uint4 (&r)[kVecPerThread]) {
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
-      int slot = u * kThreads + threadIdx.x;
-      int jt = t0 + slot / rv;
+      const int jt = t0 + u * kRowsPerPass + my_row;
       if (jt < tokens) {
-        int unit = jt / block;
-        int src = kept[unit] * block + (jt - unit * block);
-        r[u] = __ldcs(strip + (int64_t)src * rv + slot % rv);
+        int64_t src;
+        if (block == 1) {
+          src = kept[jt];
+        } else {
+          const int unit = jt / block;
+          src = (int64_t)kept[unit] * block + (jt - unit * block);
+        }
+        r[u] = __ldcs(strip + src * RV);
       }
     }
   };
   auto store_tile = [&](int t0, const uint4 (&r)[kVecPerThread]) {
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
-      int slot = u * kThreads + threadIdx.x;
-      int jt = t0 + slot / rv;
-      if (jt < tokens) strip[(int64_t)jt * rv + slot % rv] = r[u];
+      const int jt = t0 + u * kRowsPerPass + my_row;
+      if (jt < tokens) strip[(int64_t)jt * RV] = r[u];
     }
   };
 
   int t0 = first_moved;
   if (t0 >= tokens) return;
   load_tile(t0, cur);
-  for (; t0 < tokens; t0 += tile_rows) {
-    if (t0 + tile_rows < tokens) load_tile(t0 + tile_rows, nxt);
+  for (; t0 < tokens; t0 += kTileRows) {
+    if (t0 + kTileRows < tokens) load_tile(t0 + kTileRows, nxt);
     __syncthreads();            // every load of this tile has completed
     store_tile(t0, cur);
 #pragma unroll
@@ -211,7 +217,11 @@ extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const in
   p.lists = lists; p.block = block; p.k_max = k_max;
   const int64_t strips = (int64_t)c->L * c->Hkv * c->B * 2;
   if (strips > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
-  compact_kernel<<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
+  if ((((uintptr_t)c->k | (uintptr_t)c->v) & 15) != 0) return NGC_ERR_INVALID_ARG;      // rows move as 16-byte vectors
+  if (p.row_vecs == 8) compact_kernel<8><<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
+  else if (p.row_vecs == 16) compact_kernel<16><<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
+  else if (p.row_vecs == 32) compact_kernel<32><<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
+  else return NGC_ERR_UNSUPPORTED;
   int rc = launch_status();
   if (rc != NGC_OK) return rc;
   compact_lens_kernel<<<c->B, p.G > 4 ? 1024 : 128, 0, (cudaStream_t)stream>>>(p);

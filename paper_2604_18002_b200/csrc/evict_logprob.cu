@@ -7,6 +7,10 @@
 // additions only (the remaining-mass bookkeeping the paper mentions after
 // Eq. (1), arranged so that nothing is subtracted).  Reductions and the scan
 // use a fixed tree order: results are reproducible run to run.
+//
+// Lists of at most 32 units (the paper's own setting: block-level lists of
+// 16-22 units, Section 5.1) take a warp each, eight lists per CTA, the whole
+// list in registers and every reduction a shuffle.
 #include "ngc_common.cuh"
 
 namespace ngc {
@@ -131,6 +135,68 @@ __global__ void __launch_bounds__(kThreads) logprob_kernel(LogprobParams p) {
   if (tid == 0) p.logp[li] = total;
 }
 
+// ---------------------------------------------------------------- lists of at most 32 units
+
+constexpr int kTinyWarps = 8;
+
+__global__ void __launch_bounds__(kTinyWarps * 32) logprob_tiny_kernel(LogprobParams p, int64_t n_lists) {
+  const int lane = threadIdx.x & 31;
+  const int64_t li = (int64_t)blockIdx.x * kTinyWarps + (threadIdx.x >> 5);
+  if (li >= n_lists) return;
+  const int64_t outer = li / p.G;
+  const int n = p.n[outer];
+  const int P = p.n_protect ? p.n_protect[outer] : 0;
+  const int K = p.budget[outer];
+  const int Kp = K - P;
+  const float* s = p.logits + li * p.n_max;
+  const int32_t* sigma = p.kept_order + li * p.k_max;
+  const double kNaN = __longlong_as_double(0x7ff8000000000000LL);
+
+  if (!(P >= 0 && P <= K && K <= n && n <= p.n_max && Kp <= p.k_max)) {
+    if (lane == 0) { set_dev_status(p.dev_status, NGC_DEV_BAD_COUNTS); p.logp[li] = kNaN; }
+    return;
+  }
+  // lane j holds sigma_j; lane t holds logit t
+  const int sj = lane < Kp ? sigma[lane] : -1;
+  const bool in_range = lane >= Kp || (sj >= P && sj < n);
+  uint32_t drawn = 0;                 // bit t set: unit t was drawn
+  bool repeat = false;
+  for (int j = 0; j < Kp; ++j) {
+    const int t = __shfl_sync(0xffffffffu, sj, j) & 31;
+    if (drawn & (1u << t)) repeat = true;
+    drawn |= 1u << t;
+  }
+  if (!__all_sync(0xffffffffu, in_range) || repeat) {
+    if (lane == 0) { set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); p.logp[li] = kNaN; }
+    return;
+  }
+  if (Kp == 0) {
+    if (lane == 0) p.logp[li] = 0.0;
+    return;
+  }
+  const bool cand = lane >= P && lane < n;
+  const float v = cand ? s[lane] : -INFINITY;
+  if (__any_sync(0xffffffffu, cand && v != v)) {
+    if (lane == 0) { set_dev_status(p.dev_status, NGC_DEV_NAN_LOGIT); p.logp[li] = kNaN; }
+    return;
+  }
+  const double M = (double)warp_max(v);
+  const double e_t = cand ? exp((double)v - M) : 0.0;
+  // mass never drawn, then the tail sums of the drawn masses in sigma order
+  const double U = warp_sum(((drawn >> lane) & 1u) ? 0.0 : e_t);
+  const int src = sj < 0 ? 0 : sj;
+  const double z = __shfl_sync(0xffffffffu, (double)v - M, src);     // s_sigma_j - M on lane j
+  const double e = __shfl_sync(0xffffffffu, e_t, src);
+  double tail = lane < Kp ? e : 0.0;                                 // -> sum_{i >= j} e_sigma_i
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const double t = __shfl_down_sync(0xffffffffu, tail, o);
+    if (lane + o < 32) tail += t;
+  }
+  const double total = warp_sum(lane < Kp ? z - log(U + tail) : 0.0);
+  if (lane == 0) p.logp[li] = total;
+}
+
 }  // namespace
 }  // namespace ngc
 
@@ -151,6 +217,9 @@ extern "C" int ngc_evict_logprob(const float* logits, const int32_t* n, const in
   LogprobParams p;
   p.logits = logits; p.n = n; p.n_protect = n_protect; p.budget = budget; p.kept_order = kept_order;
   p.logp = logp; p.dev_status = dev_status; p.G = G; p.n_max = n_max; p.k_max = k_max;
-  logprob_kernel<<<(unsigned)lists, kThreads, smem, (cudaStream_t)stream>>>(p);
+  if (n_max <= 32)
+    logprob_tiny_kernel<<<(unsigned)((lists + kTinyWarps - 1) / kTinyWarps), kTinyWarps * 32, 0, (cudaStream_t)stream>>>(p, lists);
+  else
+    logprob_kernel<<<(unsigned)lists, kThreads, smem, (cudaStream_t)stream>>>(p);
   return launch_status();
 }

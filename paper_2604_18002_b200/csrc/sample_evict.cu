@@ -320,6 +320,65 @@ __global__ void sample_kernel(SampleParams p) {
   }
 }
 
+// ---------------------------------------------------------------- lists of at most 32 units
+//
+// The paper's own lists are this small (block-level eviction: 16-22 units, Section 5.1).  A warp
+// takes a list, a lane a unit: the rank of a candidate is the number of candidates with a larger
+// composite key, counted over 32 shuffles; ballots give the mask and the ascending list.
+
+constexpr int kTinyWarps = 8;
+
+__global__ void __launch_bounds__(kTinyWarps * 32) sample_tiny_kernel(SampleParams p, int n_lists) {
+  const int lane = threadIdx.x & 31;
+  const int li = blockIdx.x * kTinyWarps + (threadIdx.x >> 5);
+  if (li >= n_lists) return;
+  const int b = li / p.G;
+  const int n = p.n[b];
+  const int P = p.n_protect ? p.n_protect[b] : 0;
+  const int K = p.budget[b];
+  const float* s = p.logits + (int64_t)li * p.n_max;
+  int32_t* ko = p.kept_order + (int64_t)li * p.k_max;
+  int32_t* ks = p.kept_sorted + (int64_t)li * p.k_max;
+  uint8_t* km = p.keep_mask ? p.keep_mask + (int64_t)li * p.n_max : nullptr;
+
+  const bool counts_ok = P >= 0 && P <= K && K <= n && n <= p.n_max && K <= p.k_max;
+  const bool cand = counts_ok && lane >= P && lane < n;
+  const float si = cand ? s[lane] : 0.f;
+  const bool nan_seen = __any_sync(0xffffffffu, cand && si != si);
+  if (!counts_ok || nan_seen) {
+    if (lane == 0) set_dev_status(p.dev_status, counts_ok ? NGC_DEV_NAN_LOGIT : NGC_DEV_BAD_COUNTS);
+    for (int j = lane; j < p.k_max; j += 32) { ko[j] = -1; ks[j] = -1; }
+    if (km && lane < p.n_max) km[lane] = 0;
+    return;
+  }
+  const int Kp = K - P;
+  // perturbed key of this lane's unit (one Philox call serves units 4q .. 4q+3)
+  unsigned long long key = 0ull;                     // below every candidate
+  if (cand) {
+    float kf = si;
+    if (!p.greedy) {
+      const uint4 r = philox4x32_10(make_uint4((uint32_t)(lane >> 2), p.list_base + (uint32_t)li, (uint32_t)p.round,
+                                               (uint32_t)(p.round >> 32)),
+                                    make_uint2((uint32_t)p.seed, (uint32_t)(p.seed >> 32)));
+      const uint32_t w = (lane & 3) == 0 ? r.x : ((lane & 3) == 1 ? r.y : ((lane & 3) == 2 ? r.z : r.w));
+      kf = __fadd_rn(si, gumbel_from_word(w));
+    }
+    kf = __fadd_rn(kf, 0.0f);                        // -0 -> +0
+    key = ((unsigned long long)float_image(kf) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)lane);
+  }
+  int rank = 0;                                      // candidates in front of this one
+#pragma unroll
+  for (int j = 0; j < 32; ++j) rank += __shfl_sync(0xffffffffu, key, j) > key ? 1 : 0;
+  const bool drawn = cand && rank < Kp;
+  const bool kept = drawn || (lane < P);
+  if (drawn) ko[rank] = lane;
+  for (int j = Kp + lane; j < p.k_max; j += 32) ko[j] = -1;
+  const uint32_t mask = __ballot_sync(0xffffffffu, kept);
+  if (kept) ks[__popc(mask & ((1u << lane) - 1u))] = lane;
+  for (int j = K + lane; j < p.k_max; j += 32) ks[j] = -1;
+  if (km && lane < p.n_max) km[lane] = kept ? 1 : 0;
+}
+
 inline int pow2_at_least(int x) {
   int p = 1;
   while (p < x) p <<= 1;
@@ -354,7 +413,9 @@ extern "C" int ngc_sample_evict(const float* logits, const int32_t* n, const int
   const size_t bitmap_bytes = (size_t)((n_max + 31) / 32) * 4;
   int threads = p.pad_max >= 2048 ? 1024 : (p.pad_max >= 512 ? 256 : 64);
   const unsigned grid = (unsigned)(B * G);
-  if (n_max <= kSampleSmemMaxUnits) {
+  if (n_max <= 32) {
+    sample_tiny_kernel<<<(grid + kTinyWarps - 1) / kTinyWarps, kTinyWarps * 32, 0, (cudaStream_t)stream>>>(p, (int)grid);
+  } else if (n_max <= kSampleSmemMaxUnits) {
     const size_t n_al = (size_t)((n_max + 7) & ~7);
     const size_t smem = n_al * 4 + 2 * n_al * 2 + (size_t)256 * (threads / 32) * 2 + bitmap_bytes;
     if (smem > 48 * 1024)

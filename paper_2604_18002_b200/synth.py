@@ -147,4 +147,10 @@ CONFIGS = {
             budget=8192, lists=2, logit_std=1.0, steps=64, outliers=0, data_seed=0, noise_seed=1),
     5: dict(name="rollout-loop-B64", L=28, Hq=12, Hkv=2, d=128, dtype="bf16", B=64, T=256, n_protect=0,
             budget=256, lists=1, logit_std=1.0, steps=8192, cadence=512, outliers=0, data_seed=0, noise_seed=1),
+    # the paper's own eviction setting: units of 32 tokens, 5 recent queries, one list per layer scored from the
+    # real K, half of the units kept each round; 512 = 32 prompts x 16 rollouts, 2048 = 256 prompts x 8 rollouts
+    6: dict(name="paper-countdown-B512", L=28, Hq=12, Hkv=2, d=128, dtype="bf16", B=512, T=256, n_protect=0,
+            budget=8, block=32, lists=1, logit_std=1.0, steps=1024, cadence=256, outliers=0, data_seed=0, noise_seed=1),
+    7: dict(name="paper-math-B2048", L=28, Hq=12, Hkv=2, d=128, dtype="bf16", B=2048, T=352, n_protect=0,
+            budget=11, block=32, lists=1, logit_std=1.0, steps=1056, cadence=352, outliers=0, data_seed=0, noise_seed=1),
 }

@@ -265,3 +265,79 @@ def test_config5_rollout_loop_and_logprob_recompute():
     for r, bb in [(0, 0), (5, 17), (15, 63)]:
         lit, rc = oracle.evict_logprob(lg[r, bb:bb + 1], [peak], None, [K], ko[r, bb:bb + 1])
         assert rc == 0 and np.max(np.abs(lp2[r, bb].cpu().numpy() - lit[0, 0])) <= 1e-3
+
+
+def test_config6_paper_setting_block_eviction_scored_from_k():
+    """The paper's own eviction setting at full size (Section 5.1: units of 32 tokens, 5 recent queries,
+    a round every 256 tokens keeping half, one list per layer): 512 rollouts, 4 rounds.  Every round's
+    scores are checked on sampled sequences (2e-2 of the largest score), the draw for EVERY list
+    bit-exact from the scores the GPU produced, Eq. (1) literally for every list, the compacted rows
+    of the sampled sequences bit-exact, attention at a few steps."""
+    need_gpu_gb(12)
+    b = ngc()
+    from paper_2604_18002_b200.rollout import NgcRollout
+    cfg = synth.CONFIGS[6]
+    L, Hq, Hkv, d, B = cfg["L"], cfg["Hq"], cfg["Hkv"], cfg["d"], cfg["B"]
+    prompt, cadence, K, block = cfg["T"], cfg["cadence"], cfg["budget"], cfg["block"]
+    rounds = cfg["steps"] // cadence
+    peak = prompt + cadence
+    N = peak // block
+    dtype, dev, lists, w = torch.bfloat16, "cuda", cfg["lists"], 5
+    src = synth.make_cache(L, B, Hq, Hkv, d, dtype, [prompt] * B, capacity=peak, seed=4, device=dev)
+    ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=peak, n_max=N, k_max=K, lists=lists, block=block, w=w, device=dev,
+                    kv=(src.k, src.v))
+    G = ro.G
+    ro.cache.lens.copy_(src.lens)
+    del src
+    seqs = [0, 300]
+    mirror = SampledSeqs(ro.cache, seqs, peak)
+    kc, vc = mirror.k, mirror.v
+    o_lens = np.full(len(seqs), prompt, np.int32)
+    n_np, k_np = np.full(B, N, np.int32), np.full(B, K, np.int32)
+    n_t, k_t = torch.as_tensor(n_np).to(dev), torch.as_tensor(k_np).to(dev)
+    out = torch.empty((L, B, Hq, d), dtype=torch.float32, device=dev)
+    check_in_round = {0: [0, 255], 2: [77], 3: [255]}
+    step = 0
+    for r in range(rounds):
+        for s in range(cadence):
+            q = synth.make_queries(L, B, Hq, d, dtype, seed=20000 + step, device=dev)
+            nk, nv = synth.make_new_kv(L, B, Hkv, d, dtype, seed=40000 + 2 * step, device=dev)
+            ro.decode_step(q, out, nk, nv)
+            nk_h, nv_h = synth.to_numpy(nk[:, seqs]), synth.to_numpy(nv[:, seqs])
+            if s in check_in_round.get(r, []):
+                ref, rc = oracle.decode_attn(kc, vc, mirror.so, o_lens, synth.to_numpy(q[:, seqs]), nk_h, nv_h)
+                assert rc == 0
+                check_attention(out[:, seqs].cpu().numpy().astype(np.float64), ref, dtype)
+            else:
+                for i in range(len(seqs)):
+                    kc[:, :, i * peak + o_lens[i]] = nk_h[:, i]
+                    vc[:, :, i * peak + o_lens[i]] = nv_h[:, i]
+                o_lens += 1
+            step += 1
+        assert int(ro.cache.lens.max()) == peak and int(ro.cache.lens.min()) == peak
+        qr = synth.normal((L, B, Hq, w, d), 70000 + r, dtype, device=dev)
+        ro.eviction_round(n_t, None, k_t, cfg["noise_seed"], r, q_recent=qr)          # draws from the scores
+        torch.cuda.synchronize()
+        ro.check_status()
+        lg = ro.logits.cpu().numpy()
+        # scores of the sampled sequences
+        ref_s = oracle.score_evict(kc, mirror.so, o_lens, synth.to_numpy(qr[:, seqs]), block, lists, n_max=N)
+        for i, bb in enumerate(seqs):
+            for g in range(G):
+                assert np.max(np.abs(lg[bb, g] - ref_s[i, g])) <= 2e-2 * ref_s[i, g].max()
+            assert abs(lg[bb].sum() * block - G) <= 1e-2                                # each layer's psi sums to one
+        # the draw, every list, from the very logits the GPU wrote
+        r_ko, r_ks, _, st = oracle.sample_evict(lg, n_np, None, k_np, K, seed=cfg["noise_seed"], rnd=r)
+        assert not st.any()
+        assert np.array_equal(ro.kept_order.cpu().numpy(), r_ko) and np.array_equal(ro.kept_sorted.cpu().numpy(), r_ks)
+        lit, rc = oracle.evict_logprob(lg, n_np, None, k_np, r_ko)
+        assert rc == 0 and np.max(np.abs(ro.logp.cpu().numpy() - lit)) <= 1e-3
+        sel = np.array(seqs)
+        kc, vc, nl, rc = oracle.compact_kv(kc, vc, mirror.so, o_lens, r_ks[sel], k_np[sel], lists, block)
+        assert rc == 0 and np.all(nl == K * block)
+        o_lens = nl.copy()
+        after = SampledSeqs(ro.cache, seqs, peak)
+        for i in range(len(seqs)):
+            sl = slice(i * peak, i * peak + K * block)
+            assert np.array_equal(after.k[:, :, sl], kc[:, :, sl]) and np.array_equal(after.v[:, :, sl], vc[:, :, sl])
+    assert np.array_equal(ro.cache.lens.cpu().numpy(), np.full(B, K * block, np.int32))     # steady state: delta / epsilon / 2

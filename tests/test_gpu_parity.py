@@ -391,3 +391,62 @@ def test_score_window_sizes_and_ragged_lengths(Hq, Hkv, w, lens):
                 m = live[bb, g]
                 assert np.max(np.abs(got[bb, g][m] - ref[bb, g][m])) <= 2e-2 * ref[bb, g][m].max()
                 assert abs(got[bb, g][m].sum() - 1.0) <= 1e-3          # psi is a mean of probability rows
+
+
+# ------------------------------------------------------------------ lists of at most 32 units (warp-per-list kernels)
+
+@pytest.mark.parametrize("B,G,n_max", [(37, 28, 16), (19, 28, 22), (5, 3, 32), (9, 1, 2), (64, 56, 8)])
+def test_tiny_lists_sample_and_logprob(B, G, n_max):
+    """The paper's own list sizes (block-level eviction: 16-22 units per layer): sampling bit-exact,
+    log-prob within 1e-3 (fp64: far inside), ragged n, protected prefixes, K = n and K = P included."""
+    rng = np.random.default_rng(B * 1000 + n_max)
+    logits = synth.make_logits(B, G, n_max, seed=n_max + 5, std=1.3).numpy()
+    logits[0, 0, : min(4, n_max)] = 0.5                                     # ties
+    n = rng.integers(1, n_max + 1, B).astype(np.int32)
+    n[0] = n_max
+    P = np.array([rng.integers(0, x // 3 + 1) for x in n], np.int32)
+    K = np.array([rng.integers(p, x + 1) for p, x in zip(P, n)], np.int32)
+    K[0] = max(P[0], n_max // 2)
+    if B > 2:
+        K[1] = n[1]
+        K[2] = P[2]
+    k_max = int(K.max()) + 2
+    for greedy in (0, 1):
+        ref = oracle.sample_evict(logits, n, P, K, k_max, seed=5, rnd=9, greedy=greedy, list_base=3)
+        got = gpu_sample(logits, n, P, K, k_max, seed=5, rnd=9, greedy=greedy, list_base=3)
+        assert got[3] == 0 and not ref[3].any()
+        for i in range(3):
+            assert np.array_equal(got[i], ref[i])
+        lp_ref, rc = oracle.evict_logprob(logits, n, P, K, ref[0])
+        lp, st = gpu_logprob(logits, n, P, K, ref[0])
+        assert rc == 0 and st == 0
+        assert np.max(np.abs(lp - lp_ref)) <= TOL_LOGP and np.max(np.abs(lp - lp_ref)) <= 1e-9
+
+
+def test_tiny_lists_status_paths():
+    logits = synth.make_logits(4, 2, 20, seed=2).numpy()
+    n = np.array([20, 12, 20, 7], np.int32)
+    K = np.array([10, 6, 10, 3], np.int32)
+    logits[1, 1, 4] = np.nan                                              # NaN candidate -> list blanked, status 2
+    ref = oracle.sample_evict(logits, n, None, K, 10, seed=1, rnd=1)
+    got = gpu_sample(logits, n, None, K, 10, seed=1, rnd=1)
+    assert got[3] == 2 and ref[3][1, 1] == 2
+    for i in range(3):
+        assert np.array_equal(got[i], ref[i])
+    got = gpu_sample(logits, n, None, np.array([21, 6, 10, 3], np.int32), 21, seed=1, rnd=1)   # K > n -> status 1
+    assert got[3] == 1 and np.all(got[0][0] == -1) and np.all(got[1][0] == -1) and got[2][0].sum() == 0
+    # log-prob: repeated unit, out-of-range unit, NaN logit
+    logits[1, 1, 4] = 0.0
+    ko = oracle.sample_evict(logits, n, None, K, 10, seed=1, rnd=1)[0]
+    good = oracle.evict_logprob(logits, n, None, K, ko)[0]
+    bad = ko.copy()
+    bad[2, 0, 1] = bad[2, 0, 0]
+    lp, st = gpu_logprob(logits, n, None, K, bad)
+    assert st == 3 and math.isnan(lp[0, 2, 0]) and abs(lp[0, 0, 0] - good[0, 0, 0]) < 1e-9
+    bad = ko.copy()
+    bad[3, 1, 2] = 7                                                      # unit 7 of a list of 7 units
+    lp, st = gpu_logprob(logits, n, None, K, bad)
+    assert st == 3 and math.isnan(lp[0, 3, 1])
+    logits[0, 1, 3] = np.nan
+    lp, st = gpu_logprob(logits, n, None, K, ko)
+    assert st == 2 and math.isnan(lp[0, 0, 1]) and abs(lp[0, 1, 0] - good[0, 1, 0]) < 1e-9
