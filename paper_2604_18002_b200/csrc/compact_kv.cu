@@ -7,11 +7,13 @@
 // without ever seeing a moved row, as long as every load of tile i is done
 // before the first store of tile i (one __syncthreads per tile).  The leading
 // run of tokens that already sit in place is skipped.  HBM-bound: 16-byte
-// vector loads/stores, four CTAs per SM, next tile prefetched into registers
-// before the current one is stored.  (Measured alternatives that were slower
-// on B200: per-row bulk async copies, 256 bytes each, are limited by the copy
-// engine's request rate; a cp.async gather into a shared-memory ring with one
-// bulk store per 16 KB tile loses to this kernel the deeper its ring is.)
+// vector loads/stores, five CTAs per SM, next tile prefetched into registers
+// before the current one is stored.  The row width is a template parameter:
+// with run-time divisions in the per-vector index arithmetic the kernel was
+// issue-bound (ncu: 61 % issue slots busy at 60 % of DRAM throughput).
+// (Measured alternatives that were slower on B200: per-row bulk async copies,
+// 256 bytes each, are limited by the copy engine's request rate; a cp.async
+// gather into a shared-memory ring with one bulk store per 16 KB tile.)
 #include "ngc_common.cuh"
 
 namespace ngc {
