@@ -139,6 +139,26 @@ def evict_logprob_scan(logits, n, n_protect, budget, kept_order):
     return _logprob(lib().ngc_oracle_evict_logprob_scan, logits, n, n_protect, budget, kept_order)
 
 
+def evict_logprob_grad(logits, n, n_protect, budget, kept_order, grad_logp=None):
+    """d logp / d logits from Eq. (1), term by term.  Returns (grad [NB][B][G][n_max] float64, rc)."""
+    logits = _c(logits, np.float32)
+    if logits.ndim == 3:
+        logits = logits[None]
+    NB, B, G, n_max = logits.shape
+    kept_order = _c(kept_order, np.int32).reshape(NB, B, G, -1)
+    k_max = kept_order.shape[-1]
+    n = _c(np.broadcast_to(np.asarray(n, np.int32).reshape(-1, B), (NB, B)), np.int32)
+    budget = _c(np.broadcast_to(np.asarray(budget, np.int32).reshape(-1, B), (NB, B)), np.int32)
+    if n_protect is not None:
+        n_protect = _c(np.broadcast_to(np.asarray(n_protect, np.int32).reshape(-1, B), (NB, B)), np.int32)
+    if grad_logp is not None:
+        grad_logp = _c(np.broadcast_to(np.asarray(grad_logp, np.float64), (NB, B, G)), np.float64)
+    out = np.empty((NB, B, G, n_max), np.float64)
+    rc = lib().ngc_oracle_evict_logprob_grad(_p(logits), _p(n), _p(n_protect), _p(budget), _p(kept_order), _p(grad_logp),
+                                             NB, B, G, n_max, k_max, _p(out))
+    return out, rc
+
+
 def _dtype_of(a) -> int:
     if a.dtype == np.float32:
         return F32

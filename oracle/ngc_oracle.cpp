@@ -228,6 +228,51 @@ int ngc_oracle_evict_logprob(const float* logits, const int32_t* n, const int32_
   return worst;
 }
 
+/* Derivative of Eq. (1) with respect to the logits, term by term:
+ *   d/ds_i [ s_sigma_j - log sum_{t in A_j} exp s_t ] = [i == sigma_j] - [i in A_j] exp(s_i) / sum_{t in A_j} exp s_t ,
+ * A_j = candidates not drawn before step j.  One softmax over A_j per step, O(K*N).
+ * grad_logits[li][t] = grad_logp[li] * d logp / d s_t (grad_logp NULL = 1); protected units and
+ * units beyond n[b] get 0; a list that fails validation gets NaN on its first n_max entries. */
+int ngc_oracle_evict_logprob_grad(const float* logits, const int32_t* n, const int32_t* n_protect,
+                                  const int32_t* budget, const int32_t* kept_order, const double* grad_logp,
+                                  int n_batches, int B, int G, int n_max, int k_max, double* grad_logits) {
+  int worst = 0;
+#pragma omp parallel for schedule(dynamic) reduction(max : worst)
+  for (int64_t li = 0; li < (int64_t)n_batches * B * G; ++li) {
+    int64_t outer = li / G;
+    int gi = (int)(li % G);
+    ListView lv;
+    double* g = grad_logits + li * n_max;
+    for (int t = 0; t < n_max; ++t) g[t] = std::numeric_limits<double>::quiet_NaN();
+    if (!list_view(logits, n, n_protect, budget, kept_order, G, n_max, k_max, outer, gi, &lv)) { worst = 1; continue; }
+    int Kp = lv.K - lv.P;
+    bool ok = true;
+    std::vector<uint8_t> gone((size_t)lv.n, 0);
+    for (int j = 0; j < Kp && ok; ++j) {
+      int t = lv.sigma[j];
+      if (t < lv.P || t >= lv.n || gone[t]) ok = false; else gone[t] = 1;
+    }
+    if (!ok) { worst = std::max(worst, 3); continue; }
+    std::fill(gone.begin(), gone.end(), 0);
+    std::vector<long double> acc((size_t)n_max, 0.0L);
+    for (int j = 0; j < Kp; ++j) {
+      long double mx = -std::numeric_limits<long double>::infinity();
+      for (int t = lv.P; t < lv.n; ++t)
+        if (!gone[t]) mx = std::max(mx, (long double)lv.s[t]);
+      long double z = 0.0L;
+      for (int t = lv.P; t < lv.n; ++t)
+        if (!gone[t]) z += expl((long double)lv.s[t] - mx);
+      for (int t = lv.P; t < lv.n; ++t)
+        if (!gone[t]) acc[t] -= expl((long double)lv.s[t] - mx) / z;      /* softmax over A_j */
+      acc[lv.sigma[j]] += 1.0L;
+      gone[lv.sigma[j]] = 1;
+    }
+    double up = grad_logp ? grad_logp[li] : 1.0;
+    for (int t = 0; t < n_max; ++t) g[t] = (double)(acc[t] * (long double)up);
+  }
+  return worst;
+}
+
 /* Remaining-mass scan: rem_j = sum of exp(s_t) over candidates still present
  * at step j = (mass never selected) + (mass of sigma_j..sigma_K).  Built from
  * the tail by addition, so no cancellation when little mass remains. */

@@ -69,6 +69,14 @@ int ngc_oracle_evict_logprob(const float* logits, const int32_t* n, const int32_
                              const int32_t* budget, const int32_t* kept_order,
                              int n_batches, int B, int G, int n_max, int k_max, double* logp);
 
+/* Gradient of Eq. (1) with respect to the logits (the eviction half of the policy-gradient loss of
+ * Section 4.4 differentiates this log-probability), one softmax over the remaining candidates per
+ * step.  grad_logp [n_batches][B][G] (NULL = ones) scales each list; grad_logits
+ * [n_batches][B][G][n_max] double out: 0 for protected units and units beyond n[b]. */
+int ngc_oracle_evict_logprob_grad(const float* logits, const int32_t* n, const int32_t* n_protect,
+                                  const int32_t* budget, const int32_t* kept_order, const double* grad_logp,
+                                  int n_batches, int B, int G, int n_max, int k_max, double* grad_logits);
+
 /* Same quantity through the running remaining-mass scan the paper alludes to
  * after Eq. (1) (O(N)); accumulates the remaining mass by addition from the
  * tail.  Cross-checked against the literal form in the tests. */

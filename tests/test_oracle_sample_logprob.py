@@ -236,3 +236,65 @@ def test_sampler_infinities_and_status():
     s[0, 0, 0] = np.nan
     st = oracle.sample_evict(s, [8], [2], [4], 7, seed=5, rnd=5)[3]
     assert st[0, 0] == 0
+
+
+# ------------------------------------------------------------------ gradient of Eq. (1)
+
+def test_logprob_grad_matches_finite_differences_of_eq1():
+    """The gradient routine against central differences of the (independently pinned) literal Eq. (1)."""
+    rng = np.random.default_rng(5)
+    B, G, n_max = 2, 2, 9
+    logits = rng.normal(0, 1.2, (B, G, n_max)).astype(np.float32)
+    n = np.array([9, 7], np.int32)
+    P = np.array([1, 0], np.int32)
+    K = np.array([5, 3], np.int32)
+    ko = oracle.sample_evict(logits, n, P, K, 5, seed=2, rnd=0)[0]
+    grad, rc = oracle.evict_logprob_grad(logits, n, P, K, ko)
+    assert rc == 0
+    h = 2.0 ** -7
+    for b in range(B):
+        for g in range(G):
+            for t in range(n_max):
+                up, dn = logits.copy(), logits.copy()
+                up[b, g, t] += h
+                dn[b, g, t] -= h
+                fd = (oracle.evict_logprob(up, n, P, K, ko)[0][0, b, g] - oracle.evict_logprob(dn, n, P, K, ko)[0][0, b, g]) / \
+                     (float(up[b, g, t]) - float(dn[b, g, t]))
+                want = fd if P[b] <= t < n[b] else 0.0
+                assert abs(grad[0, b, g, t] - want) < 2e-4, (b, g, t)
+
+
+def test_logprob_grad_closed_forms_and_invariants():
+    from scipy.special import softmax
+    rng = np.random.default_rng(6)
+    n_max = 12
+    logits = rng.normal(0, 1, (3, 1, n_max)).astype(np.float32)
+    n = np.array([12, 10, 12], np.int32)
+    P = np.array([0, 2, 0], np.int32)
+    K = np.array([1, 6, 12], np.int32)
+    ko = oracle.sample_evict(logits, n, P, K, 12, seed=4, rnd=1)[0]
+    grad, rc = oracle.evict_logprob_grad(logits, n, P, K, ko)
+    assert rc == 0
+    # one draw: one-hot minus softmax (textbook)
+    want = -softmax(logits[0, 0].astype(np.float64))
+    want[ko[0, 0, 0]] += 1.0
+    assert np.allclose(grad[0, 0, 0], want, atol=1e-12)
+    # Eq. (1) is invariant to a common shift of the logits: the gradient sums to zero; protected units get none
+    assert np.allclose(grad[0, :, 0].sum(-1), 0.0, atol=1e-12)
+    assert np.all(grad[0, 1, 0, :2] == 0.0) and np.all(grad[0, 1, 0, 10:] == 0.0)
+    # constant logits: drawn at step m -> 1 - sum_{j<=m} 1/(N-j+1); never drawn -> -sum_{j<=K} 1/(N-j+1)
+    const = np.full((1, 1, 10), 0.7, np.float32)
+    order = np.array([[[3, 9, 0, 5]]], np.int32)
+    g2, rc = oracle.evict_logprob_grad(const, [10], None, [4], order)
+    H = np.cumsum(1.0 / (10 - np.arange(4)))
+    want = np.full(10, -H[3])
+    for m, t in enumerate(order[0, 0]):
+        want[t] = 1.0 - H[m]
+    assert rc == 0 and np.allclose(g2[0, 0, 0], want, atol=1e-12)
+    # upstream gradient scales the list; invalid list -> NaN
+    g3, _ = oracle.evict_logprob_grad(const, [10], None, [4], order, grad_logp=np.array([[[-2.5]]]))
+    assert np.allclose(g3, -2.5 * g2)
+    bad = order.copy()
+    bad[0, 0, 1] = 3
+    g4, rc = oracle.evict_logprob_grad(const, [10], None, [4], bad)
+    assert rc == 3 and np.isnan(g4).all()
