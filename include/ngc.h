@@ -173,6 +173,24 @@ int ngc_evict_logprob(const float* logits, const int32_t* n, const int32_t* n_pr
                       void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
 
 /*
+ * Gradient of that log-probability with respect to the logits -- what the
+ * eviction half of the policy-gradient loss (Section 4.4, L_mem: the sum over
+ * layers and rounds of -log pi(sigma) * advantage) sends back into the scores:
+ *   d log p / d s_i = [i in sigma] - exp(s_i) * sum_{j : i not drawn before step j} 1 / rem_j ,
+ * rem_j = the mass still present at step j (the same scan as the forward call).
+ *   grad_logp   fp64 [n_batches][B][G] upstream gradient per list, or NULL (= 1)
+ *   grad_logits fp32 [n_batches][B][G][n_max] out; every entry of a list is
+ *               written: 0 for protected units and units >= n[b], NaN for a
+ *               list reported in *dev_status.
+ * Other arguments as in ngc_evict_logprob.  Lists with more than about 24 K
+ * drawn units are refused with NGC_ERR_UNSUPPORTED.
+ */
+int ngc_evict_logprob_backward(const float* logits, const int32_t* n, const int32_t* n_protect,
+                               const int32_t* budget, const int32_t* kept_order, const double* grad_logp,
+                               int n_batches, int B, int G, int n_max, int k_max, float* grad_logits,
+                               void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
+
+/*
  * Physical eviction -- Section 4.1 ("permanently evicts the rest").  In place:
  * in every (layer, KV head, sequence) strip of K and V the tokens of the kept
  * units move to the front in ascending original order, and lens[b] becomes

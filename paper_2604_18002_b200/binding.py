@@ -25,7 +25,7 @@ DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "
               5: "lists disagree", 6: "timeout"}
 
 EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
-           "ngc_sample_evict", "ngc_evict_logprob", "ngc_compact_kv", "ngc_decode_attn_ragged",
+           "ngc_sample_evict", "ngc_evict_logprob", "ngc_evict_logprob_backward", "ngc_compact_kv", "ngc_decode_attn_ragged",
            "ngc_decode_attn_ragged_static"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -62,6 +62,8 @@ def _load():
     lib.ngc_sample_evict.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, u64, u64, u32, i32, vp, vp, vp, vp, sz, vp, vp]
     lib.ngc_evict_logprob.restype = i32
     lib.ngc_evict_logprob.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp, vp]
+    lib.ngc_evict_logprob_backward.restype = i32
+    lib.ngc_evict_logprob_backward.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp, vp]
     lib.ngc_compact_kv.restype = i32
     lib.ngc_compact_kv.argtypes = [C.POINTER(CacheDesc), vp, vp, i32, i32, i32, vp, vp]
     lib.ngc_decode_attn_ragged.restype = i32
@@ -203,6 +205,21 @@ def ngc_evict_logprob(logits: torch.Tensor, n: torch.Tensor, n_protect: Optional
     rc = lib.ngc_evict_logprob(_ptr(logits), _ptr(n), _ptr(n_protect), _ptr(budget), _ptr(kept_order),
                                NB, B, G, n_max, k_max, _ptr(logp), None, 0, _ptr(status), _stream())
     _check(rc, "ngc_evict_logprob")
+
+
+def ngc_evict_logprob_backward(logits: torch.Tensor, n: torch.Tensor, n_protect: Optional[torch.Tensor], budget: torch.Tensor,
+                               kept_order: torch.Tensor, grad_logits: torch.Tensor, grad_logp: Optional[torch.Tensor] = None,
+                               status: Optional[torch.Tensor] = None):
+    """grad_logits fp32, same shape as logits; grad_logp fp64 [NB][B][G] or None (= ones)."""
+    if logits.dim() == 3:
+        NB = 1
+        B, G, n_max = logits.shape
+    else:
+        NB, B, G, n_max = logits.shape
+    k_max = kept_order.shape[-1]
+    rc = lib.ngc_evict_logprob_backward(_ptr(logits), _ptr(n), _ptr(n_protect), _ptr(budget), _ptr(kept_order), _ptr(grad_logp),
+                                        NB, B, G, n_max, k_max, _ptr(grad_logits), None, 0, _ptr(status), _stream())
+    _check(rc, "ngc_evict_logprob_backward")
 
 
 def ngc_compact_kv(cache: NgcCache, kept_sorted: torch.Tensor, budget: torch.Tensor, lists: int, block: int = 1,

@@ -123,7 +123,7 @@ __global__ void sample_kernel(SampleParams p) {
   uint32_t* img = nullptr;             // [n_max] key images (radix)
   uint16_t* idx_a = nullptr;           // [n_max] candidate order, ping
   uint16_t* idx_b = nullptr;           // [n_max] pong
-  uint16_t* hist = nullptr;            // [256][n_warps] digit counts, then output offsets
+  uint16_t* hist = nullptr;            // [n_warps][256] digit counts, then output offsets
   unsigned long long* keys = nullptr;  // composite keys (bitonic)
   uint32_t* bitmap;
   if (kRadix) {
@@ -204,16 +204,20 @@ __global__ void sample_kernel(SampleParams p) {
         const bool live = i < seg_hi;
         const uint32_t d = live ? 255u - ((img[src[i]] >> shift) & 255u) : 0u;
         const uint32_t peers = same_digit_lanes(d, live);
-        if (live && (peers & lt_mask) == 0) hist[d * n_warps + warp] += (uint16_t)__popc(peers);
+        if (live && (peers & lt_mask) == 0) hist[warp * 256 + d] += (uint16_t)__popc(peers);
         __syncwarp();
       }
       __syncthreads();
-      // exclusive scan over (digit, warp): 8 consecutive entries per thread
+      // exclusive scan in (digit, warp) order, 8 consecutive entries of that order per thread
+      // (the counters are stored [warp][digit] so that the walks above and below spread over the banks)
       {
-        uint16_t* hp = hist + 8 * tid;
         int c[8], sum = 0;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { c[e] = hp[e]; sum += c[e]; }
+        for (int e = 0; e < 8; ++e) {
+          const int q = 8 * tid + e;
+          c[e] = hist[(q % n_warps) * 256 + q / n_warps];
+          sum += c[e];
+        }
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -225,7 +229,11 @@ __global__ void sample_kernel(SampleParams p) {
         int run = incl - sum;
         for (int w2 = 0; w2 < warp; ++w2) run += s_warp_tot[w2];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { hp[e] = (uint16_t)run; run += c[e]; }
+        for (int e = 0; e < 8; ++e) {
+          const int q = 8 * tid + e;
+          hist[(q % n_warps) * 256 + q / n_warps] = (uint16_t)run;
+          run += c[e];
+        }
       }
       __syncthreads();
       // scatter: rank = offset of (digit, warp) + position inside the group
@@ -235,9 +243,9 @@ __global__ void sample_kernel(SampleParams p) {
         const uint16_t cand = live ? src[i] : (uint16_t)0;
         const uint32_t d = live ? 255u - ((img[cand] >> shift) & 255u) : 0u;
         const uint32_t peers = same_digit_lanes(d, live);
-        if (live) dst[hist[d * n_warps + warp] + __popc(peers & lt_mask)] = cand;
+        if (live) dst[hist[warp * 256 + d] + __popc(peers & lt_mask)] = cand;
         __syncwarp();
-        if (live && (peers & lt_mask) == 0) hist[d * n_warps + warp] += (uint16_t)__popc(peers);
+        if (live && (peers & lt_mask) == 0) hist[warp * 256 + d] += (uint16_t)__popc(peers);
         __syncwarp();
       }
       __syncthreads();

@@ -62,6 +62,26 @@ def gpu_logprob(logits, n, n_protect, budget, kept_order):
     return lp.cpu().numpy(), status_value(st)
 
 
+def gpu_logprob_grad(logits, n, n_protect, budget, kept_order, grad_logp=None):
+    b = ngc()
+    dev = "cuda"
+    lg = np.ascontiguousarray(logits, np.float32)
+    if lg.ndim == 3:
+        lg = lg[None]
+    NB, B, G, n_max = lg.shape
+    ko = np.ascontiguousarray(kept_order, np.int32).reshape(NB, B, G, -1)
+
+    def bc(a):
+        return torch.as_tensor(np.ascontiguousarray(np.broadcast_to(np.asarray(a, np.int32).reshape(-1, B), (NB, B))).copy()).to(dev)
+    out = torch.full((NB, B, G, n_max), 77.0, dtype=torch.float32, device=dev)
+    up = None if grad_logp is None else torch.as_tensor(np.ascontiguousarray(np.broadcast_to(grad_logp, (NB, B, G)), np.float64).copy()).to(dev)
+    st = b.new_status()
+    b.ngc_evict_logprob_backward(torch.as_tensor(lg).to(dev), bc(n), None if n_protect is None else bc(n_protect), bc(budget),
+                                 torch.as_tensor(ko).to(dev), out, up, status=st)
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), status_value(st)
+
+
 def max_rel_err_per_vector(got: np.ndarray, ref: np.ndarray) -> float:
     """max over (.., head) vectors of ||got - ref||_inf / ||ref||_inf."""
     num = np.abs(got.astype(np.float64) - ref).max(-1)

@@ -9,7 +9,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import gpu_logprob, gpu_sample, max_rel_err_per_vector, ngc, status_value, to_device_cache
+from helpers import gpu_logprob, gpu_logprob_grad, gpu_sample, max_rel_err_per_vector, ngc, status_value, to_device_cache
 from paper_2604_18002_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -450,3 +450,50 @@ def test_tiny_lists_status_paths():
     logits[0, 1, 3] = np.nan
     lp, st = gpu_logprob(logits, n, None, K, ko)
     assert st == 2 and math.isnan(lp[0, 0, 1]) and abs(lp[0, 1, 0] - good[0, 1, 0]) < 1e-9
+
+
+# ------------------------------------------------------------------ gradient of the log-prob
+
+TOL_GRAD = 2e-6      # fp32 output of an fp64 computation; entries are O(1)
+
+
+@pytest.mark.parametrize("NB,B,G,n_max,frac", [(1, 3, 2, 700, 0.5), (3, 2, 2, 768, 1 / 3), (1, 2, 1, 4096, 0.5), (1, 1, 2, 16384, 0.5),
+                                                (2, 2, 1, 40, 1.0), (2, 9, 28, 16, 0.5), (1, 7, 28, 22, 0.5), (1, 4, 1, 32, 0.25)])
+def test_logprob_grad_matches_oracle(NB, B, G, n_max, frac):
+    rng = np.random.default_rng(n_max + 7 * NB)
+    logits = synth.make_logits(NB * B, G, n_max, seed=n_max + 1, std=1.5).numpy().reshape(NB, B, G, n_max)
+    n = rng.integers(max(1, n_max // 2), n_max + 1, (NB, B)).astype(np.int32)
+    P = rng.integers(0, 3, (NB, B)).astype(np.int32)
+    P = np.minimum(P, n)
+    K = np.minimum(n, np.maximum(P, np.ceil(n * frac).astype(np.int32)))
+    k_max = int(K.max())
+    ko = np.stack([oracle.sample_evict(logits[r], n[r], P[r], K[r], k_max, seed=3, rnd=r)[0] for r in range(NB)])
+    up = rng.normal(0, 1, (NB, B, G))
+    ref, rc = oracle.evict_logprob_grad(logits, n, P, K, ko, grad_logp=up)
+    assert rc == 0
+    got, st = gpu_logprob_grad(logits, n, P, K, ko, grad_logp=up)
+    assert st == 0
+    assert np.max(np.abs(got - ref)) <= TOL_GRAD
+    # no upstream gradient given = ones; every entry written (padding and protected units are zero)
+    got1, st = gpu_logprob_grad(logits, n, P, K, ko)
+    ref1, _ = oracle.evict_logprob_grad(logits, n, P, K, ko)
+    assert st == 0 and np.max(np.abs(got1 - ref1)) <= TOL_GRAD
+    assert np.max(np.abs(got1.sum(-1))) <= 1e-4                     # shift invariance of Eq. (1)
+
+
+@pytest.mark.parametrize("n_max", [20, 300])
+def test_logprob_grad_bad_lists(n_max):
+    logits = synth.make_logits(3, 1, n_max, seed=1).numpy()
+    n = np.array([n_max, n_max - 3, n_max], np.int32)
+    K = np.array([n_max // 2, n_max // 4, n_max // 2], np.int32)
+    ko = oracle.sample_evict(logits, n, None, K, int(K.max()), seed=8, rnd=0)[0]
+    good = oracle.evict_logprob_grad(logits, n, None, K, ko)[0]
+    bad = ko.copy()
+    bad[1, 0, 1] = bad[1, 0, 0]                                      # repeated unit
+    got, st = gpu_logprob_grad(logits, n, None, K, bad)
+    assert st == 3 and np.isnan(got[0, 1, 0]).all() and np.max(np.abs(got[0, 0] - good[0, 0])) <= TOL_GRAD
+    got, st = gpu_logprob_grad(logits, n, None, np.array([n_max + 1, K[1], K[2]], np.int32), ko)
+    assert st == 1 and np.isnan(got[0, 0, 0]).all()
+    logits[2, 0, 5] = np.nan
+    got, st = gpu_logprob_grad(logits, n, None, K, ko)
+    assert st == 2 and np.isnan(got[0, 2, 0]).all() and np.max(np.abs(got[0, 1] - good[0, 1])) <= TOL_GRAD
