@@ -223,6 +223,54 @@ int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* new_k, const
                            void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
 
 /*
+ * Paged variant -- Section 4.2 notes that block-level eviction "maps naturally
+ * onto paged KV cache systems": with one eviction unit = one page, evicting is
+ * an edit of a page table and no K/V row moves.
+ *
+ *   k, v       : [L][Hkv][B * pages_cap][page][d] elements (bf16, d = 128)
+ *   page_table : int32 [B][G][pages_cap]; the j-th page of tokens of list gi of
+ *                sequence b lives in physical page  b * pages_cap + page_table[b][gi][j]
+ *                of every (layer, KV head) plane the list covers.  Each row of the
+ *                table is a permutation of 0 .. pages_cap-1: entries at and beyond
+ *                ceil(lens[b] / page) name the sequence's free pages.
+ *   lens       : int32 [B] alive tokens (same for every list of b)
+ *   lists      : ngc_lists, fixes G and which planes a list covers
+ *   page       : tokens per page, 32 or 64
+ */
+typedef struct {
+  void* k;
+  void* v;
+  int32_t* page_table;
+  int32_t* lens;
+  int32_t L, B, Hq, Hkv, d;
+  int32_t dtype;
+  int32_t page, pages_cap, lists;
+} ngc_paged_cache;
+
+/*
+ * Eviction on a paged cache: for every list the pages named by kept_sorted
+ * (ascending unit = page indices, as written by ngc_sample_evict) move to the
+ * front of the list's page-table row in that order, the other pages follow as
+ * free pages, and lens[b] becomes the number of kept tokens (a partly filled
+ * last page stays last if it is kept).  No K/V row is touched.  A corrupt list
+ * leaves its row and lens[b] unchanged and is reported in *dev_status.
+ */
+int ngc_evict_pages(ngc_paged_cache* c, const int32_t* kept_sorted, const int32_t* budget, int k_max,
+                    int32_t* dev_status, ngc_stream stream);
+
+/*
+ * ngc_decode_attn_ragged over a paged cache: same arguments, results and
+ * append semantics; the token tiles are fetched page by page through the
+ * table.  The appended row goes to position lens[b] of the list's pages (a
+ * sequence is full at pages_cap * page tokens).  Workspace as for
+ * NGC_OP_DECODE of a cache with the same L, B, Hq, Hkv.
+ */
+int ngc_decode_attn_paged(ngc_paged_cache* c, const void* q, const void* new_k, const void* new_v,
+                          int layer_begin, int layer_end, float scale,
+                          void* out, int out_dtype,
+                          void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
+
+/*
  * ngc_decode_attn_ragged without a caller-supplied workspace.  (The paper has
  * no counterpart: this entry exists for the library's users, not the method.)
  *

@@ -26,7 +26,7 @@ DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "
 
 EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
            "ngc_sample_evict", "ngc_evict_logprob", "ngc_evict_logprob_backward", "ngc_compact_kv", "ngc_decode_attn_ragged",
-           "ngc_decode_attn_ragged_static"]
+           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -39,6 +39,13 @@ class CacheDesc(C.Structure):
     _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("seq_off", C.c_void_p), ("lens", C.c_void_p),
                 ("rows", C.c_int64), ("L", C.c_int32), ("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
                 ("d", C.c_int32), ("dtype", C.c_int32), ("max_len", C.c_int32)]
+
+
+class PagedCacheDesc(C.Structure):
+    """Mirror of ``ngc_paged_cache``."""
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("page_table", C.c_void_p), ("lens", C.c_void_p),
+                ("L", C.c_int32), ("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32),
+                ("dtype", C.c_int32), ("page", C.c_int32), ("pages_cap", C.c_int32), ("lists", C.c_int32)]
 
 
 def _load():
@@ -70,6 +77,10 @@ def _load():
     lib.ngc_decode_attn_ragged.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, sz, vp, vp]
     lib.ngc_decode_attn_ragged_static.restype = i32
     lib.ngc_decode_attn_ragged_static.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, vp]
+    lib.ngc_evict_pages.restype = i32
+    lib.ngc_evict_pages.argtypes = [C.POINTER(PagedCacheDesc), vp, vp, i32, vp, vp]
+    lib.ngc_decode_attn_paged.restype = i32
+    lib.ngc_decode_attn_paged.argtypes = [C.POINTER(PagedCacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, sz, vp, vp]
     return lib
 
 
@@ -262,3 +273,49 @@ def ngc_decode_attn_ragged_static(cache: NgcCache, q: torch.Tensor, out: torch.T
     rc = lib.ngc_decode_attn_ragged_static(C.byref(d), _ptr(q), _ptr(new_k), _ptr(new_v), layer_begin, layer_end,
                                            scale, _ptr(out), _dtype_code(out), _ptr(status), _stream())
     _check(rc, "ngc_decode_attn_ragged_static")
+
+
+@dataclass
+class NgcPagedCache:
+    """Paged device K/V cache: one eviction unit = one page; eviction edits ``page_table`` only."""
+    k: torch.Tensor           # [L][Hkv][B * pages_cap][page][d] bf16
+    v: torch.Tensor
+    page_table: torch.Tensor  # int32 [B][G][pages_cap], each row a permutation of 0..pages_cap-1
+    lens: torch.Tensor        # int32 [B]
+    Hq: int
+    lists: int
+
+    def desc(self) -> PagedCacheDesc:
+        L, Hkv, n_pages, page, d = self.k.shape
+        B, G, pages_cap = self.page_table.shape
+        assert n_pages == B * pages_cap and G == lists_G(self.lists, L, Hkv)
+        return PagedCacheDesc(_ptr(self.k), _ptr(self.v), _ptr(self.page_table), _ptr(self.lens), L, B, self.Hq, Hkv, d,
+                              _dtype_code(self.k), page, pages_cap, self.lists)
+
+    def as_contiguous_desc(self) -> "NgcCache":
+        """Shape-only view for workspace sizing (same L, B, Hq, Hkv)."""
+        L, Hkv, n_pages, page, d = self.k.shape
+        B, _, pages_cap = self.page_table.shape
+        flat = self.k.view(L, Hkv, n_pages * page, d)
+        return NgcCache(flat, flat, torch.zeros(1, dtype=torch.int64, device=self.k.device), self.lens, self.Hq, pages_cap * page)
+
+
+def ngc_evict_pages(cache: NgcPagedCache, kept_sorted: torch.Tensor, budget: torch.Tensor, status: Optional[torch.Tensor] = None):
+    d = cache.desc()
+    rc = lib.ngc_evict_pages(C.byref(d), _ptr(kept_sorted), _ptr(budget), kept_sorted.shape[2], _ptr(status), _stream())
+    _check(rc, "ngc_evict_pages")
+
+
+def ngc_decode_attn_paged(cache: NgcPagedCache, q: torch.Tensor, out: torch.Tensor, new_k: Optional[torch.Tensor] = None,
+                          new_v: Optional[torch.Tensor] = None, layer_begin: int = 0, layer_end: Optional[int] = None,
+                          scale: Optional[float] = None, ws: Optional[torch.Tensor] = None,
+                          status: Optional[torch.Tensor] = None):
+    L, d = cache.k.shape[0], cache.k.shape[4]
+    if layer_end is None:
+        layer_end = L
+    if scale is None:
+        scale = 1.0 / (d ** 0.5)
+    desc = cache.desc()
+    rc = lib.ngc_decode_attn_paged(C.byref(desc), _ptr(q), _ptr(new_k), _ptr(new_v), layer_begin, layer_end, scale,
+                                   _ptr(out), _dtype_code(out), _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
+    _check(rc, "ngc_decode_attn_paged")

@@ -195,6 +195,71 @@ __global__ void compact_lens_kernel(CompactParams p) {
   }
 }
 
+// ---------------------------------------------------------------- paged caches: eviction edits the page table
+//
+// One CTA per sequence, a warp per list.  The warp checks its kept list, then rewrites the
+// list's page-table row: kept pages first, in kept order, the other pages behind them as
+// free pages (relative order kept).  The old row is staged in shared memory; positions come
+// from ballots and popcounts.  When every list of the sequence is valid and they agree on the
+// kept token count, lens[b] is updated.
+
+struct PageEvictParams {
+  int32_t* page_table;     // [B][G][pages_cap]
+  int32_t* lens;
+  const int32_t* kept_sorted;
+  const int32_t* budget;
+  int32_t* dev_status;
+  int B, G, k_max, page, pages_cap;
+};
+
+__global__ void evict_pages_kernel(PageEvictParams p) {
+  extern __shared__ int32_t s_rows[];                  // [n_warps][pages_cap] old table rows
+  __shared__ int s_bad, s_min, s_max;
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  const int len = p.lens[b];
+  const int K = p.budget[b];
+  if (threadIdx.x == 0) { s_bad = 0; s_min = 0x7fffffff; s_max = -1; }
+  __syncthreads();
+  int32_t* old_row = s_rows + warp * p.pages_cap;
+  const int n_units = (len + p.page - 1) / p.page;
+  for (int gi = warp; gi < p.G; gi += n_warps) {
+    const int32_t* kept = p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max;
+    int32_t* row = p.page_table + ((int64_t)b * p.G + gi) * p.pages_cap;
+    const int t = n_units <= p.pages_cap ? validate_list_warp(kept, K, p.k_max, len, p.page) : -1;
+    if (t < 0) {
+      if (lane == 0) { atomicOr(&s_bad, 1); set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); }
+      continue;
+    }
+    if (lane == 0) { atomicMin(&s_min, t); atomicMax(&s_max, t); }
+    for (int j = lane; j < p.pages_cap; j += 32) old_row[j] = row[j];
+    __syncwarp();
+    // kept pages to the front
+    for (int j = lane; j < K; j += 32) row[j] = old_row[kept[j]];
+    // the others behind them: walk the old row 32 entries at a time; an entry is kept iff it
+    // appears in the (ascending) kept list, found by binary search
+    int out = K;
+    for (int j0 = 0; j0 < p.pages_cap; j0 += 32) {
+      const int j = j0 + lane;
+      bool is_free = false;
+      if (j < p.pages_cap) {
+        int lo = 0, hi = K;                              // first kept[x] >= j
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (kept[mid] < j) lo = mid + 1; else hi = mid; }
+        is_free = !(lo < K && kept[lo] == j);
+      }
+      const uint32_t m = __ballot_sync(0xffffffffu, is_free);
+      if (is_free) row[out + __popc(m & ((1u << lane) - 1u))] = old_row[j];
+      out += __popc(m);
+    }
+    __syncwarp();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && !s_bad) {
+    if (s_min != s_max) set_dev_status(p.dev_status, NGC_DEV_LISTS_DISAGREE);
+    else p.lens[b] = s_min;
+  }
+}
+
 }  // namespace
 }  // namespace ngc
 
@@ -227,5 +292,23 @@ extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const in
   int rc = launch_status();
   if (rc != NGC_OK) return rc;
   compact_lens_kernel<<<c->B, p.G > 4 ? 1024 : 128, 0, (cudaStream_t)stream>>>(p);
+  return launch_status();
+}
+
+extern "C" int ngc_evict_pages(ngc_paged_cache* c, const int32_t* kept_sorted, const int32_t* budget, int k_max,
+                               int32_t* dev_status, ngc_stream stream) {
+  using namespace ngc;
+  if (!c || !c->page_table || !c->lens || !kept_sorted || !budget || k_max <= 0 || c->B <= 0 || c->L <= 0 || c->Hkv <= 0 ||
+      c->pages_cap <= 0 || c->page <= 0 || c->lists < 0 || c->lists > 2)
+    return NGC_ERR_INVALID_ARG;
+  PageEvictParams p;
+  p.page_table = c->page_table; p.lens = c->lens; p.kept_sorted = kept_sorted; p.budget = budget; p.dev_status = dev_status;
+  p.B = c->B; p.G = lists_G(c->lists, c->L, c->Hkv); p.k_max = k_max; p.page = c->page; p.pages_cap = c->pages_cap;
+  const int threads = p.G > 4 ? 256 : 32 * (p.G < 1 ? 1 : p.G);
+  const size_t smem = (size_t)(threads / 32) * c->pages_cap * 4;
+  if (smem > 96 * 1024) return NGC_ERR_UNSUPPORTED;
+  if (smem > 48 * 1024)
+    NGC_CUDA_TRY(cudaFuncSetAttribute(evict_pages_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  evict_pages_kernel<<<c->B, threads, smem, (cudaStream_t)stream>>>(p);
   return launch_status();
 }

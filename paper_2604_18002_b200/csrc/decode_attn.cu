@@ -53,14 +53,19 @@ struct DecodeParams {
   int L, B, Hq, Hkv, d, g;
   int layer_begin, n_layers, n_split, append, out_bf16;
   float scale_log2;   // scale * log2(e)
+  // paged layout (page_table != null): rows of a plane = B * pages_cap * page, seq_off unused
+  const int32_t* page_table;   // [B][G][pages_cap]
+  int page, pages_cap, lists, G;
 };
 
 // Visible length of sequence b for this call; -1 if the appended row does not fit.
+__device__ __forceinline__ int64_t seq_capacity(const DecodeParams& p, int b) {
+  return p.page_table ? (int64_t)p.pages_cap * p.page : p.seq_off[b + 1] - p.seq_off[b];
+}
 __device__ __forceinline__ int visible_len(const DecodeParams& p, int b) {
   const int len = p.lens[b];
   if (!p.append) return len;
-  const int64_t cap = p.seq_off[b + 1] - p.seq_off[b];
-  return (len + 1 > cap) ? -1 : len + 1;
+  return (len + 1 > seq_capacity(p, b)) ? -1 : len + 1;
 }
 
 // ---------------------------------------------------------------- lens bump
@@ -71,8 +76,7 @@ __global__ void bump_lens_kernel(DecodeParams p) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= p.B) return;
   const int len = p.lens[b];
-  const int64_t cap = p.seq_off[b + 1] - p.seq_off[b];
-  if (len + 1 <= cap) p.lens[b] = len + 1;
+  if (len + 1 <= seq_capacity(p, b)) p.lens[b] = len + 1;
 }
 
 // ---------------------------------------------------------------- output helpers
@@ -252,6 +256,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
   const int lr = item / (p.Hkv * p.B);
   const int l = p.layer_begin + lr;
   const int g = p.g;
+  const int32_t* table = p.page_table
+      ? p.page_table + ((int64_t)b * p.G + list_of(p.lists, l, h, p.Hkv)) * p.pages_cap : nullptr;
 
   if (tid == 0) {
 #pragma unroll
@@ -286,7 +292,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     // ------------------------------------------------ producer
     if (lane == 0 && n_tiles > 0) {
       const int plane = l * p.Hkv + h;
-      const int row0 = (int)p.seq_off[b];
+      const int row0 = table ? 0 : (int)p.seq_off[b];
+      const int n_sub = table ? kTileT / p.page : 1;          // pages per 64-token tile
+      const int sub_bytes = (kTileT / n_sub) * 128;
       for (int it = 0; it < n_tiles; ++it) {
         const int s = it % kStages;
         if (it >= kStages) {
@@ -294,11 +302,22 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         }
         uint8_t* st = stage_base + s * kStageBytes;
         ptx::mbar_expect_tx(&bar_full[s], kStageBytes);
-        const int y = row0 + (tile_lo + it) * kTileT;
-        ptx::tma_load_3d(st, &map_k, 0, y, plane, &bar_full[s]);
-        ptx::tma_load_3d(st + kBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
-        ptx::tma_load_3d(st + kTileBytes, &map_v, 0, y, plane, &bar_full[s]);
-        ptx::tma_load_3d(st + kTileBytes + kBoxBytes, &map_v, 64, y, plane, &bar_full[s]);
+        for (int sb = 0; sb < n_sub; ++sb) {
+          int y;
+          if (table) {
+            // every table entry names a page of this sequence, free ones included, so a tile that
+            // reaches past the live pages still loads mapped memory (those tokens are masked)
+            const int j = min(p.pages_cap - 1, (tile_lo + it) * n_sub + sb);
+            y = (b * p.pages_cap + table[j]) * p.page;
+          } else {
+            y = row0 + (tile_lo + it) * kTileT;
+          }
+          uint8_t* dst = st + sb * sub_bytes;
+          ptx::tma_load_3d(dst, &map_k, 0, y, plane, &bar_full[s]);
+          ptx::tma_load_3d(dst + kBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
+          ptx::tma_load_3d(dst + kTileBytes, &map_v, 0, y, plane, &bar_full[s]);
+          ptx::tma_load_3d(dst + kTileBytes + kBoxBytes, &map_v, 64, y, plane, &bar_full[s]);
+        }
       }
     }
     __syncwarp();
@@ -347,7 +366,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         const int isv = lane >> 4, c = lane & 15, r = t_new - tile_t0;
         uint8_t* dst = st + isv * kTileBytes + (c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
         *reinterpret_cast<uint4*>(dst) = piece;
-        ((uint4*)(isv ? p.v : p.k))[((int64_t)(l * p.Hkv + h) * p.rows + p.seq_off[b] + t_new) * 16 + c] = piece;
+        const int64_t row = table ? ((int64_t)b * p.pages_cap + table[t_new / p.page]) * p.page + t_new % p.page
+                                  : p.seq_off[b] + t_new;
+        ((uint4*)(isv ? p.v : p.k))[((int64_t)(l * p.Hkv + h) * p.rows + row) * 16 + c] = piece;
         ptx::fence_proxy_async();      // the stage is refilled by TMA later: order this generic write before it
         __syncwarp();
       }
@@ -528,13 +549,16 @@ size_t decode_workspace_bytes(const ngc_cache* c, int layers) {
 
 }  // namespace ngc
 
-extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* new_k, const void* new_v,
-                                      int layer_begin, int layer_end, float scale,
-                                      void* out, int out_dtype,
-                                      void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream_) {
-  using namespace ngc;
-  cudaStream_t stream = (cudaStream_t)stream_;
-  if (!valid_cache(c) || !q || !out || layer_begin < 0 || layer_end > c->L || layer_begin >= layer_end)
+namespace ngc {
+namespace {
+
+// Paged layout of a call (table == nullptr: contiguous strips addressed through seq_off).
+struct PagedView { const int32_t* table; int page, pages_cap, lists; };
+
+int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* new_k, const void* new_v,
+                int layer_begin, int layer_end, float scale, void* out, int out_dtype,
+                void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {
+  if (!q || !out || layer_begin < 0 || layer_end > c->L || layer_begin >= layer_end)
     return NGC_ERR_INVALID_ARG;
   if ((new_k == nullptr) != (new_v == nullptr)) return NGC_ERR_INVALID_ARG;
   if ((((uintptr_t)q | (uintptr_t)new_k | (uintptr_t)new_v | (uintptr_t)out | (uintptr_t)c->k | (uintptr_t)c->v) & 15) != 0)
@@ -552,6 +576,8 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
   p.scale_log2 = scale * 1.4426950408889634f;
   p.n_split = decode_n_split(c, p.n_layers);
   p.part_o = nullptr; p.part_ml = nullptr;
+  p.page_table = pv.table; p.page = pv.page; p.pages_cap = pv.pages_cap; p.lists = pv.lists;
+  p.G = lists_G(pv.lists, c->L, c->Hkv);
   if (p.n_split > 1) {
     const size_t items = (size_t)p.n_layers * c->B * c->Hq * p.n_split;
     const size_t need = align256(items * c->d * 4) + align256(items * 8);
@@ -561,9 +587,11 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
   }
 
   const bool stream_path = c->dtype == NGC_BF16 && c->d == 128 && p.g <= 16 && c->rows < 0x7fffffffLL;
+  if (pv.table && !stream_path) return NGC_ERR_UNSUPPORTED;          // paged caches: bf16, d = 128, groups of up to 16 heads
   if (stream_path) {
     CUtensorMap map_k, map_v;
-    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, kTileT) || !make_kv_map(&map_v, c->v, c->rows, c->L * c->Hkv, kTileT))
+    const int box_rows = pv.table ? pv.page : kTileT;                 // a page is fetched as its own box
+    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, box_rows) || !make_kv_map(&map_v, c->v, c->rows, c->L * c->Hkv, box_rows))
       return NGC_ERR_UNSUPPORTED;
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hkv * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
@@ -590,6 +618,40 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
   if (p.append && layer_end == c->L)
     NGC_CUDA_TRY(launch_pdl(bump_lens_kernel, dim3((c->B + 255) / 256), dim3(256), 0, stream, p));
   return NGC_OK;
+}
+
+}  // namespace
+}  // namespace ngc
+
+extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* new_k, const void* new_v,
+                                      int layer_begin, int layer_end, float scale,
+                                      void* out, int out_dtype,
+                                      void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  using namespace ngc;
+  if (!valid_cache(c)) return NGC_ERR_INVALID_ARG;
+  const PagedView none = {nullptr, 0, 0, NGC_LISTS_SHARED};
+  return decode_impl(c, none, q, new_k, new_v, layer_begin, layer_end, scale, out, out_dtype, ws, ws_bytes, dev_status,
+                     (cudaStream_t)stream);
+}
+
+extern "C" int ngc_decode_attn_paged(ngc_paged_cache* pc, const void* q, const void* new_k, const void* new_v,
+                                     int layer_begin, int layer_end, float scale,
+                                     void* out, int out_dtype,
+                                     void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  using namespace ngc;
+  if (!pc || !pc->k || !pc->v || !pc->page_table || !pc->lens || pc->L <= 0 || pc->B <= 0 || pc->Hq <= 0 || pc->Hkv <= 0 ||
+      pc->Hq % pc->Hkv != 0 || pc->pages_cap <= 0 || (pc->page != 32 && pc->page != 64) || pc->lists < 0 || pc->lists > 2)
+    return NGC_ERR_INVALID_ARG;
+  if (pc->dtype != NGC_BF16 || pc->d != 128) return NGC_ERR_UNSUPPORTED;
+  // the same kernels run on a descriptor whose planes are the page pools
+  ngc_cache c;
+  c.k = pc->k; c.v = pc->v; c.seq_off = nullptr; c.lens = pc->lens;
+  c.rows = (int64_t)pc->B * pc->pages_cap * pc->page;
+  c.L = pc->L; c.B = pc->B; c.Hq = pc->Hq; c.Hkv = pc->Hkv; c.d = pc->d; c.dtype = pc->dtype;
+  c.max_len = pc->pages_cap * pc->page;
+  const PagedView pv = {pc->page_table, pc->page, pc->pages_cap, pc->lists};
+  return decode_impl(&c, pv, q, new_k, new_v, layer_begin, layer_end, scale, out, out_dtype, ws, ws_bytes, dev_status,
+                     (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------- allocation-free variant
