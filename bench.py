@@ -351,19 +351,35 @@ def run_other(args):
     names = ["score", "sample", "logprob", "compact", "decode", "recompute"]
     acc = {n: [] for n in names}
 
+    paged = None
+    if args.paged:
+        # same memory viewed as page pools (one eviction unit = one page): eviction edits the tables only
+        assert loop and block in (32, 64), "--paged needs a block-eviction workload (--config 6 or 7)"
+        pages_cap = (prompt + cadence) // block
+        table = torch.arange(pages_cap, dtype=torch.int32, device=dev).repeat(B, G, 1).contiguous()
+        table0 = table.clone()
+        paged = ngc.NgcPagedCache(ro.cache.k.view(L, Hkv, B * pages_cap, block, d), ro.cache.v.view(L, Hkv, B * pages_cap, block, d),
+                                  table, ro.cache.lens, Hq, lists)
+
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
     def eviction(rnd, t):
         e = [ev() for _ in range(5)]
         e[0].record()
-        ngc.ngc_score_evict(ro.cache, q_recent, ro.block, lists, ro.score_logits, ws=ro.ws_score, status=ro.status)
+        if paged is not None:
+            ngc.ngc_score_evict_paged(paged, q_recent, ro.score_logits, ws=ro.ws_score, status=ro.status)
+        else:
+            ngc.ngc_score_evict(ro.cache, q_recent, ro.block, lists, ro.score_logits, ws=ro.ws_score, status=ro.status)
         e[1].record()
         ngc.ngc_sample_evict(logits, n_t, None, k_t, cfg["noise_seed"], rnd, ro.kept_order, ro.kept_sorted, None, ws=ro.ws_sample, status=ro.status)
         e[2].record()
         ngc.ngc_evict_logprob(logits, n_t, None, k_t, ro.kept_order, ro.logp, status=ro.status)
         e[3].record()
-        ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, lists, block, status=ro.status)
+        if paged is not None:
+            ngc.ngc_evict_pages(paged, ro.kept_sorted, k_t, status=ro.status)
+        else:
+            ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, lists, block, status=ro.status)
         e[4].record()
         ro.launches += 7          # score 3, sample 1, log-prob 1, compaction 2
         t.append(e)
@@ -372,7 +388,11 @@ def run_other(args):
         e0, e1 = ev(), ev()
         e0.record()
         for s in range(n):
-            ro.decode_step(q[s % ring], out[s % ring], nk[s % ring], nv[s % ring])
+            if paged is not None:
+                ngc.ngc_decode_attn_paged(paged, q[s % ring], out[s % ring], nk[s % ring], nv[s % ring], ws=ro.ws_decode, status=ro.status)
+                ro.launches += 2
+            else:
+                ro.decode_step(q[s % ring], out[s % ring], nk[s % ring], nv[s % ring])
         e1.record()
         t.append((e0, e1))
 
@@ -384,6 +404,8 @@ def run_other(args):
 
     def one_step(i, rec):
         ro.cache.lens.copy_(lens0, non_blocking=True)
+        if paged is not None:
+            paged.page_table.copy_(table0, non_blocking=True)
         ev_t, dec_t, rc = [], [], None
         if loop:
             for r in range(rounds):
@@ -446,7 +468,8 @@ def run_other(args):
     cmp_gbs = compact_bytes / (med["compact"] * 1e-3) / 1e9
     result = {"metric": "evict+compact+decode tokens/sec", "value": round(tokens / (ms_per_step * 1e-3), 1), "unit": "tokens/s", "n_gpus": 1,
               "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "dtype": "bf16", "data": "synthetic",
-              "config": {"workload": OTHER_WORKLOADS[cid], "batch": B, "decode_steps": steps, "input_ring": ring},
+              "config": {"workload": OTHER_WORKLOADS[cid], "batch": B, "decode_steps": steps, "input_ring": ring,
+                         "layout": "paged (eviction edits page tables, no K/V movement)" if paged is not None else "contiguous strips, in-place compaction"},
               "per_call_ms": med,
               "roofline": {"bound": "hbm", "kernel": "decode_stream_kernel (all decode calls of a step, launch gaps included)",
                            "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
@@ -541,6 +564,7 @@ def main():
     ap.add_argument("--cpu-decode-steps", type=int, default=48)
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5, 6, 7],
                     help="2 = the benchmark workload (default); 3..7 = the other workloads, one GPU, per-phase timing only")
+    ap.add_argument("--paged", action="store_true", help="--config 6|7 only: paged cache, one eviction unit = one page")
     ap.add_argument("--ring", type=int, default=8, help="distinct decode-input steps kept on the device for --config 3|4|5")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per decode launch from an ncu capture (profiles/)")
     args = ap.parse_args()

@@ -248,6 +248,17 @@ typedef struct {
 } ngc_paged_cache;
 
 /*
+ * ngc_score_evict over a paged cache: units are pages (block = page), the
+ * lists are the cache's own (c->lists); K is read page by page through the
+ * table.  logits [B][G][n_max], n_max >= pages_cap.  Workspace as for
+ * NGC_OP_SCORE of a contiguous cache with rows = B * pages_cap * page and
+ * max_len = pages_cap * page.
+ */
+int ngc_score_evict_paged(const ngc_paged_cache* c, const void* q_recent, int w, int log_transform,
+                          float* logits, int n_max, void* ws, size_t ws_bytes, int32_t* dev_status,
+                          ngc_stream stream);
+
+/*
  * Eviction on a paged cache: for every list the pages named by kept_sorted
  * (ascending unit = page indices, as written by ngc_sample_evict) move to the
  * front of the list's page-table row in that order, the other pages follow as

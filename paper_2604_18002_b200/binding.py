@@ -26,7 +26,7 @@ DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "
 
 EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
            "ngc_sample_evict", "ngc_evict_logprob", "ngc_evict_logprob_backward", "ngc_compact_kv", "ngc_decode_attn_ragged",
-           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged"]
+           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -77,6 +77,8 @@ def _load():
     lib.ngc_decode_attn_ragged.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, sz, vp, vp]
     lib.ngc_decode_attn_ragged_static.restype = i32
     lib.ngc_decode_attn_ragged_static.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, vp]
+    lib.ngc_score_evict_paged.restype = i32
+    lib.ngc_score_evict_paged.argtypes = [C.POINTER(PagedCacheDesc), vp, i32, i32, vp, i32, vp, sz, vp, vp]
     lib.ngc_evict_pages.restype = i32
     lib.ngc_evict_pages.argtypes = [C.POINTER(PagedCacheDesc), vp, vp, i32, vp, vp]
     lib.ngc_decode_attn_paged.restype = i32
@@ -319,3 +321,12 @@ def ngc_decode_attn_paged(cache: NgcPagedCache, q: torch.Tensor, out: torch.Tens
     rc = lib.ngc_decode_attn_paged(C.byref(desc), _ptr(q), _ptr(new_k), _ptr(new_v), layer_begin, layer_end, scale,
                                    _ptr(out), _dtype_code(out), _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
     _check(rc, "ngc_decode_attn_paged")
+
+
+def ngc_score_evict_paged(cache: NgcPagedCache, q_recent: torch.Tensor, logits: torch.Tensor, log_transform: int = 0,
+                          ws: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
+    """q_recent [L][B][Hq][w][d] -> logits [B][G][n_max] fp32 (units = pages)."""
+    d = cache.desc()
+    rc = lib.ngc_score_evict_paged(C.byref(d), _ptr(q_recent), q_recent.shape[3], log_transform, _ptr(logits), logits.shape[2],
+                                   _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
+    _check(rc, "ngc_score_evict_paged")

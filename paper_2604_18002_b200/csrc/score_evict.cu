@@ -47,7 +47,15 @@ struct ScoreParams {
   int n_chunks, block, lists, G, n_max, log_transform;
   int n_split;       // token ranges per strip (streaming path)
   float inv_sqrt_d;
+  // paged layout (page_table != null): K rows of a plane = B * pages_cap * page, seq_off unused;
+  // psi is indexed by logical token: sequence b starts at b * pages_cap * page
+  const int32_t* page_table;   // [B][G_tab][pages_cap]
+  int page, pages_cap, tab_lists, tab_G;
 };
+
+__device__ __forceinline__ int64_t psi_row0(const ScoreParams& p, int b) {
+  return p.page_table ? (int64_t)b * p.pages_cap * p.page : p.seq_off[b];
+}
 
 template <typename T> __device__ __forceinline__ void load8(const T* p, float (&x)[8]);
 template <> __device__ __forceinline__ void load8<float>(const float* p, float (&x)[8]) {
@@ -257,7 +265,11 @@ score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, fl
     if (lane == 0 && n_tiles > 0) {
       ptx::prefetch_tensormap(&map_k);
       const int plane = l * p.Hkv + h;
-      const int row0 = (int)p.seq_off[b];
+      const int32_t* table = p.page_table
+          ? p.page_table + ((int64_t)b * p.tab_G + list_of(p.tab_lists, l, h, p.Hkv)) * p.pages_cap : nullptr;
+      const int row0 = table ? 0 : (int)p.seq_off[b];
+      const int n_sub = table ? kSTileT / p.page : 1;          // pages per 64-token tile
+      const int sub_bytes = (kSTileT / n_sub) * 128;
       for (int it = 0; it < n_tiles; ++it) {
         const int s = it % kSStages;
         if (it >= kSStages) {
@@ -265,9 +277,17 @@ score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, fl
         }
         uint8_t* sp = stage_base + s * kSStageBytes;
         ptx::mbar_expect_tx(&bar_full[s], kSStageBytes);
-        const int y = row0 + (tile_lo + it) * kSTileT;
-        ptx::tma_load_3d(sp, &map_k, 0, y, plane, &bar_full[s]);
-        ptx::tma_load_3d(sp + kSBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
+        for (int sb = 0; sb < n_sub; ++sb) {
+          int y;
+          if (table) {
+            const int j = min(p.pages_cap - 1, (tile_lo + it) * n_sub + sb);   // free pages are mapped too
+            y = (b * p.pages_cap + table[j]) * p.page;
+          } else {
+            y = row0 + (tile_lo + it) * kSTileT;
+          }
+          ptx::tma_load_3d(sp + sb * sub_bytes, &map_k, 0, y, plane, &bar_full[s]);
+          ptx::tma_load_3d(sp + sb * sub_bytes + kSBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
+        }
       }
     }
     __syncwarp();
@@ -314,7 +334,7 @@ score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, fl
       }
     const uint32_t a_lane_off = (uint32_t)((16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * 128);
     const uint32_t x7 = (uint32_t)(lane & 7);
-    float* psi_strip = p.psi + (int64_t)(l * p.Hkv + h) * p.rows_R + p.seq_off[b];
+    float* psi_strip = p.psi + (int64_t)(l * p.Hkv + h) * p.rows_R + psi_row0(p, b);
 
     for (int it = 0; it < n_tiles; ++it) {
       const int s = it % kSStages;
@@ -435,7 +455,7 @@ __global__ void __launch_bounds__(256) score_finish_kernel(ScoreParams p) {
   for (int t = t0; t < t1; ++t) {
     float m = 0.f;
     for (int l = l0; l < l1; ++l)
-      for (int h = h0; h < h1; ++h) m += p.psi[(int64_t)(l * p.Hkv + h) * p.rows_R + p.seq_off[b] + t];
+      for (int h = h0; h < h1; ++h) m += p.psi[(int64_t)(l * p.Hkv + h) * p.rows_R + psi_row0(p, b) + t];
     acc += m / n_rows_list;
   }
   const float s = acc / (float)(t1 - t0);
@@ -493,12 +513,15 @@ size_t score_workspace_bytes(const ngc_cache* c, int G, int n_max) {
 
 }  // namespace ngc
 
-extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, int lists,
-                               int log_transform, float* logits, int n_max,
-                               void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream_) {
-  using namespace ngc;
-  cudaStream_t stream = (cudaStream_t)stream_;
-  if (!valid_cache(c) || !q_recent || !logits || w <= 0 || w > 16 || block <= 0 || lists < 0 || lists > 2 || n_max <= 0)
+namespace ngc {
+namespace {
+
+struct PagedView { const int32_t* table; int page, pages_cap, lists; };
+
+int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, int w, int block, int lists,
+               int log_transform, float* logits, int n_max,
+               void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {
+  if (!q_recent || !logits || w <= 0 || w > 16 || block <= 0 || lists < 0 || lists > 2 || n_max <= 0)
     return NGC_ERR_INVALID_ARG;
   const int g = c->Hq / c->Hkv;
   if (g * w > 128) return NGC_ERR_UNSUPPORTED;
@@ -517,15 +540,19 @@ extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, 
   p.block = block; p.lists = lists; p.G = lists_G(lists, c->L, c->Hkv); p.n_max = n_max;
   p.log_transform = log_transform;
   p.inv_sqrt_d = 1.0f / sqrtf((float)c->d);
+  p.page_table = pv.table; p.page = pv.page; p.pages_cap = pv.pages_cap; p.tab_lists = pv.lists;
+  p.tab_G = lists_G(pv.lists, c->L, c->Hkv);
 
   p.n_split = 1;
   int rc;
-  if (score_stream_shape(c, w) && ((uintptr_t)c->k & 15) == 0 && ((uintptr_t)q_recent & 3) == 0) {
+  const bool stream_ok = score_stream_shape(c, w) && ((uintptr_t)c->k & 15) == 0 && ((uintptr_t)q_recent & 3) == 0;
+  if (pv.table && !stream_ok) return NGC_ERR_UNSUPPORTED;      // paged caches: bf16, d = 128, at most 40 rows per strip
+  if (stream_ok) {
     p.n_split = score_n_split(c);
     const int64_t ctas = (int64_t)c->L * c->B * c->Hkv * p.n_split;
     if (ctas > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
     CUtensorMap map_k;
-    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, kSTileT)) return NGC_ERR_UNSUPPORTED;
+    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, pv.table ? pv.page : kSTileT)) return NGC_ERR_UNSUPPORTED;
     const float scale_log2 = p.inv_sqrt_d * 1.4426950408889634f;
     const unsigned grid = (unsigned)ctas;
     switch ((p.n_rows + 7) / 8) {
@@ -564,4 +591,34 @@ extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, 
   if (fgrid.y > 65535) return NGC_ERR_UNSUPPORTED;
   score_finish_kernel<<<fgrid, 256, 0, stream>>>(p);
   return launch_status();
+}
+
+}  // namespace
+}  // namespace ngc
+
+extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, int lists,
+                               int log_transform, float* logits, int n_max,
+                               void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  using namespace ngc;
+  if (!valid_cache(c)) return NGC_ERR_INVALID_ARG;
+  const PagedView none = {nullptr, 0, 0, NGC_LISTS_SHARED};
+  return score_impl(c, none, q_recent, w, block, lists, log_transform, logits, n_max, ws, ws_bytes, dev_status, (cudaStream_t)stream);
+}
+
+extern "C" int ngc_score_evict_paged(const ngc_paged_cache* pc, const void* q_recent, int w, int log_transform,
+                                     float* logits, int n_max, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                     ngc_stream stream) {
+  using namespace ngc;
+  if (!pc || !pc->k || !pc->page_table || !pc->lens || pc->L <= 0 || pc->B <= 0 || pc->Hq <= 0 || pc->Hkv <= 0 ||
+      pc->Hq % pc->Hkv != 0 || pc->pages_cap <= 0 || (pc->page != 32 && pc->page != 64) || pc->lists < 0 || pc->lists > 2)
+    return NGC_ERR_INVALID_ARG;
+  if (pc->dtype != NGC_BF16 || pc->d != 128) return NGC_ERR_UNSUPPORTED;
+  ngc_cache c;
+  c.k = pc->k; c.v = pc->v; c.seq_off = nullptr; c.lens = pc->lens;
+  c.rows = (int64_t)pc->B * pc->pages_cap * pc->page;
+  c.L = pc->L; c.B = pc->B; c.Hq = pc->Hq; c.Hkv = pc->Hkv; c.d = pc->d; c.dtype = pc->dtype;
+  c.max_len = pc->pages_cap * pc->page;
+  const PagedView pv = {pc->page_table, pc->page, pc->pages_cap, pc->lists};
+  return score_impl(&c, pv, q_recent, w, pc->page, pc->lists, log_transform, logits, n_max, ws, ws_bytes, dev_status,
+                    (cudaStream_t)stream);
 }

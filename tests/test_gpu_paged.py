@@ -107,6 +107,22 @@ def test_paged_evict_and_decode_match_oracle(page, lists, lens):
     assert max_rel_err_per_vector(out.cpu().numpy().astype(np.float64), ref) <= 2e-2
     decode_steps(3, 10)
 
+    # scores through the page table against the oracle's scores of the contiguous cache (units = pages)
+    w = 5
+    qr = synth.normal((L, B, Hq, w, d), 77, dtype)
+    ref_s = oracle.score_evict(k_ref, so, o_lens, synth.to_numpy(qr), page, lists, n_max=pages_cap)
+    lg = torch.full((B, G, pages_cap), -5.0, dtype=torch.float32, device="cuda")
+    ws_s = b.alloc_workspace(b.workspace_bytes(b.OP_SCORE, pc.as_contiguous_desc(), G, pages_cap))
+    b.ngc_score_evict_paged(pc, qr.cuda(), lg, ws=ws_s, status=st)
+    torch.cuda.synchronize()
+    got_s = lg.cpu().numpy().astype(np.float64)
+    live = ~np.isnan(ref_s)
+    assert status_value(st) == 0 and np.all(got_s[~live] == -5.0)
+    for bb in range(B):
+        for g in range(G):
+            m = live[bb, g]
+            assert np.max(np.abs(got_s[bb, g][m] - ref_s[bb, g][m])) <= 2e-2 * ref_s[bb, g][m].max()
+
     # one eviction round: units are pages; keep about half
     n_units = (o_lens + page - 1) // page
     budget = np.maximum(1, (n_units + 1) // 2).astype(np.int32)
