@@ -1,0 +1,110 @@
+"""Pins of the replay-visibility oracle (paper Appendix A.3 and the replay-mask figure of
+Section 4.5): the figure's printed example, a token-by-token simulation of the cache with Python
+sets, block-level units with a short last unit, and the steady-state alive-set size of the
+proposition in Appendix A.2."""
+import json
+import os
+
+import numpy as np
+
+from oracle import replay
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "replay_mask_figure.json")
+
+
+def units_from_evicted(alive, evicted):
+    """Ascending compacted indices of the entries of `alive` that are not evicted (block = 1)."""
+    return [i for i, t in enumerate(alive) if t not in evicted]
+
+
+def test_figure_example_rows_and_survivors():
+    g = json.load(open(GOLDEN))
+    T = g["tokens"]
+    total_before = [r["after_token"] + 1 for r in g["rounds"]]                   # [5, 8]
+    alive = list(range(total_before[0]))                                         # A_0 = block_0
+    kept_lists, alive_before = [], []
+    for i, r in enumerate(g["rounds"]):
+        alive_before.append(len(alive))
+        kept_lists.append(units_from_evicted(alive, set(r["evicts"])))
+        alive = [alive[j] for j in kept_lists[-1]]
+        if i + 1 < len(total_before):
+            alive += list(range(total_before[i], total_before[i + 1]))          # block_{r+1}
+    k_max = max(len(k) for k in kept_lists)
+    ks = np.full((2, 1, 1, k_max), -1, np.int32)
+    for r, k in enumerate(kept_lists):
+        ks[r, 0, 0, : len(k)] = k
+    pos, count, rc = replay.alive_positions(ks, [[len(k)] for k in kept_lists], [[a] for a in alive_before],
+                                            [[t] for t in total_before])
+    assert rc == 0
+    assert list(pos[0, 0, 0, : count[0, 0, 0]]) == [0, 2, 4]                     # round 1 evicts t1, t3
+    assert list(pos[1, 0, 0, : count[1, 0, 0]]) == g["final_survivors"]          # round 2 evicts t2, t5
+    M = replay.dense_mask(T, total_before, [pos[r, 0, 0, : count[r, 0, 0]] for r in range(2)])
+    for row, vis in g["visible"].items():
+        assert list(np.nonzero(M[int(row)])[0]) == vis
+    for t in range(total_before[0]):                                             # before the first round: plain causal
+        assert list(np.nonzero(M[t])[0]) == list(range(t + 1))
+
+
+def simulate_with_sets(T, boundaries, decisions):
+    """Token-by-token cache simulation: visible[t] = the alive set when token t is generated (itself
+    included); at a boundary the decision (set of evicted original positions) is applied."""
+    alive, vis = set(), []
+    for t in range(T):
+        alive.add(t)
+        vis.append(set(alive))
+        if t + 1 in boundaries:
+            alive -= decisions[boundaries.index(t + 1)]
+    return vis
+
+
+def test_dense_mask_equals_set_simulation_random_blocks():
+    rng = np.random.default_rng(3)
+    for trial in range(20):
+        block = int(rng.choice([1, 1, 2, 4]))
+        R = int(rng.integers(1, 5))
+        grows = [int(rng.integers(2, 9)) for _ in range(R + 1)]
+        boundaries = list(np.cumsum(grows[:-1]))
+        T = int(sum(grows))
+        alive, kept_lists, alive_before, evicted_sets = list(range(grows[0])), [], [], []
+        for r in range(R):
+            n_units = (len(alive) + block - 1) // block
+            K = int(rng.integers(0, n_units + 1))
+            units = sorted(rng.choice(n_units, K, replace=False).tolist())
+            keep_idx = [i for u in units for i in range(u * block, min((u + 1) * block, len(alive)))]
+            alive_before.append(len(alive))
+            kept_lists.append(units)
+            evicted_sets.append(set(alive) - {alive[i] for i in keep_idx})
+            alive = [alive[i] for i in keep_idx] + list(range(boundaries[r], boundaries[r] + grows[r + 1]))
+        k_max = max(1, max(len(k) for k in kept_lists))
+        ks = np.full((R, 1, 1, k_max), -1, np.int32)
+        for r, k in enumerate(kept_lists):
+            ks[r, 0, 0, : len(k)] = k
+        pos, count, rc = replay.alive_positions(ks, [[len(k)] for k in kept_lists], [[a] for a in alive_before],
+                                                [[int(t)] for t in boundaries], block)
+        assert rc == 0
+        M = replay.dense_mask(T, boundaries, [pos[r, 0, 0, : count[r, 0, 0]] for r in range(R)])
+        vis = simulate_with_sets(T, [int(x) for x in boundaries], evicted_sets)
+        for t in range(T):
+            assert set(np.nonzero(M[t])[0].tolist()) == vis[t], (trial, t)
+
+
+def test_steady_state_alive_size_and_error_codes():
+    # delta = 512 new tokens per round, keep one third of 768: the alive set returns to delta / epsilon = 768
+    R, delta, K = 5, 512, 256
+    rng = np.random.default_rng(1)
+    ks = np.stack([np.sort(rng.choice(768, K, replace=False)) for _ in range(R)]).astype(np.int32).reshape(R, 1, 1, K)
+    pos, count, rc = replay.alive_positions(ks, np.full((R, 1), K), np.full((R, 1), 768), [[768 + r * delta] for r in range(R)])
+    assert rc == 0 and np.all(count == K)
+    for r in range(R):
+        p = pos[r, 0, 0]
+        assert np.all(np.diff(p) > 0) and p.max() < 768 + r * delta
+        if r:
+            assert np.sum(p >= 768 + (r - 1) * delta) == np.sum(ks[r, 0, 0] >= K)     # survivors of the newest block
+    bad = ks.copy()
+    bad[2, 0, 0, 5] = bad[2, 0, 0, 4]
+    _, c2, rc = replay.alive_positions(bad, np.full((R, 1), K), np.full((R, 1), 768), [[768 + r * delta] for r in range(R)])
+    assert rc == 3 and np.all(c2[:2] == K) and np.all(c2[2:] == -1)
+    fewer = np.full((R, 1), 768)
+    fewer[1] = 100                      # fewer tokens alive at round 1 than round 0 kept
+    _, _, rc = replay.alive_positions(ks, np.full((R, 1), K), fewer, [[768 + r * delta] for r in range(R)])
+    assert rc == 1
