@@ -191,6 +191,30 @@ int ngc_evict_logprob_backward(const float* logits, const int32_t* n, const int3
                                void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
 
 /*
+ * Replay visibility -- Appendix A.3 ("Reconstructing Replay Attention Masks
+ * from Retention Decisions") and the replay-mask figure of Section 4.5.  The
+ * training pass must show every token exactly the keys it saw at rollout time:
+ * a query generated after round r sees kept_r (what round r left alive) plus,
+ * causally, the tokens generated since.  This call turns the stored decisions
+ * of all R rounds -- kept units in the coordinates of the cache at that round
+ * -- into kept_r as ORIGINAL token positions, one ascending list per (round,
+ * list), instead of the paper's dense B x T x T masks.
+ *   kept_sorted  [R][B][G][k_max] as written by ngc_sample_evict at round r
+ *   budget       [R][B] kept units;  alive_before [R][B] tokens alive when round
+ *                r fired (lens[b] at that time);  total_before [R][B] sequence
+ *                length when round r fired (the tokens appended since the last
+ *                round are the positions just below it)
+ *   block        tokens per unit;  alive_max (host) >= every alive_before
+ *   alive_pos    [R][B][G][k_max*block] out, ascending, -1 padded
+ *   alive_count  [R][B][G] out (tokens), -1 for a list that failed
+ * A list with inconsistent counts or a corrupt kept list is reported in
+ * *dev_status and gets -1 from the failing round on.
+ */
+int ngc_replay_visibility(const int32_t* kept_sorted, const int32_t* budget, const int32_t* alive_before,
+                          const int32_t* total_before, int R, int B, int G, int k_max, int block, int alive_max,
+                          int32_t* alive_pos, int32_t* alive_count, int32_t* dev_status, ngc_stream stream);
+
+/*
  * Physical eviction -- Section 4.1 ("permanently evicts the rest").  In place:
  * in every (layer, KV head, sequence) strip of K and V the tokens of the kept
  * units move to the front in ascending original order, and lens[b] becomes

@@ -26,7 +26,7 @@ DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "
 
 EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
            "ngc_sample_evict", "ngc_evict_logprob", "ngc_evict_logprob_backward", "ngc_compact_kv", "ngc_decode_attn_ragged",
-           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged"]
+           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged", "ngc_replay_visibility"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -79,6 +79,8 @@ def _load():
     lib.ngc_decode_attn_ragged_static.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, vp]
     lib.ngc_score_evict_paged.restype = i32
     lib.ngc_score_evict_paged.argtypes = [C.POINTER(PagedCacheDesc), vp, i32, i32, vp, i32, vp, sz, vp, vp]
+    lib.ngc_replay_visibility.restype = i32
+    lib.ngc_replay_visibility.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.ngc_evict_pages.restype = i32
     lib.ngc_evict_pages.argtypes = [C.POINTER(PagedCacheDesc), vp, vp, i32, vp, vp]
     lib.ngc_decode_attn_paged.restype = i32
@@ -330,3 +332,13 @@ def ngc_score_evict_paged(cache: NgcPagedCache, q_recent: torch.Tensor, logits: 
     rc = lib.ngc_score_evict_paged(C.byref(d), _ptr(q_recent), q_recent.shape[3], log_transform, _ptr(logits), logits.shape[2],
                                    _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
     _check(rc, "ngc_score_evict_paged")
+
+
+def ngc_replay_visibility(kept_sorted: torch.Tensor, budget: torch.Tensor, alive_before: torch.Tensor, total_before: torch.Tensor,
+                          block: int, alive_max: int, alive_pos: torch.Tensor, alive_count: torch.Tensor,
+                          status: Optional[torch.Tensor] = None):
+    """kept_sorted [R][B][G][k_max] -> alive_pos [R][B][G][k_max*block], alive_count [R][B][G] (int32)."""
+    R, B, G, k_max = kept_sorted.shape
+    rc = lib.ngc_replay_visibility(_ptr(kept_sorted), _ptr(budget), _ptr(alive_before), _ptr(total_before), R, B, G, k_max, block,
+                                   alive_max, _ptr(alive_pos), _ptr(alive_count), _ptr(status), _stream())
+    _check(rc, "ngc_replay_visibility")
