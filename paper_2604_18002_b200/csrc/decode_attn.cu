@@ -237,6 +237,8 @@ constexpr int kBoxBytes = kTileT * 128;       // one 64 x 64 bf16 box
 constexpr int kTileBytes = 2 * kBoxBytes;     // K (or V) tile: two boxes (channels 0-63, 64-127)
 constexpr int kStageBytes = 2 * kTileBytes;   // K + V
 constexpr int kStages = 3;
+constexpr int kTStages = 2;                   // ring depth and CTAs per SM of the variant for groups of <= 8 heads
+constexpr int kTMinCtas = 3;
 constexpr int kORowStride = 132;              // floats; merge buffer row stride (bank spread)
 
 __global__ void __launch_bounds__(kStreamThreads, 2)
@@ -519,6 +521,270 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
   }
 }
 
+// Variant for groups of at most 8 query heads (every GQA shape in the paper's model family).
+template <int kNStages, int kMinCtas>
+__global__ void __launch_bounds__(kStreamThreads, kMinCtas)
+decode_stream_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, DecodeParams p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ uint64_t bar_full[kNStages], bar_empty[kNStages];
+  __shared__ float sm_m[kConsumerWarps][8], sm_l[kConsumerWarps][8];
+
+  uint8_t* stage_base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+
+  int item = blockIdx.x;
+  const int split = item % p.n_split; item /= p.n_split;
+  const int h = item % p.Hkv;
+  const int b = (item / p.Hkv) % p.B;
+  const int lr = item / (p.Hkv * p.B);
+  const int l = p.layer_begin + lr;
+  const int g = p.g;
+  const int32_t* table = p.page_table
+      ? p.page_table + ((int64_t)b * p.G + list_of(p.lists, l, h, p.Hkv)) * p.pages_cap : nullptr;
+
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < kNStages; ++s) { ptx::mbar_init(&bar_full[s], 1); ptx::mbar_init(&bar_empty[s], kConsumerWarps); }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&map_k);
+    ptx::prefetch_tensormap(&map_v);
+  }
+  ptx::grid_dep_wait();           // lens and the cache rows of earlier calls are final from here on
+  ptx::grid_dep_launch();
+
+  int len = visible_len(p, b);
+  if (len < 0) {
+    if (tid == 0) set_dev_status(p.dev_status, NGC_DEV_STRIP_FULL);
+    len = 0;
+  }
+  const int t_new = (p.append && len > 0) ? len - 1 : -1;      // position of the appended row
+  const int nt = (len + kTileT - 1) / kTileT;
+  const int tps = (nt + p.n_split - 1) / p.n_split;
+  const int tile_lo = min(nt, split * tps);
+  const int tile_hi = min(nt, tile_lo + tps);
+  const int n_tiles = tile_hi - tile_lo;
+  __syncthreads();
+
+  // O^T accumulators: o_acc[mt] = channels 16*mt + {gid, gid+8} x heads {2*tig, 2*tig+1}
+  float o_acc[8][4];
+  float m_run[2] = {-INFINITY, -INFINITY};      // running max / sum of heads 2*tig, 2*tig+1 (log2 domain)
+  float l_run[2] = {0.f, 0.f};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { o_acc[i][0] = 0.f; o_acc[i][1] = 0.f; o_acc[i][2] = 0.f; o_acc[i][3] = 0.f; }
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------ producer
+    if (lane == 0 && n_tiles > 0) {
+      const int plane = l * p.Hkv + h;
+      const int row0 = table ? 0 : (int)p.seq_off[b];
+      const int n_sub = table ? kTileT / p.page : 1;          // pages per 64-token tile
+      const int sub_bytes = (kTileT / n_sub) * 128;
+      for (int it = 0; it < n_tiles; ++it) {
+        const int s = it % kNStages;
+        if (it >= kNStages) {
+          if (!ptx::mbar_wait_bounded(&bar_empty[s], ((it / kNStages) - 1) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
+        }
+        uint8_t* st = stage_base + s * kStageBytes;
+        ptx::mbar_expect_tx(&bar_full[s], kStageBytes);
+        for (int sb = 0; sb < n_sub; ++sb) {
+          int y;
+          if (table) {
+            // every table entry names a page of this sequence, free ones included, so a tile that
+            // reaches past the live pages still loads mapped memory (those tokens are masked)
+            const int j = min(p.pages_cap - 1, (tile_lo + it) * n_sub + sb);
+            y = (b * p.pages_cap + table[j]) * p.page;
+          } else {
+            y = row0 + (tile_lo + it) * kTileT;
+          }
+          uint8_t* dst = st + sb * sub_bytes;
+          ptx::tma_load_3d(dst, &map_k, 0, y, plane, &bar_full[s]);
+          ptx::tma_load_3d(dst + kBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
+          ptx::tma_load_3d(dst + kTileBytes, &map_v, 0, y, plane, &bar_full[s]);
+          ptx::tma_load_3d(dst + kTileBytes + kBoxBytes, &map_v, 64, y, plane, &bar_full[s]);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------ consumers
+    // Transposed products: S^T = K Q^T (16 tokens x 8 heads) and O^T = V^T P^T (128 channels x 8
+    // heads), so the at most 8 heads of the group sit on the N = 8 axis of the MMA with no padding.
+    // Q^T fragments (B operand, column n = head gid): zero beyond g.
+    uint32_t qb[8][2];
+    {
+      const uint32_t* q0 = (const uint32_t*)((const __nv_bfloat16*)p.q + (((int64_t)l * p.B + b) * p.Hq + h * g + gid) * 128);
+      const bool live = gid < g;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        qb[ks][0] = live ? q0[8 * ks + tig] : 0u;
+        qb[ks][1] = live ? q0[8 * ks + tig + 4] : 0u;
+      }
+    }
+    // lane-dependent parts of the swizzled shared-memory addresses
+    const uint32_t k_lane_off = (uint32_t)((16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * 128);   // A operand, K rows
+    const uint32_t v_lane_off = (uint32_t)((16 * warp + (lane & 7) + 8 * (lane >> 4)) * 128);         // A operand, V^T
+    const uint32_t x7 = (uint32_t)(lane & 7);
+
+    const bool own_new = t_new >= 0 && tile_hi == nt && n_tiles > 0 && ((t_new % kTileT) >> 4) == warp;
+    uint4 piece = make_uint4(0, 0, 0, 0);
+    if (own_new)
+      piece = ((const uint4*)((lane >> 4) ? p.new_v : p.new_k))[(((int64_t)l * p.B + b) * p.Hkv + h) * 16 + (lane & 15)];
+
+    for (int it = 0; it < n_tiles; ++it) {
+      const int s = it % kNStages;
+      if (!ptx::mbar_wait_bounded(&bar_full[s], (it / kNStages) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
+      uint8_t* st = stage_base + s * kStageBytes;
+      const uint32_t k_st = ptx::smem_u32(st);
+      const uint32_t v_st = k_st + kTileBytes;
+      const int tile_t0 = (tile_lo + it) * kTileT;
+      const int valid = len - tile_t0 - 16 * warp;      // live tokens in this warp's slice (may exceed 16)
+
+      if (own_new && it == n_tiles - 1) {
+        // the appended row: from the caller's buffer into the tile and into the cache
+        const int isv = lane >> 4, c = lane & 15, r = t_new - tile_t0;
+        uint8_t* dst = st + isv * kTileBytes + (c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(dst) = piece;
+        const int64_t row = table ? ((int64_t)b * p.pages_cap + table[t_new / p.page]) * p.page + t_new % p.page
+                                  : p.seq_off[b] + t_new;
+        ((uint4*)(isv ? p.v : p.k))[((int64_t)(l * p.Hkv + h) * p.rows + row) * 16 + c] = piece;
+        ptx::fence_proxy_async();
+        __syncwarp();
+      }
+      if (valid > 0) {
+        if (valid < 16) {
+          // dead V rows may hold anything (NaN x 0 would poison the sum): zero them
+          for (int i = lane; i < 16 * 16; i += 32) {
+            const int r = i >> 4, c = i & 15;
+            if (r >= valid) {
+              uint8_t* rowp = st + kTileBytes + (c >> 3) * kBoxBytes + (16 * warp + r) * 128 + (c & 7) * 16;
+              *reinterpret_cast<uint4*>(rowp) = make_uint4(0, 0, 0, 0);
+            }
+          }
+          __syncwarp();
+        }
+        // ---- S^T = K Q^T: 16 tokens x 8 heads ----
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};     // (tok gid, head 2tig), (gid, 2tig+1), (gid+8, 2tig), (gid+8, 2tig+1)
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t chunk = (uint32_t)(2 * (ks & 3) + (lane >> 4));
+          const uint32_t addr = k_st + (ks >> 2) * kBoxBytes + k_lane_off + ((chunk ^ x7) << 4);
+          uint32_t a[4];
+          ptx::ldmatrix_x4(addr, a[0], a[1], a[2], a[3]);
+          ptx::mma_bf16_16816(sc, a, qb[ks][0], qb[ks][1]);
+        }
+        // ---- online softmax per head (log2 domain) ----
+        sc[0] = gid < valid ? sc[0] * p.scale_log2 : -INFINITY;
+        sc[1] = gid < valid ? sc[1] * p.scale_log2 : -INFINITY;
+        sc[2] = gid + 8 < valid ? sc[2] * p.scale_log2 : -INFINITY;
+        sc[3] = gid + 8 < valid ? sc[3] * p.scale_log2 : -INFINITY;
+        float mx[2] = {fmaxf(sc[0], sc[2]), fmaxf(sc[1], sc[3])};
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 4));
+          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 8));
+          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 16));
+        }
+        float m_new[2], alpha[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          m_new[r] = fmaxf(m_run[r], mx[r]);          // finite: token 0 of the slice is live
+          alpha[r] = ptx::ex2_approx(m_run[r] - m_new[r]);
+        }
+        const bool changed = (m_new[0] != m_run[0]) || (m_new[1] != m_run[1]);
+        if (__any_sync(0xffffffffu, changed)) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            o_acc[i][0] *= alpha[0]; o_acc[i][1] *= alpha[1];
+            o_acc[i][2] *= alpha[0]; o_acc[i][3] *= alpha[1];
+          }
+          l_run[0] *= alpha[0];
+          l_run[1] *= alpha[1];
+          m_run[0] = m_new[0];
+          m_run[1] = m_new[1];
+        }
+        float pr[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          pr[e] = ptx::ex2_approx(sc[e] - m_run[e & 1]);
+          l_run[e & 1] += pr[e];
+        }
+        // P^T as B operand (k = token, n = head): transpose the two 8 x 8 (token x head) blocks
+        const uint32_t pb0 = ptx::movmatrix_trans(ptx::pack_bf16x2(pr[0], pr[1]));
+        const uint32_t pb1 = ptx::movmatrix_trans(ptx::pack_bf16x2(pr[2], pr[3]));
+        // ---- O^T += V^T P^T (128 channels x 8 heads) ----
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          const uint32_t chunk = (uint32_t)(2 * (mt & 3) + ((lane >> 3) & 1));
+          const uint32_t addr = v_st + (mt >> 2) * kBoxBytes + v_lane_off + ((chunk ^ x7) << 4);
+          uint32_t a[4];
+          ptx::ldmatrix_x4_trans(addr, a[0], a[1], a[2], a[3]);
+          ptx::mma_bf16_16816(o_acc[mt], a, pb0, pb1);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&bar_empty[s]);
+    }
+    // row sums over the tokens of the slice (spread over gid), then publish this warp's state
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 4);
+      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 8);
+      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 16);
+    }
+    if (gid == 0) {
+      sm_m[warp][2 * tig] = m_run[0]; sm_m[warp][2 * tig + 1] = m_run[1];
+      sm_l[warp][2 * tig] = l_run[0]; sm_l[warp][2 * tig + 1] = l_run[1];
+    }
+  }
+  __syncthreads();   // every stage has been consumed; the ring is free for the merge buffer
+
+  float* obuf = reinterpret_cast<float*>(stage_base);      // [warp][8 heads][kORowStride]
+  if (warp < kConsumerWarps) {
+    float f[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int row = 2 * tig + r;
+      float mg = sm_m[0][row];
+#pragma unroll
+      for (int w = 1; w < kConsumerWarps; ++w) mg = fmaxf(mg, sm_m[w][row]);
+      f[r] = m_run[r] == -INFINITY ? 0.f : ptx::ex2_approx(m_run[r] - mg);
+    }
+    float* ob = obuf + warp * 8 * kORowStride;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      ob[(2 * tig) * kORowStride + 16 * i + gid] = o_acc[i][0] * f[0];
+      ob[(2 * tig + 1) * kORowStride + 16 * i + gid] = o_acc[i][1] * f[1];
+      ob[(2 * tig) * kORowStride + 16 * i + gid + 8] = o_acc[i][2] * f[0];
+      ob[(2 * tig + 1) * kORowStride + 16 * i + gid + 8] = o_acc[i][3] * f[1];
+    }
+  }
+  __syncthreads();
+  if (tid < 128) {
+    const int c = tid;
+    for (int row = 0; row < g; ++row) {
+      float mg = sm_m[0][row];
+#pragma unroll
+      for (int w = 1; w < kConsumerWarps; ++w) mg = fmaxf(mg, sm_m[w][row]);
+      float o = 0.f, ls = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) {
+        o += obuf[(w * 8 + row) * kORowStride + c];
+        const float mw = sm_m[w][row];
+        ls += mw == -INFINITY ? 0.f : sm_l[w][row] * ptx::ex2_approx(mw - mg);
+      }
+      const int hq = h * g + row;
+      if (p.n_split == 1) {
+        store_out(p, (((int64_t)l * p.B + b) * p.Hq + hq) * 128 + c, ls > 0.f ? o / ls : 0.f);
+      } else {
+        const int64_t pit = (((int64_t)lr * p.B + b) * p.Hq + hq) * p.n_split + split;
+        p.part_o[pit * 128 + c] = o;
+        if (c == 0) p.part_ml[pit] = make_float2(mg, ls);
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------- host side
 
 constexpr int kTargetCtas = 148 * 2 * 2;   // two waves of two CTAs per SM
@@ -595,14 +861,22 @@ int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* ne
       return NGC_ERR_UNSUPPORTED;
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hkv * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
-    const int smem = kStages * kStageBytes + 1024;
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(attr_once, [&] {
-      attr_err = cudaFuncSetAttribute(decode_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      attr_err = cudaFuncSetAttribute(decode_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      kStages * kStageBytes + 1024);
+      if (attr_err == cudaSuccess)
+        attr_err = cudaFuncSetAttribute(decode_stream_t_kernel<kTStages, kTMinCtas>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kTStages * kStageBytes + 1024);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
-    NGC_CUDA_TRY(launch_pdl(decode_stream_kernel, dim3((unsigned)items), dim3(kStreamThreads), smem, stream, map_k, map_v, p));
+    if (p.g <= 8)      // heads on the N axis of the MMA: no padded rows
+      NGC_CUDA_TRY(launch_pdl(decode_stream_t_kernel<kTStages, kTMinCtas>, dim3((unsigned)items), dim3(kStreamThreads),
+                              kTStages * kStageBytes + 1024, stream, map_k, map_v, p));
+    else
+      NGC_CUDA_TRY(launch_pdl(decode_stream_kernel, dim3((unsigned)items), dim3(kStreamThreads), kStages * kStageBytes + 1024,
+                              stream, map_k, map_v, p));
   } else {
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hq * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
