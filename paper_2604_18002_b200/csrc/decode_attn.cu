@@ -241,8 +241,47 @@ constexpr int kTStages = 2;                   // ring depth and CTAs per SM of t
 constexpr int kTMinCtas = 3;
 constexpr int kORowStride = 132;              // floats; merge buffer row stride (bank spread)
 
+// Tensor maps of a launch: K and V with the full-tile box (64 rows, or one page) and with a
+// 16-row box for the last, partly filled tile of a strip.
+struct KvMaps { CUtensorMap k, v, k16, v16; };
+
+// Issues the TMA loads of 64-token tile `tile` of a strip into stage `st` (K rows at 0, V rows at
+// kTileBytes; channels 64-127 one box further).  A full tile is fetched whole (page by page on a
+// paged cache).  The strip's last tile is fetched in 16-row boxes, only as many as hold live
+// tokens: with caches of a few hundred tokens a whole tile for the tail would be several per cent
+// of the traffic.  Sets the stage's expected byte count itself.
+__device__ __forceinline__ void issue_tile(const DecodeParams& p, const KvMaps& m, const int32_t* table, int row0, int b,
+                                           int plane, int tile, int len, uint8_t* st, uint64_t* bar) {
+  const int t0 = tile * kTileT;
+  if (t0 + kTileT <= len) {
+    ptx::mbar_expect_tx(bar, kStageBytes);
+    const int n_sub = table ? kTileT / p.page : 1;          // pages per 64-token tile
+    const int sub_bytes = (kTileT / n_sub) * 128;
+    for (int sb = 0; sb < n_sub; ++sb) {
+      const int y = table ? (b * p.pages_cap + table[tile * n_sub + sb]) * p.page : row0 + t0;
+      uint8_t* dst = st + sb * sub_bytes;
+      ptx::tma_load_3d(dst, &m.k, 0, y, plane, bar);
+      ptx::tma_load_3d(dst + kBoxBytes, &m.k, 64, y, plane, bar);
+      ptx::tma_load_3d(dst + kTileBytes, &m.v, 0, y, plane, bar);
+      ptx::tma_load_3d(dst + kTileBytes + kBoxBytes, &m.v, 64, y, plane, bar);
+    }
+  } else {
+    const int n16 = (len - t0 + 15) >> 4;                   // 1..4 groups of 16 rows
+    ptx::mbar_expect_tx(bar, (uint32_t)n16 * 4 * 16 * 128);
+    for (int r = 0; r < n16; ++r) {
+      const int t = t0 + 16 * r;
+      const int y = table ? (b * p.pages_cap + table[t / p.page]) * p.page + t % p.page : row0 + t;
+      uint8_t* dst = st + r * 16 * 128;
+      ptx::tma_load_3d(dst, &m.k16, 0, y, plane, bar);
+      ptx::tma_load_3d(dst + kBoxBytes, &m.k16, 64, y, plane, bar);
+      ptx::tma_load_3d(dst + kTileBytes, &m.v16, 0, y, plane, bar);
+      ptx::tma_load_3d(dst + kTileBytes + kBoxBytes, &m.v16, 64, y, plane, bar);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kStreamThreads, 2)
-decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, DecodeParams p) {
+decode_stream_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ uint64_t bar_full[kStages], bar_empty[kStages];
   __shared__ float sm_m[kConsumerWarps][16], sm_l[kConsumerWarps][16];
@@ -265,8 +304,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 #pragma unroll
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&bar_full[s], 1); ptx::mbar_init(&bar_empty[s], kConsumerWarps); }
     ptx::fence_barrier_init();
-    ptx::prefetch_tensormap(&map_k);
-    ptx::prefetch_tensormap(&map_v);
+    ptx::prefetch_tensormap(&maps.k);
+    ptx::prefetch_tensormap(&maps.v);
   }
   ptx::grid_dep_wait();           // lens and the cache rows of earlier calls are final from here on
   ptx::grid_dep_launch();
@@ -295,31 +334,12 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     if (lane == 0 && n_tiles > 0) {
       const int plane = l * p.Hkv + h;
       const int row0 = table ? 0 : (int)p.seq_off[b];
-      const int n_sub = table ? kTileT / p.page : 1;          // pages per 64-token tile
-      const int sub_bytes = (kTileT / n_sub) * 128;
       for (int it = 0; it < n_tiles; ++it) {
         const int s = it % kStages;
         if (it >= kStages) {
           if (!ptx::mbar_wait_bounded(&bar_empty[s], ((it / kStages) - 1) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
         }
-        uint8_t* st = stage_base + s * kStageBytes;
-        ptx::mbar_expect_tx(&bar_full[s], kStageBytes);
-        for (int sb = 0; sb < n_sub; ++sb) {
-          int y;
-          if (table) {
-            // every table entry names a page of this sequence, free ones included, so a tile that
-            // reaches past the live pages still loads mapped memory (those tokens are masked)
-            const int j = min(p.pages_cap - 1, (tile_lo + it) * n_sub + sb);
-            y = (b * p.pages_cap + table[j]) * p.page;
-          } else {
-            y = row0 + (tile_lo + it) * kTileT;
-          }
-          uint8_t* dst = st + sb * sub_bytes;
-          ptx::tma_load_3d(dst, &map_k, 0, y, plane, &bar_full[s]);
-          ptx::tma_load_3d(dst + kBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
-          ptx::tma_load_3d(dst + kTileBytes, &map_v, 0, y, plane, &bar_full[s]);
-          ptx::tma_load_3d(dst + kTileBytes + kBoxBytes, &map_v, 64, y, plane, &bar_full[s]);
-        }
+        issue_tile(p, maps, table, row0, b, plane, tile_lo + it, len, stage_base + s * kStageBytes, &bar_full[s]);
       }
     }
     __syncwarp();
@@ -524,7 +544,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
 // Variant for groups of at most 8 query heads (every GQA shape in the paper's model family).
 template <int kNStages, int kMinCtas>
 __global__ void __launch_bounds__(kStreamThreads, kMinCtas)
-decode_stream_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, DecodeParams p) {
+decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ uint64_t bar_full[kNStages], bar_empty[kNStages];
   __shared__ float sm_m[kConsumerWarps][8], sm_l[kConsumerWarps][8];
@@ -547,8 +567,8 @@ decode_stream_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
 #pragma unroll
     for (int s = 0; s < kNStages; ++s) { ptx::mbar_init(&bar_full[s], 1); ptx::mbar_init(&bar_empty[s], kConsumerWarps); }
     ptx::fence_barrier_init();
-    ptx::prefetch_tensormap(&map_k);
-    ptx::prefetch_tensormap(&map_v);
+    ptx::prefetch_tensormap(&maps.k);
+    ptx::prefetch_tensormap(&maps.v);
   }
   ptx::grid_dep_wait();           // lens and the cache rows of earlier calls are final from here on
   ptx::grid_dep_launch();
@@ -578,31 +598,12 @@ decode_stream_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_c
     if (lane == 0 && n_tiles > 0) {
       const int plane = l * p.Hkv + h;
       const int row0 = table ? 0 : (int)p.seq_off[b];
-      const int n_sub = table ? kTileT / p.page : 1;          // pages per 64-token tile
-      const int sub_bytes = (kTileT / n_sub) * 128;
       for (int it = 0; it < n_tiles; ++it) {
         const int s = it % kNStages;
         if (it >= kNStages) {
           if (!ptx::mbar_wait_bounded(&bar_empty[s], ((it / kNStages) - 1) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
         }
-        uint8_t* st = stage_base + s * kStageBytes;
-        ptx::mbar_expect_tx(&bar_full[s], kStageBytes);
-        for (int sb = 0; sb < n_sub; ++sb) {
-          int y;
-          if (table) {
-            // every table entry names a page of this sequence, free ones included, so a tile that
-            // reaches past the live pages still loads mapped memory (those tokens are masked)
-            const int j = min(p.pages_cap - 1, (tile_lo + it) * n_sub + sb);
-            y = (b * p.pages_cap + table[j]) * p.page;
-          } else {
-            y = row0 + (tile_lo + it) * kTileT;
-          }
-          uint8_t* dst = st + sb * sub_bytes;
-          ptx::tma_load_3d(dst, &map_k, 0, y, plane, &bar_full[s]);
-          ptx::tma_load_3d(dst + kBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
-          ptx::tma_load_3d(dst + kTileBytes, &map_v, 0, y, plane, &bar_full[s]);
-          ptx::tma_load_3d(dst + kTileBytes + kBoxBytes, &map_v, 64, y, plane, &bar_full[s]);
-        }
+        issue_tile(p, maps, table, row0, b, plane, tile_lo + it, len, stage_base + s * kStageBytes, &bar_full[s]);
       }
     }
     __syncwarp();
@@ -855,9 +856,11 @@ int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* ne
   const bool stream_path = c->dtype == NGC_BF16 && c->d == 128 && p.g <= 16 && c->rows < 0x7fffffffLL;
   if (pv.table && !stream_path) return NGC_ERR_UNSUPPORTED;          // paged caches: bf16, d = 128, groups of up to 16 heads
   if (stream_path) {
-    CUtensorMap map_k, map_v;
+    KvMaps maps;
     const int box_rows = pv.table ? pv.page : kTileT;                 // a page is fetched as its own box
-    if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, box_rows) || !make_kv_map(&map_v, c->v, c->rows, c->L * c->Hkv, box_rows))
+    const int planes = c->L * c->Hkv;
+    if (!make_kv_map(&maps.k, c->k, c->rows, planes, box_rows) || !make_kv_map(&maps.v, c->v, c->rows, planes, box_rows) ||
+        !make_kv_map(&maps.k16, c->k, c->rows, planes, 16) || !make_kv_map(&maps.v16, c->v, c->rows, planes, 16))
       return NGC_ERR_UNSUPPORTED;
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hkv * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
@@ -873,10 +876,10 @@ int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* ne
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
     if (p.g <= 8)      // heads on the N axis of the MMA: no padded rows
       NGC_CUDA_TRY(launch_pdl(decode_stream_t_kernel<kTStages, kTMinCtas>, dim3((unsigned)items), dim3(kStreamThreads),
-                              kTStages * kStageBytes + 1024, stream, map_k, map_v, p));
+                              kTStages * kStageBytes + 1024, stream, maps, p));
     else
       NGC_CUDA_TRY(launch_pdl(decode_stream_kernel, dim3((unsigned)items), dim3(kStreamThreads), kStages * kStageBytes + 1024,
-                              stream, map_k, map_v, p));
+                              stream, maps, p));
   } else {
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hq * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;

@@ -497,3 +497,43 @@ def test_logprob_grad_bad_lists(n_max):
     logits[2, 0, 5] = np.nan
     got, st = gpu_logprob_grad(logits, n, None, K, ko)
     assert st == 2 and np.isnan(got[0, 2, 0]).all() and np.max(np.abs(got[0, 1] - good[0, 1])) <= TOL_GRAD
+
+
+# ------------------------------------------------------------------ many short strips
+
+@pytest.mark.parametrize("Hq,Hkv", [(12, 2), (28, 4), (8, 8)])
+def test_decode_many_short_strips(Hq, Hkv):
+    """Hundreds of short strips (the paper's own cache sizes): ragged lengths incl. empty and single-token
+    sequences, lengths on tile borders, two appending steps, every sequence checked."""
+    b = ngc()
+    L, B, d, dtype = 4, 230, 128, torch.bfloat16
+    rng = np.random.default_rng(Hq)
+    lens = rng.integers(0, 700, B).astype(np.int32)
+    lens[:8] = [0, 1, 63, 64, 65, 127, 128, 699]
+    c = synth.make_cache(L, B, Hq, Hkv, d, dtype, lens, capacity=702, seed=21, outlier_channels=4)
+    dc = to_device_cache(c, 702)
+    k_ref, v_ref = synth.to_numpy(c.k).copy(), synth.to_numpy(c.v).copy()
+    so, o_lens = c.seq_off.numpy(), lens.copy()
+    ws = b.alloc_workspace(b.workspace_bytes(b.OP_DECODE, dc))
+    st = b.new_status()
+    out = torch.full((L, B, Hq, d), 7.0, dtype=torch.float32, device="cuda")
+    for s in range(2):
+        q = synth.make_queries(L, B, Hq, d, dtype, seed=30 + s)
+        nk, nv = synth.make_new_kv(L, B, Hkv, d, dtype, seed=40 + 2 * s)
+        b.ngc_decode_attn_ragged(dc, q.cuda(), out, nk.cuda(), nv.cuda(), ws=ws, status=st)
+        ref, rc = oracle.decode_attn(k_ref, v_ref, so, o_lens, synth.to_numpy(q), synth.to_numpy(nk), synth.to_numpy(nv))
+        assert rc == 0
+        assert max_rel_err_per_vector(out.cpu().numpy().astype(np.float64), ref) <= TOL_ATTN_BF16
+    torch.cuda.synchronize()
+    assert status_value(st) == 0 and np.array_equal(dc.lens.cpu().numpy(), o_lens)
+    kg, vg = synth.to_numpy(dc.k), synth.to_numpy(dc.v)
+    for bb in range(B):
+        sl = slice(so[bb], so[bb] + o_lens[bb])
+        assert np.array_equal(kg[:, :, sl], k_ref[:, :, sl]) and np.array_equal(vg[:, :, sl], v_ref[:, :, sl])
+    # read-only call (no append): the empty sequences give zeros
+    dc.lens.copy_(torch.as_tensor(lens))
+    q = synth.make_queries(L, B, Hq, d, dtype, seed=50)
+    b.ngc_decode_attn_ragged(dc, q.cuda(), out, ws=ws, status=st)
+    ref, _ = oracle.decode_attn(k_ref, v_ref, so, lens.copy(), synth.to_numpy(q))
+    got = out.cpu().numpy().astype(np.float64)
+    assert max_rel_err_per_vector(got, ref) <= TOL_ATTN_BF16 and np.all(got[:, 0] == 0.0)
