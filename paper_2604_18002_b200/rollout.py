@@ -82,9 +82,14 @@ class NgcRollout:
 
 class HostStep:
     """Host-buffer driver for one whole step (eviction round + decode steps): pinned host
-    inputs in, attention outputs and eviction results out, copies overlapped with compute."""
+    inputs in, attention outputs and eviction results out, copies overlapped with compute.
 
-    def __init__(self, ro: NgcRollout, steps: int, chunk: int = 16):
+    The K/V cache is by far the largest input.  With ``double_buffer=True`` the driver owns a
+    second K/V pair on the device: ``run(..., prefetch_next=(h_k, h_v))`` uploads the NEXT
+    step's cache into the spare pair on the copy stream while the current step computes, and
+    the next ``run`` adopts that pair instead of waiting for its own upload."""
+
+    def __init__(self, ro: NgcRollout, steps: int, chunk: int = 16, double_buffer: bool = False):
         self.ro, self.steps, self.chunk = ro, steps, chunk
         dev = ro.device
         L, B, Hq, Hkv, d = ro.L, ro.B, ro.Hq, ro.Hkv, ro.d
@@ -94,16 +99,37 @@ class HostStep:
         self.d_out = torch.empty((steps, L, B, Hq, d), dtype=torch.float32, device=dev)
         self.copy_in = torch.cuda.Stream(device=dev)
         self.copy_out = torch.cuda.Stream(device=dev)
+        self.spare = (torch.empty_like(ro.cache.k), torch.empty_like(ro.cache.v)) if double_buffer else None
+        self.staged = None          # event: the spare pair holds the next step's cache
+
+    def _stage_next(self, h_k, h_v):
+        """Upload the next step's cache into the spare pair (copy stream); returns the bytes enqueued."""
+        main = torch.cuda.current_stream()
+        self.copy_in.wait_stream(main)      # the spare pair was the previous step's cache: its kernels must be done
+        with torch.cuda.stream(self.copy_in):
+            self.spare[0].copy_(h_k, non_blocking=True)
+            self.spare[1].copy_(h_v, non_blocking=True)
+            self.staged = torch.cuda.Event()
+            self.staged.record(self.copy_in)
+        return h_k.numel() * h_k.element_size() + h_v.numel() * h_v.element_size()
 
     def run(self, h_k, h_v, h_lens, h_logits, h_q, h_nk, h_nv, h_out, h_kept_order, h_logp, n, n_protect, budget,
-            seed, rnd, h_q_recent=None, d_q_recent=None):
-        """All ``h_*`` are pinned host tensors.  Returns (h2d_bytes, d2h_bytes)."""
+            seed, rnd, h_q_recent=None, d_q_recent=None, prefetch_next=None):
+        """All ``h_*`` are pinned host tensors.  Returns (h2d_bytes, d2h_bytes) enqueued by this call."""
         ro = self.ro
         main = torch.cuda.current_stream()
         h2d = 0
         d2h = 0
-        # cache, lengths and logits are needed first: copy them on the compute stream
-        for dst, src in ((ro.cache.k, h_k), (ro.cache.v, h_v), (ro.cache.lens, h_lens), (ro.logits, h_logits)):
+        if self.staged is not None:
+            # this step's cache was uploaded during the previous step: adopt the pair, no copy now
+            main.wait_event(self.staged)
+            self.staged = None
+            (ro.cache.k, ro.cache.v), self.spare = self.spare, (ro.cache.k, ro.cache.v)
+            first = ((ro.cache.lens, h_lens), (ro.logits, h_logits))
+        else:
+            first = ((ro.cache.k, h_k), (ro.cache.v, h_v), (ro.cache.lens, h_lens), (ro.logits, h_logits))
+        # what the eviction round needs first is copied on the compute stream
+        for dst, src in first:
             dst.copy_(src, non_blocking=True)
             h2d += src.numel() * src.element_size()
         if h_q_recent is not None:
@@ -121,6 +147,8 @@ class HostStep:
                 ev = torch.cuda.Event()
                 ev.record(self.copy_in)
                 in_events.append(ev)
+        if prefetch_next is not None and self.spare is not None:
+            h2d += self._stage_next(*prefetch_next)          # behind this step's decode inputs on the copy stream
         ro.eviction_round(n, n_protect, budget, seed, rnd, q_recent=d_q_recent, logits=ro.logits)
         h_kept_order.copy_(ro.kept_order, non_blocking=True)
         h_logp.copy_(ro.logp, non_blocking=True)
