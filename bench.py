@@ -51,8 +51,8 @@ OTHER_WORKLOADS = {
 METRIC = "evict+compact+decode tokens/sec at B=64"
 W_RECENT = 5
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic K/V bytes for decode_stream_kernel, from the ncu
-# capture summarised in profiles/decode_stream_kernel_config2.md (small case, scaled by tokens processed)
-NCU_TRAFFIC_RATIO = 1.0387
+# capture summarised in profiles/decode_stream_t_kernel_config2.md (small case, scaled by tokens processed)
+NCU_TRAFFIC_RATIO = 1.0154
 
 
 def peaks():
@@ -231,11 +231,11 @@ def run_ngc(args):
     bytes_per_launch = algorithmic_decode_bytes(cfg, visible_total)
     peak, peak_kind = peaks()
     achieved = bytes_per_launch / (mean_dec_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (time per ngc_decode_attn_ragged call: attention with fused append + lens bump, launch gaps included)",
+    roofline = {"bound": "hbm", "kernel": "decode_stream_t_kernel (time per ngc_decode_attn_ragged call: attention with fused append + lens bump, launch gaps included)",
                 "achieved": round(achieved, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": round(achieved / peak, 4),
                 "traffic": int(args.traffic if args.traffic else NCU_TRAFFIC_RATIO * bytes_per_launch),
-                "traffic_source": "ncu capture of a B=16 launch scaled by tokens processed (profiles/decode_stream_kernel_config2.md)", "bytes_per_launch": int(bytes_per_launch),
+                "traffic_source": "ncu capture of a B=16 launch scaled by tokens processed (profiles/decode_stream_t_kernel_config2.md)", "bytes_per_launch": int(bytes_per_launch),
                 "ms_per_launch": round(mean_dec_ms, 4), "decode_share_of_step": round(sum(dec_ms) / ms_total, 4)}
 
     result = {"metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -471,7 +471,7 @@ def run_other(args):
               "config": {"workload": OTHER_WORKLOADS[cid], "batch": B, "decode_steps": steps, "input_ring": ring,
                          "layout": "paged (eviction edits page tables, no K/V movement)" if paged is not None else "contiguous strips, in-place compaction"},
               "per_call_ms": med,
-              "roofline": {"bound": "hbm", "kernel": "decode_stream_kernel (all decode calls of a step, launch gaps included)",
+              "roofline": {"bound": "hbm", "kernel": "decode_stream_t_kernel (all decode calls of a step, launch gaps included)",
                            "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                            "frac": round(dec_gbs / peak, 4), "decode_ms_per_step": round(dec_ms, 3), "decode_calls": steps, "traffic": None},
               "compact": {"bytes": int(compact_bytes), "GB/s": round(cmp_gbs, 1), "frac_of_peak": round(cmp_gbs / peak, 4),
