@@ -788,14 +788,17 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
 
 // ---------------------------------------------------------------- host side
 
-constexpr int kTargetCtas = 148 * 2 * 2;   // two waves of two CTAs per SM
+constexpr int kTargetCtas = 148 * 2 * 2;    // two waves of two CTAs per SM
+constexpr int kTargetCtasT = 148 * 3 * 2;   // ... of three per SM (the kernel for groups of <= 8 heads)
 
 }  // namespace
 
 int decode_n_split(const ngc_cache* c, int layers) {
   const int64_t strips = (int64_t)layers * c->B * c->Hkv;
-  if (strips >= kTargetCtas) return 1;
-  int ns = (int)((kTargetCtas + strips - 1) / strips);
+  const bool t_kernel = c->dtype == NGC_BF16 && c->d == 128 && c->Hq / c->Hkv <= 8;
+  const int target = t_kernel ? kTargetCtasT : kTargetCtas;
+  if (strips >= target) return 1;
+  int ns = (int)((target + strips - 1) / strips);
   const int by_len = (c->max_len + 1 + 4 * kTileT - 1) / (4 * kTileT);   // at least 4 tiles per split
   if (ns > by_len) ns = by_len;
   if (ns > 64) ns = 64;

@@ -1,5 +1,5 @@
 // Thin wrappers over the sm_100a PTX this library uses: mbarrier, TMA tensor
-// loads (no multicast anywhere), ldmatrix and the bf16 warp-level MMA.
+// loads (every CTA fetches its own tiles), ldmatrix and the bf16 warp-level MMA.
 #pragma once
 
 #include <cuda.h>
