@@ -231,3 +231,25 @@ def score_evict(k, seq_off, lens, q_recent, block, lists, log_transform=0, n_max
                                  _p(q_recent), int(w), int(block), int(lists), int(log_transform),
                                  _p(out), int(n_max))
     return out
+
+
+def score_evict_grad(k, seq_off, lens, q_recent, block, lists, grad_logits, log_transform=0):
+    """Gradient of the scores w.r.t. q_recent and k.  grad_logits [B][G][n_max] float64.
+    Returns (grad_q [L][B][Hq][w][d], grad_k [L][Hkv][R][d]) float64."""
+    L, Hkv, R, d = k.shape
+    dt = _dtype_of(k)
+    k = np.ascontiguousarray(k)
+    seq_off = _c(seq_off, np.int64)
+    lens = _c(lens, np.int32)
+    B = lens.shape[0]
+    q_recent = np.ascontiguousarray(q_recent)
+    assert _dtype_of(q_recent) == dt
+    Hq, w = q_recent.shape[2], q_recent.shape[3]
+    grad_logits = _c(grad_logits, np.float64)
+    n_max = grad_logits.shape[2]
+    gq = np.zeros((L, B, Hq, w, d), np.float64)
+    gk = np.zeros((L, Hkv, R, d), np.float64)
+    rc = lib().ngc_oracle_score_evict_grad(_p(k), _p(seq_off), _p(lens), L, B, Hq, Hkv, d, dt, _p(q_recent), w, int(block),
+                                           int(lists), int(log_transform), _p(grad_logits), n_max, _p(gq), _p(gk))
+    assert rc == 0
+    return gq, gk

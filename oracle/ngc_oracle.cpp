@@ -467,4 +467,77 @@ int ngc_oracle_score_evict(const void* k, const int64_t* seq_off, const int32_t*
   return 0;
 }
 
+/* Gradient of the eviction scores with respect to the recent queries and the keys: the chain
+ * rule through the block mean, the row average and the softmax of Section 4.2, written out.
+ * With u(t) the unit of token t, |u| its size and n_rows the number of attention rows of the list:
+ *   dL/dA[r][t]  = grad_logits[u(t)] / |u(t)| / n_rows        (divided by s_u as well when logit = log s)
+ *   dL/dz[r][t]  = A[r][t] * (dL/dA[r][t] - sum_t' A[r][t'] dL/dA[r][t'])           (softmax)
+ *   dL/dq[r]     = sum_t dL/dz[r][t] k[t] / sqrt(d),   dL/dk[t] += dL/dz[r][t] q[r] / sqrt(d). */
+int ngc_oracle_score_evict_grad(const void* k, const int64_t* seq_off, const int32_t* lens,
+                                int L, int B, int Hq, int Hkv, int d, int dtype,
+                                const void* q_recent, int w, int block, int lists, int log_transform,
+                                const double* grad_logits, int n_max, double* grad_q, double* grad_k) {
+  const int G = lists_G(lists, L, Hkv);
+  const int64_t R = seq_off[B];
+  const int g = Hq / Hkv;
+  const double inv_sqrt_d = 1.0 / std::sqrt((double)d);
+  std::fill(grad_q, grad_q + (int64_t)L * B * Hq * w * d, 0.0);
+  std::fill(grad_k, grad_k + (int64_t)L * Hkv * R * d, 0.0);
+  std::vector<double> s_lin;                   /* forward scores, linear (needed for the log variant) */
+  if (log_transform) {
+    s_lin.assign((size_t)B * G * n_max, 0.0);
+    ngc_oracle_score_evict(k, seq_off, lens, L, B, Hq, Hkv, d, dtype, q_recent, w, block, lists, 0, s_lin.data(), n_max);
+  }
+#pragma omp parallel for schedule(dynamic)
+  for (int b = 0; b < B; ++b) {
+    int T = lens[b];
+    if (T <= 0) continue;
+    int w_eff = std::min(w, T);
+    std::vector<int64_t> rows((size_t)G, 0);
+    for (int l = 0; l < L; ++l)
+      for (int hq = 0; hq < Hq; ++hq) rows[list_of(lists, l, hq / g, Hkv)] += w_eff;
+    /* dL/dA for any row of list gi, per token */
+    std::vector<std::vector<double>> dA((size_t)G, std::vector<double>((size_t)T, 0.0));
+    for (int gi = 0; gi < G; ++gi)
+      for (int t = 0; t < T; ++t) {
+        int u = t / block;
+        if (u >= n_max) continue;
+        int size = std::min((u + 1) * block, T) - u * block;
+        double up = grad_logits[((int64_t)b * G + gi) * n_max + u];
+        if (log_transform) up /= s_lin[((int64_t)b * G + gi) * n_max + u];
+        dA[gi][t] = up / (double)size / (double)rows[gi];
+      }
+    std::vector<double> a((size_t)T);
+    for (int l = 0; l < L; ++l)
+      for (int hq = 0; hq < Hq; ++hq) {
+        int h = hq / g;
+        int gi = list_of(lists, l, h, Hkv);
+        int64_t base = ((int64_t)(l * Hkv + h) * R + seq_off[b]);
+        for (int j = w - w_eff; j < w; ++j) {
+          int pos = T - w + j;
+          int64_t qo = ((((int64_t)l * B + b) * Hq + hq) * w + j) * d;
+          double mx = -std::numeric_limits<double>::infinity();
+          for (int t = 0; t <= pos; ++t) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += widen(q_recent, qo + c, dtype) * widen(k, (base + t) * d + c, dtype);
+            a[t] = acc * inv_sqrt_d;
+            mx = std::max(mx, a[t]);
+          }
+          double den = 0.0;
+          for (int t = 0; t <= pos; ++t) { a[t] = std::exp(a[t] - mx); den += a[t]; }
+          double dot = 0.0;
+          for (int t = 0; t <= pos; ++t) { a[t] /= den; dot += a[t] * dA[gi][t]; }
+          for (int t = 0; t <= pos; ++t) {
+            double dz = a[t] * (dA[gi][t] - dot) * inv_sqrt_d;
+            for (int c = 0; c < d; ++c) {
+              grad_q[qo + c] += dz * widen(k, (base + t) * d + c, dtype);
+              grad_k[(base + t) * d + c] += dz * widen(q_recent, qo + c, dtype);
+            }
+          }
+        }
+      }
+  }
+  return 0;
+}
+
 }  // extern "C"

@@ -117,6 +117,15 @@ int ngc_oracle_score_evict(const void* k, const int64_t* seq_off, const int32_t*
                            const void* q_recent, int w, int block, int lists, int log_transform,
                            double* logits, int n_max);
 
+/* Gradient of ngc_oracle_score_evict's logits with respect to q_recent and k (Section 4.4: the
+ * eviction loss reaches the model through the scores; Section 4.5 recomputes them on the autograd
+ * graph).  grad_logits [B][G][n_max]; grad_q [L][B][Hq][w][d] and grad_k [L][Hkv][R][d] double out
+ * (zero where nothing contributes). */
+int ngc_oracle_score_evict_grad(const void* k, const int64_t* seq_off, const int32_t* lens,
+                                int L, int B, int Hq, int Hkv, int d, int dtype,
+                                const void* q_recent, int w, int block, int lists, int log_transform,
+                                const double* grad_logits, int n_max, double* grad_q, double* grad_k);
+
 /* Number of OpenMP threads the oracle will use. */
 int ngc_oracle_threads(void);
 

@@ -299,3 +299,62 @@ def test_score_single_query_equals_decode_attention_weights():
     weights = out[0, 0, :, :T].mean(0)                      # mean over the heads of the group
     s = oracle.score_evict(k, so, np.array([T], np.int32), q.reshape(L, B, Hq, 1, d), 1, 2)[0, 0]
     assert np.allclose(s, weights, atol=1e-14)
+
+
+# ------------------------------------------------------------------ gradient of the eviction scores
+
+def _score_loss(k, so, lens, qr, block, lists, up, log_transform):
+    s = oracle.score_evict(k, so, lens, qr, block, lists, log_transform=log_transform, n_max=up.shape[2])
+    return float(np.nansum(np.where(np.isnan(s), 0.0, s) * up))
+
+
+@pytest.mark.parametrize("lists,block,log_transform", [(0, 1, 0), (1, 3, 0), (2, 1, 1), (1, 4, 1)])
+def test_score_grad_matches_finite_differences(lists, block, log_transform):
+    """Central differences of the (separately pinned) forward scores, on fp32 inputs."""
+    rng = np.random.default_rng(7 + lists)
+    L, B, Hq, Hkv, d, w = 2, 2, 4, 2, 8, 3
+    lens = np.array([7, 2], np.int32)                       # the second sequence is shorter than the window
+    so = np.array([0, 8, 11], np.int64)
+    k = rng.normal(0, 1, (L, Hkv, 11, d)).astype(np.float32)
+    qr = rng.normal(0, 1, (L, B, Hq, w, d)).astype(np.float32)
+    G = oracle.lists_G(lists, L, Hkv)
+    n_max = (8 + block - 1) // block
+    up = rng.normal(0, 1, (B, G, n_max))
+    gq, gk = oracle.score_evict_grad(k, so, lens, qr, block, lists, up, log_transform=log_transform)
+    h = 2.0 ** -9
+    for _ in range(40):
+        if rng.random() < 0.5:
+            idx = tuple(rng.integers(0, s) for s in qr.shape)
+            a, b2 = qr.copy(), qr.copy()
+            a[idx] += h
+            b2[idx] -= h
+            fd = (_score_loss(k, so, lens, a, block, lists, up, log_transform) - _score_loss(k, so, lens, b2, block, lists, up, log_transform)) / \
+                 (float(a[idx]) - float(b2[idx]))
+            assert abs(fd - gq[idx]) <= 1e-4 * max(1.0, abs(fd)), ("q", idx)
+        else:
+            idx = tuple(rng.integers(0, s) for s in k.shape)
+            a, b2 = k.copy(), k.copy()
+            a[idx] += h
+            b2[idx] -= h
+            fd = (_score_loss(a, so, lens, qr, block, lists, up, log_transform) - _score_loss(b2, so, lens, qr, block, lists, up, log_transform)) / \
+                 (float(a[idx]) - float(b2[idx]))
+            assert abs(fd - gk[idx]) <= 1e-4 * max(1.0, abs(fd)), ("k", idx)
+    # rows beyond a sequence's length and queries before its start get no gradient
+    assert np.all(gk[:, :, 7:8] == 0) and np.all(gk[:, :, 10:] == 0) and np.all(gq[:, 1, :, 0] == 0)
+
+
+def test_score_grad_vanishes_along_the_normalisation():
+    """sum_j |B_j| s_j = 1 whatever q and k are: an upstream gradient proportional to the unit sizes gives zero."""
+    rng = np.random.default_rng(2)
+    L, B, Hq, Hkv, d, w, block = 1, 1, 4, 2, 16, 5, 4
+    lens = np.array([14], np.int32)
+    so = np.array([0, 14], np.int64)
+    k = rng.normal(0, 1, (L, Hkv, 14, d)).astype(np.float32)
+    qr = rng.normal(0, 1, (L, B, Hq, w, d)).astype(np.float32)
+    up = np.array([[[4, 4, 4, 2]]], np.float64) * 0.37             # unit sizes 4, 4, 4, 2
+    gq, gk = oracle.score_evict_grad(k, so, lens, qr, block, 1, up)
+    assert np.max(np.abs(gq)) <= 1e-12 and np.max(np.abs(gk)) <= 1e-12
+    up2 = up.copy()
+    up2[0, 0, 1] += 1.0
+    gq2, gk2 = oracle.score_evict_grad(k, so, lens, qr, block, 1, up2)
+    assert np.max(np.abs(gq2)) > 1e-4 and np.max(np.abs(gk2)) > 1e-4
