@@ -74,7 +74,8 @@ typedef enum {
 
 typedef enum { NGC_F32 = 0, NGC_BF16 = 1 } ngc_dtype;
 typedef enum { NGC_LISTS_SHARED = 0, NGC_LISTS_PER_LAYER = 1, NGC_LISTS_PER_LAYER_KVHEAD = 2 } ngc_lists;
-typedef enum { NGC_OP_SCORE = 0, NGC_OP_SAMPLE = 1, NGC_OP_LOGPROB = 2, NGC_OP_COMPACT = 3, NGC_OP_DECODE = 4 } ngc_op;
+typedef enum { NGC_OP_SCORE = 0, NGC_OP_SAMPLE = 1, NGC_OP_LOGPROB = 2, NGC_OP_COMPACT = 3, NGC_OP_DECODE = 4,
+               NGC_OP_SCORE_BACKWARD = 5 } ngc_op;
 
 /* Describes the cache; owns nothing.  `rows` and `max_len` are host copies the
  * launch geometry needs: rows = seq_off[B]; max_len >= every lens[b] at the
@@ -129,6 +130,25 @@ int ngc_decode_splits(const ngc_cache* c, int layers);
 int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, int lists,
                     int log_transform, float* logits, int n_max,
                     void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
+
+/*
+ * Gradient of the eviction scores with respect to the recent queries and the
+ * keys -- Sections 4.4 and 4.5: the eviction loss reaches the model through
+ * the scores, whose inputs are recomputed "on the autograd graph".  The chain
+ * rule through the block mean, the average over attention rows and the
+ * softmax of ngc_score_evict:
+ *   grad_logits   [B][G][n_max] fp32 upstream gradient (e.g. from ngc_evict_logprob_backward)
+ *   logits        the forward output; read only when log_transform != 0 (else may be NULL)
+ *   grad_q_recent [L][B][Hq][w][d] fp32 out (zero for window queries before the sequence start)
+ *   grad_k        [L][Hkv][R][d] out, cache dtype; rows >= lens[b] are not written
+ * Other arguments as in ngc_score_evict.  Built for bf16 caches with d = 128 and at most 40
+ * (head, query) rows per KV head (Hq/Hkv * w <= 40); NGC_ERR_UNSUPPORTED otherwise.  K is read
+ * twice and grad_k written once.  Workspace: ngc_workspace_bytes(NGC_OP_SCORE_BACKWARD, ...).
+ */
+int ngc_score_evict_backward(const ngc_cache* c, const void* q_recent, int w, int block, int lists, int log_transform,
+                             const float* logits, const float* grad_logits, int n_max,
+                             float* grad_q_recent, void* grad_k,
+                             void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
 
 /*
  * Sampling the keep set -- Section 4.3 (Gumbel-top-k): perturbed key =

@@ -19,14 +19,14 @@ LIB_PATH = os.path.join(_HERE, "libngc_b200.so")
 
 F32, BF16 = 0, 1
 LISTS_SHARED, LISTS_PER_LAYER, LISTS_PER_LAYER_KVHEAD = 0, 1, 2
-OP_SCORE, OP_SAMPLE, OP_LOGPROB, OP_COMPACT, OP_DECODE = range(5)
+OP_SCORE, OP_SAMPLE, OP_LOGPROB, OP_COMPACT, OP_DECODE, OP_SCORE_BACKWARD = range(6)
 
 DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "strip full",
               5: "lists disagree", 6: "timeout"}
 
 EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
            "ngc_sample_evict", "ngc_evict_logprob", "ngc_evict_logprob_backward", "ngc_compact_kv", "ngc_decode_attn_ragged",
-           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged", "ngc_replay_visibility"]
+           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged", "ngc_replay_visibility", "ngc_score_evict_backward"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -79,6 +79,8 @@ def _load():
     lib.ngc_decode_attn_ragged_static.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, vp]
     lib.ngc_score_evict_paged.restype = i32
     lib.ngc_score_evict_paged.argtypes = [C.POINTER(PagedCacheDesc), vp, i32, i32, vp, i32, vp, sz, vp, vp]
+    lib.ngc_score_evict_backward.restype = i32
+    lib.ngc_score_evict_backward.argtypes = [C.POINTER(CacheDesc), vp, i32, i32, i32, i32, vp, vp, i32, vp, vp, vp, sz, vp, vp]
     lib.ngc_replay_visibility.restype = i32
     lib.ngc_replay_visibility.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.ngc_evict_pages.restype = i32
@@ -342,3 +344,14 @@ def ngc_replay_visibility(kept_sorted: torch.Tensor, budget: torch.Tensor, alive
     rc = lib.ngc_replay_visibility(_ptr(kept_sorted), _ptr(budget), _ptr(alive_before), _ptr(total_before), R, B, G, k_max, block,
                                    alive_max, _ptr(alive_pos), _ptr(alive_count), _ptr(status), _stream())
     _check(rc, "ngc_replay_visibility")
+
+
+def ngc_score_evict_backward(cache: NgcCache, q_recent: torch.Tensor, block: int, lists: int, grad_logits: torch.Tensor,
+                             grad_q_recent: torch.Tensor, grad_k: torch.Tensor, logits: Optional[torch.Tensor] = None,
+                             log_transform: int = 0, ws: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
+    """grad_logits [B][G][n_max] fp32 -> grad_q_recent fp32 (shape of q_recent), grad_k (shape and dtype of cache.k)."""
+    d = cache.desc()
+    rc = lib.ngc_score_evict_backward(C.byref(d), _ptr(q_recent), q_recent.shape[3], block, lists, log_transform, _ptr(logits),
+                                      _ptr(grad_logits), grad_logits.shape[2], _ptr(grad_q_recent), _ptr(grad_k),
+                                      _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
+    _check(rc, "ngc_score_evict_backward")

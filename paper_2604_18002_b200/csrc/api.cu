@@ -37,6 +37,7 @@ size_t ngc_workspace_bytes(int op, const ngc_cache* c, int G, int n_max, int k_m
     case NGC_OP_LOGPROB: return 0;
     case NGC_OP_COMPACT: return 0;
     case NGC_OP_DECODE: return c ? ngc::decode_workspace_bytes(c, c->L) : 0;
+    case NGC_OP_SCORE_BACKWARD: return c ? ngc::score_backward_workspace_bytes(c) : 0;
     default: return 0;
   }
 }

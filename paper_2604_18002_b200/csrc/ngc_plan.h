@@ -19,5 +19,6 @@ size_t decode_workspace_bytes(const ngc_cache* c, int layers);
 size_t sample_workspace_bytes(int B, int G, int n_max);
 
 size_t score_workspace_bytes(const ngc_cache* c, int G, int n_max);
+size_t score_backward_workspace_bytes(const ngc_cache* c);
 
 }  // namespace ngc
