@@ -10,7 +10,7 @@
 // bf16, d = 128, at most 40 rows per strip (the shapes of the streaming forward kernel).  Two
 // launches stream K through the same TMA + mbarrier ring as the forward pass:
 //   1. per (strip, token range): row max, sum of exponentials and sum of exponentials times P;
-//   2. same geometry, one CTA per SM: the merged statistics give A and c; S^T = K Q^T is
+//   2. same geometry: the merged statistics give A and c; S^T = K Q^T is
 //      recomputed on the tensor cores, dz formed in registers, then
 //        dK  (16 tokens x 128 channels per warp) = dZ Q          -- A operand straight from the
 //                                                                   accumulators, written out as bf16;
@@ -36,7 +36,7 @@ constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kBoxBytes = kTileT * 128;           // 64 tokens x 64 channels of bf16
 constexpr int kStageBytes = 2 * kBoxBytes;
 constexpr int kStagesA = 4;                       // statistics pass, two CTAs per SM
-constexpr int kStagesB = 6;                       // gradient pass, one CTA per SM
+constexpr int kStagesB = 4;                       // gradient pass, two CTAs per SM
 constexpr int kMaxRows = 40;
 constexpr int kQRowBytes = 272;                   // query row in shared memory: 256 bytes + 16 (conflict-free ldmatrix)
 constexpr int kQBytes = 48 * kQRowBytes;          // rows padded to 48 (three 16-row MMA steps)
@@ -259,7 +259,7 @@ score_bwd_stats_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
 
 template <int NT>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ uint64_t bar_full[kStagesB], bar_empty[kStagesB];
@@ -393,28 +393,30 @@ score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
       asm volatile("st.shared.b32 [%0], %1;" ::"r"(dz_buf + off), "r"(lo[t8]) : "memory");
       asm volatile("st.shared.b32 [%0], %1;" ::"r"(dz_buf + off + 8 * kDzRowBytes), "r"(hi[t8]) : "memory");
     }
-    // ---- dK = dZ Q (16 tokens x 128 channels): A operand straight from the packed dz ----
-    {
-      float dk[16][4];
+    // ---- dK = dZ Q (16 tokens x 128 channels, 64 at a time): A operand straight from the packed dz ----
 #pragma unroll
-      for (int n = 0; n < 16; ++n) { dk[n][0] = 0.f; dk[n][1] = 0.f; dk[n][2] = 0.f; dk[n][3] = 0.f; }
+    for (int half = 0; half < 2; ++half) {
+      float dk[8][4];
+#pragma unroll
+      for (int n = 0; n < 8; ++n) { dk[n][0] = 0.f; dk[n][1] = 0.f; dk[n][2] = 0.f; dk[n][3] = 0.f; }
 #pragma unroll
       for (int kk = 0; kk < 3; ++kk) {
         if (16 * kk < 8 * NT) {
           const uint32_t a[4] = {lo[2 * kk], hi[2 * kk], lo[2 * kk + 1], hi[2 * kk + 1]};
 #pragma unroll
-          for (int np = 0; np < 8; ++np) {
+          for (int np = 0; np < 4; ++np) {
             uint32_t r0, r1, r2, r3;
-            ptx::ldmatrix_x4_trans(q_u32 + (uint32_t)(16 * kk) * kQRowBytes + qk_lane + np * 32, r0, r1, r2, r3);
+            ptx::ldmatrix_x4_trans(q_u32 + (uint32_t)(16 * kk) * kQRowBytes + qk_lane + (4 * half + np) * 32, r0, r1, r2, r3);
             ptx::mma_bf16_16816(dk[2 * np], a, r0, r1);
             ptx::mma_bf16_16816(dk[2 * np + 1], a, r2, r3);
           }
         }
       }
 #pragma unroll
-      for (int n = 0; n < 16; ++n) {
-        if (t0 < T_b) *reinterpret_cast<uint32_t*>(gk_strip + (int64_t)t0 * 128 + 8 * n + 2 * tig) = ptx::pack_bf16x2(dk[n][0], dk[n][1]);
-        if (t1 < T_b) *reinterpret_cast<uint32_t*>(gk_strip + (int64_t)t1 * 128 + 8 * n + 2 * tig) = ptx::pack_bf16x2(dk[n][2], dk[n][3]);
+      for (int n = 0; n < 8; ++n) {
+        const int ch = 64 * half + 8 * n + 2 * tig;
+        if (t0 < T_b) *reinterpret_cast<uint32_t*>(gk_strip + (int64_t)t0 * 128 + ch) = ptx::pack_bf16x2(dk[n][0], dk[n][1]);
+        if (t1 < T_b) *reinterpret_cast<uint32_t*>(gk_strip + (int64_t)t1 * 128 + ch) = ptx::pack_bf16x2(dk[n][2], dk[n][3]);
       }
     }
     consumer_bar();              // the tile's dz is complete and dead K rows are zero
