@@ -82,3 +82,27 @@ def dense_mask(T, total_before, kept_positions):
                 M[t, np.asarray(kept_positions[r - 1], np.int64)] = True   # every query of block r sees kept_{r-1}
     M[np.arange(T), np.arange(T)] = True                         # the diagonal
     return M
+
+
+def replay_attention(q, k, v, masks, scale=None):
+    """Attention of every token under its replay mask, in float64 (paper Section 4.5: one forward pass
+    whose per-layer masks reproduce what each token saw at rollout time).
+
+    q [Hq][T][d], k/v [Hkv][T][d] float64 (ONE layer of ONE sequence), masks [G_l][T][T] bool with
+    G_l = 1 (one mask for the layer) or Hkv (one per KV head).  Returns out [Hq][T][d]."""
+    Hq, T, d = q.shape
+    Hkv = k.shape[0]
+    g = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    out = np.zeros((Hq, T, d))
+    for hq in range(Hq):
+        h = hq // g
+        M = masks[h if masks.shape[0] == Hkv else 0]
+        z = (q[hq] @ k[h].T) * scale
+        z = np.where(M, z, -np.inf)
+        z -= z.max(-1, keepdims=True)
+        p = np.exp(z)
+        p /= p.sum(-1, keepdims=True)
+        out[hq] = p @ v[h]
+    return out

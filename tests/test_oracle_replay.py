@@ -108,3 +108,46 @@ def test_steady_state_alive_size_and_error_codes():
     fewer[1] = 100                      # fewer tokens alive at round 1 than round 0 kept
     _, _, rc = replay.alive_positions(ks, np.full((R, 1), K), fewer, [[768 + r * delta] for r in range(R)])
     assert rc == 1
+
+
+def test_replay_attention_pins():
+    """Causal mask -> the library's scaled_dot_product_attention; and the paper's claim itself: under the
+    replay mask, token t's attention equals decode attention over the cache as it stood at rollout time
+    (two separately written oracle routines: dense numpy here, the C++ ragged decode + compaction there)."""
+    import torch
+    import oracle
+    rng = np.random.default_rng(0)
+    q, k, v = rng.normal(size=(4, 9, 8)), rng.normal(size=(2, 9, 8)), rng.normal(size=(2, 9, 8))
+    o = replay.replay_attention(q, k, v, np.tril(np.ones((9, 9), bool))[None])
+    ref = torch.nn.functional.scaled_dot_product_attention(torch.tensor(q)[None], torch.tensor(k).repeat_interleave(2, 0)[None],
+                                                           torch.tensor(v).repeat_interleave(2, 0)[None], is_causal=True)[0].numpy()
+    assert np.abs(o - ref).max() < 1e-12
+    # rollout: 1 layer, prompt of 6 tokens, rounds after 6 and 11 tokens keep 3 of 6 and 4 of 8 cache entries
+    L, B, Hq, Hkv, d, T = 1, 1, 4, 2, 64, 15
+    kf = rng.normal(size=(L, Hkv, T, d)).astype(np.float32)
+    vf = rng.normal(size=(L, Hkv, T, d)).astype(np.float32)
+    qf = rng.normal(size=(L, B, Hq, T, d)).astype(np.float32)
+    total_before, kept_lists = [6, 11], [[0, 2, 5], [1, 2, 4, 7]]
+    cache_k = np.zeros((L, Hkv, T, d), np.float32)
+    cache_v = np.zeros_like(cache_k)
+    so, lens = np.array([0, T], np.int64), np.zeros(1, np.int32)
+    rollout_out = np.zeros((Hq, T, d))
+    r = 0
+    for t in range(T):
+        out, rc = oracle.decode_attn(cache_k, cache_v, so, lens, qf[:, :, :, t], kf[:, None, :, t].copy(), vf[:, None, :, t].copy())
+        assert rc == 0
+        rollout_out[:, t] = out[0, 0]
+        if r < 2 and t + 1 == total_before[r]:
+            ks = np.array(kept_lists[r], np.int32)[None, None]
+            cache_k, cache_v, nl, rc = oracle.compact_kv(cache_k, cache_v, so, lens, ks, [len(kept_lists[r])], 0)
+            assert rc == 0
+            lens = nl.copy()
+            r += 1
+    k_max = 4
+    ks = np.full((2, 1, 1, k_max), -1, np.int32)
+    ks[0, 0, 0, :3], ks[1, 0, 0, :4] = kept_lists[0], kept_lists[1]
+    pos, cnt, rc = replay.alive_positions(ks, [[3], [4]], [[6], [8]], [[6], [11]])
+    assert rc == 0
+    M = replay.dense_mask(T, total_before, [pos[i, 0, 0, : cnt[i, 0, 0]] for i in range(2)])
+    rep = replay.replay_attention(qf[0, 0].astype(np.float64), kf[0].astype(np.float64), vf[0].astype(np.float64), M[None])
+    assert np.abs(rep - rollout_out).max() < 1e-10
