@@ -235,6 +235,29 @@ int ngc_replay_visibility(const int32_t* kept_sorted, const int32_t* budget, con
                           int32_t* alive_pos, int32_t* alive_count, int32_t* dev_status, ngc_stream stream);
 
 /*
+ * Replay attention -- Section 4.5: one pass over ALL tokens of a rollout in
+ * which every query sees exactly the keys it saw when it was generated, so
+ * that token and eviction log-probabilities are recomputed on-policy.  The
+ * masks of Appendix A.3 are not materialised: the query at position t attends
+ * to kept_r (alive_pos of the last round that fired at or before t, from
+ * ngc_replay_visibility) and, causally, to the tokens from that round's
+ * boundary up to t itself; queries before the first round are plain causal.
+ *   c            the FULL sequences: k, v [L][Hkv][R][d] hold every token in original
+ *                order, lens[b] = T_b tokens (bf16, d = 128)
+ *   q            [L][B][Hq][t_max][d] bf16; rows >= lens[b] are ignored
+ *   alive_pos    [n_rounds][B][G][kt_max], alive_count [n_rounds][B][G], total_before
+ *                [n_rounds][B] (ascending per sequence); n_rounds = 0: causal attention
+ *   lists        how G maps to (layer, KV head), as everywhere
+ *   out          [L][B][Hq][t_max][d] fp32 or bf16; rows >= lens[b] are not written
+ * fp32 scores, softmax and accumulation; probabilities rounded to bf16 for P*V.
+ * Needs no workspace.
+ */
+int ngc_replay_attn(const ngc_cache* c, const void* q, int t_max,
+                    const int32_t* alive_pos, const int32_t* alive_count, const int32_t* total_before,
+                    int n_rounds, int kt_max, int lists, float scale, void* out, int out_dtype,
+                    int32_t* dev_status, ngc_stream stream);
+
+/*
  * Physical eviction -- Section 4.1 ("permanently evicts the rest").  In place:
  * in every (layer, KV head, sequence) strip of K and V the tokens of the kept
  * units move to the front in ascending original order, and lens[b] becomes
