@@ -50,7 +50,7 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
   return (uint32_t)((c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(kThreads, 2) replay_attn_kernel(ReplayAttnParams p) {
+__global__ void __launch_bounds__(kThreads, 3) replay_attn_kernel(ReplayAttnParams p) {
   extern __shared__ uint8_t smem_dyn[];
   // key sources of this query tile: the kept lists of the rounds it straddles, then the contiguous run
   __shared__ int s_seg_rho[kMaxSeg], s_seg_n[kMaxSeg], s_seg_first[kMaxSeg + 1];
