@@ -482,6 +482,83 @@ def run_other(args):
     print(json.dumps(result), flush=True)
 
 
+# ------------------------------------------------------------------------------------ training-side kernels (measurement aid)
+
+def run_kernel(args):
+    """Times one training-side call on one GPU: `--kernel score_backward` (gradient of the eviction scores at
+    the config-2 shape) or `--kernel replay_attn` (replay attention over the rollout-loop history of config 5,
+    `--layers` of its 28 layers)."""
+    from paper_2604_18002_b200 import binding as ngc
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    peak_hbm, peak_kind = peaks()
+    st = ngc.new_status(dev)
+
+    def best_of(fn, reps):
+        best = 1e9
+        for rep in range(reps + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            if rep:
+                best = min(best, e0.elapsed_time(e1))
+        return best
+
+    if args.kernel == "score_backward":
+        cfg = synth.CONFIGS[2]
+        L, Hq, Hkv, d, T, B = cfg["L"], cfg["Hq"], cfg["Hkv"], cfg["d"], cfg["T"], args.batch or cfg["B"]
+        c = synth.make_cache(L, B, Hq, Hkv, d, torch.bfloat16, [T] * B, capacity=T, seed=0, device=dev)
+        dc = ngc.NgcCache(c.k, c.v, c.seq_off, c.lens, Hq, T)
+        qr = synth.normal((L, B, Hq, W_RECENT, d), 1, torch.bfloat16, device=dev)
+        up = synth.make_logits(B, 1, T, seed=2, device=dev)
+        gq = torch.empty(qr.shape, dtype=torch.float32, device=dev)
+        gk = torch.empty_like(c.k)
+        ws = ngc.alloc_workspace(ngc.workspace_bytes(ngc.OP_SCORE_BACKWARD, dc), dev)
+        ms = best_of(lambda: ngc.ngc_score_evict_backward(dc, qr, 1, ngc.LISTS_SHARED, up, gq, gk, ws=ws, status=st), args.steps)
+        nbytes = 3 * L * Hkv * B * T * d * 2
+        res = {"kernel": "ngc_score_evict_backward", "workload": f"config-2 shape, B={B}, T={T}, w={W_RECENT}, shared list", "ms": round(ms, 3),
+               "roofline": {"bound": "hbm", "achieved": round(nbytes / ms / 1e6, 1), "peak": peak_hbm, "peak_kind": f"of {peak_kind}",
+                            "unit": "GB/s", "frac": round(nbytes / ms / 1e6 / peak_hbm, 4), "bytes": "K read twice + dK written once"}}
+    else:
+        cfg = synth.CONFIGS[5]
+        L, Hq, Hkv, d, B = args.layers, cfg["Hq"], cfg["Hkv"], cfg["d"], args.batch or cfg["B"]
+        K, delta, prompt = cfg["budget"], cfg["cadence"], cfg["T"]
+        R, alive = cfg["steps"] // delta, prompt + delta
+        T = prompt + R * delta
+        g = torch.Generator(device=dev)
+        g.manual_seed(0)
+        u = torch.rand((R, B, L, alive), device=dev, generator=g)
+        ks = torch.sort(torch.topk(u, K, dim=-1).indices, dim=-1).values.to(torch.int32).contiguous()
+        del u
+        budget = torch.full((R, B), K, dtype=torch.int32, device=dev)
+        alive_before = torch.full((R, B), alive, dtype=torch.int32, device=dev)
+        total_before = (alive + delta * torch.arange(R, device=dev, dtype=torch.int32))[:, None].repeat(1, B).contiguous()
+        pos = torch.empty((R, B, L, K), dtype=torch.int32, device=dev)
+        cnt = torch.empty((R, B, L), dtype=torch.int32, device=dev)
+        ngc.ngc_replay_visibility(ks, budget, alive_before, total_before, 1, alive, pos, cnt, status=st)
+        c = synth.make_cache(L, B, Hq, Hkv, d, torch.bfloat16, [T] * B, capacity=T, seed=0, device=dev)
+        dc = ngc.NgcCache(c.k, c.v, c.seq_off, c.lens, Hq, T)
+        q = synth.normal((L, B, Hq, T, d), 1, torch.bfloat16, device=dev)
+        out = torch.empty((L, B, Hq, T, d), dtype=torch.bfloat16, device=dev)
+        ms = best_of(lambda: ngc.ngc_replay_attn(dc, q, out, pos, cnt, total_before, lists=ngc.LISTS_PER_LAYER, status=st), args.steps)
+        vis = sum(t + 1 for t in range(alive)) + sum(sum(K + s + 1 for s in range(min(delta, T - (alive + (r - 1) * delta)))) for r in range(1, R + 1))
+        flops = 4.0 * d * vis * Hq * L * B
+        tf_peak = 1590.0
+        pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(pk):
+            with open(pk) as f:
+                tf_peak = float(json.load(f)["bf16_tflops"])
+        res = {"kernel": "ngc_replay_attn", "workload": f"config-5 history: {L} layers, B={B}, T={T}, {R} rounds, {K} kept per round and layer",
+               "ms": round(ms, 3),
+               "roofline": {"bound": "tensor", "achieved": round(flops / ms / 1e9, 1), "peak": tf_peak, "unit": "TFLOP/s",
+                            "frac": round(flops / ms / 1e9 / tf_peak, 4), "flops": "4*d per visible key per query per head (masked keys not counted)"}}
+    torch.cuda.synchronize()
+    res["dev_status"] = int(st.item())
+    print(json.dumps(res), flush=True)
+
+
 # ------------------------------------------------------------------------------------ CPU oracle arm
 
 def oracle_step(cache_np, logits, q, nk, nv, qr, K, rnd, decode_steps, seed):
@@ -564,6 +641,9 @@ def main():
     ap.add_argument("--cpu-decode-steps", type=int, default=48)
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5, 6, 7],
                     help="2 = the benchmark workload (default); 3..7 = the other workloads, one GPU, per-phase timing only")
+    ap.add_argument("--kernel", default=None, choices=["score_backward", "replay_attn"],
+                    help="time one training-side call instead of the benchmark step (one GPU)")
+    ap.add_argument("--layers", type=int, default=4, help="--kernel replay_attn: layers of the history to run")
     ap.add_argument("--paged", action="store_true", help="--config 6|7 only: paged cache, one eviction unit = one page")
     ap.add_argument("--ring", type=int, default=8, help="distinct decode-input steps kept on the device for --config 3|4|5")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per decode launch from an ncu capture (profiles/)")
@@ -575,7 +655,9 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the CPU oracle")
-        if args.config != 2:
+        if args.kernel:
+            run_kernel(args)
+        elif args.config != 2:
             run_other(args)
         else:
             run_ngc(args)

@@ -188,9 +188,13 @@ score_bwd_stats_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
 
     for (int i = 0; i < it.n_tiles; ++i) {
       const int s = i % kStagesA;
+      const int t_base = (it.tile_lo + i) * kTileT + 16 * warp;
+      // the tokens' upstream weights are fetched before the wait, so that their latency hides behind it
+      const int t0 = t_base + gid, t1 = t0 + 8;
+      const float P0 = token_weight(p, it.b, it.gi, t0, T_b, inv_rows);
+      const float P1 = token_weight(p, it.b, it.gi, t1, T_b, inv_rows);
       if (!ptx::mbar_wait_bounded(&bar_full[s], (i / kStagesA) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
       const uint32_t k_st = ptx::smem_u32(stage_base + s * kStageBytes);
-      const int t_base = (it.tile_lo + i) * kTileT + 16 * warp;
       if (t_base < T_b) {
         float acc[NT][4];
 #pragma unroll
@@ -204,9 +208,6 @@ score_bwd_stats_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
 #pragma unroll
           for (int t8 = 0; t8 < NT; ++t8) ptx::mma_bf16_16816(acc[t8], a, qb[t8][ks][0], qb[t8][ks][1]);
         }
-        const int t0 = t_base + gid, t1 = t0 + 8;
-        const float P0 = token_weight(p, it.b, it.gi, t0, T_b, inv_rows);
-        const float P1 = token_weight(p, it.b, it.gi, t1, T_b, inv_rows);
 #pragma unroll
         for (int t8 = 0; t8 < NT; ++t8)
 #pragma unroll
@@ -336,11 +337,14 @@ score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
 
   for (int i = 0; i < it.n_tiles; ++i) {
     const int s = i % kStagesB;
+    const int t_base = (it.tile_lo + i) * kTileT + 16 * warp;
+    const int t0 = t_base + gid, t1 = t0 + 8;
+    const float P0 = token_weight(p, it.b, it.gi, t0, T_b, inv_rows);       // fetched ahead of the wait
+    const float P1 = token_weight(p, it.b, it.gi, t1, T_b, inv_rows);
     if (!ptx::mbar_wait_bounded(&bar_full[s], (i / kStagesB) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
     uint8_t* st = stage_base + s * kStageBytes;
     const uint32_t k_st = ptx::smem_u32(st);
     const uint32_t dz_buf = dz_u32 + (uint32_t)(i & 1) * kDzBytes;
-    const int t_base = (it.tile_lo + i) * kTileT + 16 * warp;
     const int valid = T_b - t_base;                       // live tokens of this warp's slice
     if (valid < 16) {
       // rows beyond the sequence may hold anything; every warp multiplies them by dz = 0 below: zero them
@@ -369,9 +373,6 @@ score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
       }
     }
     // ---- dz = A (P - c) / sqrt(d), packed to bf16: lo = token gid, hi = token gid + 8 ----
-    const int t0 = t_base + gid, t1 = t0 + 8;
-    const float P0 = token_weight(p, it.b, it.gi, t0, T_b, inv_rows);
-    const float P1 = token_weight(p, it.b, it.gi, t1, T_b, inv_rows);
     uint32_t lo[6], hi[6];
 #pragma unroll
     for (int t8 = 0; t8 < 6; ++t8) {
