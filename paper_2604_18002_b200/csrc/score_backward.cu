@@ -73,9 +73,9 @@ __device__ __forceinline__ void merge3(float& m, float& s, float& n, float mo, f
 // dL/dA of a token for the rows of list gi (0 beyond the sequence)
 __device__ __forceinline__ float token_weight(const BwdParams& p, int b, int gi, int t, int T_b, float inv_rows) {
   if (t >= T_b) return 0.f;
-  const int u = t / p.block;
+  const int u = p.block == 1 ? t : t / p.block;
   if (u >= p.n_max) return 0.f;
-  const int size = min((u + 1) * p.block, T_b) - u * p.block;
+  const int size = p.block == 1 ? 1 : min((u + 1) * p.block, T_b) - u * p.block;
   const int64_t idx = ((int64_t)b * p.G + gi) * p.n_max + u;
   float up = p.grad_logits[idx];
   if (p.log_transform) up *= __expf(-p.logits[idx]);        // d log s = ds / s
@@ -208,14 +208,19 @@ score_bwd_stats_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
 #pragma unroll
           for (int t8 = 0; t8 < NT; ++t8) ptx::mma_bf16_16816(acc[t8], a, qb[t8][ks][0], qb[t8][ks][1]);
         }
+        // tokens of this slice that some row cannot see: the window itself and the tail beyond T_b
+        const bool masked = t_base + 16 > T_b - p.w;
 #pragma unroll
         for (int t8 = 0; t8 < NT; ++t8)
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            const float a0 = t0 <= lim[t8][e] ? acc[t8][e] : -INFINITY;
-            const float a1 = t1 <= lim[t8][e] ? acc[t8][e + 2] : -INFINITY;
+            float a0 = acc[t8][e], a1 = acc[t8][e + 2];
+            if (masked) {
+              a0 = t0 <= lim[t8][e] ? a0 : -INFINITY;
+              a1 = t1 <= lim[t8][e] ? a1 : -INFINITY;
+            }
             const float mx = fmaxf(fmaxf(m_run[t8][e], a0), a1);
-            const float ms = mx == -INFINITY ? 0.f : mx;
+            const float ms = masked && mx == -INFINITY ? 0.f : mx;
             const float neg = -ms * p.scale_log2;
             const float e_old = ptx::ex2_approx(fmaf(m_run[t8][e], p.scale_log2, neg));
             const float e0 = ptx::ex2_approx(fmaf(a0, p.scale_log2, neg));
