@@ -5,11 +5,10 @@
 // image of the fp32 key, sorted descending by a STABLE sort of the candidates
 // taken in index order.
 //  * Lists of up to kSampleSmemMaxUnits candidates: least-significant-digit
-//    radix sort in shared memory, four passes of 8 bits.  Each warp owns a
-//    contiguous segment of the list; per pass it counts its digits (lanes with
-//    equal digits found with one ballot per digit bit, counted with popc), a
-//    CTA-wide prefix scan over (digit, warp) turns the counts into output
-//    offsets, and the warp walks its segment again scattering 16-bit candidate
+//    radix sort in shared memory, seven passes of 5 bits.  Each thread owns a
+//    run of consecutive candidates and a private counter per digit; a CTA-wide
+//    prefix scan over (digit, thread) turns the counts into stable output
+//    offsets, and the thread walks its run again scattering 16-bit candidate
 //    indices to their ranks.  No atomics.
 //  * Longer lists: 64-bit composite keys (image, inverted index) ordered by a
 //    bitonic network in the caller's workspace.
@@ -69,19 +68,6 @@ __device__ __forceinline__ uint32_t float_image(float f) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// Lanes of the warp that are live and hold the same 8-bit digit as the caller: one ballot per
-// digit bit (match.any costs one round per distinct value, about thirty here).
-__device__ __forceinline__ uint32_t same_digit_lanes(uint32_t d, bool live) {
-  uint32_t peers = __ballot_sync(0xffffffffu, live);
-#pragma unroll
-  for (int bit = 0; bit < 8; ++bit) {
-    const bool one = (d >> bit) & 1u;
-    const uint32_t bal = __ballot_sync(0xffffffffu, one);
-    peers &= one ? bal : ~bal;
-  }
-  return peers;
-}
-
 struct SampleParams {
   const float* logits;
   const int32_t* n;
@@ -123,16 +109,17 @@ __global__ void sample_kernel(SampleParams p) {
   uint32_t* img = nullptr;             // [n_max] key images (radix)
   uint16_t* idx_a = nullptr;           // [n_max] candidate order, ping
   uint16_t* idx_b = nullptr;           // [n_max] pong
-  uint16_t* hist = nullptr;            // [n_warps][256] digit counts, then output offsets
+  uint16_t* hist = nullptr;            // [32 digits][threads] private digit counts, then output offsets (padded)
   unsigned long long* keys = nullptr;  // composite keys (bitonic)
   uint32_t* bitmap;
   if (kRadix) {
     const int n_al = (p.n_max + 7) & ~7;
+    const int n_slots = max(p.pad_max, nthr);          // order arrays: a power-of-two run per thread
     img = reinterpret_cast<uint32_t*>(smem_raw);
     idx_a = reinterpret_cast<uint16_t*>(smem_raw + (size_t)n_al * 4);
-    idx_b = idx_a + n_al;
-    hist = idx_b + n_al;
-    bitmap = reinterpret_cast<uint32_t*>(hist + 256 * n_warps);
+    idx_b = idx_a + n_slots;
+    hist = idx_b + n_slots;
+    bitmap = reinterpret_cast<uint32_t*>(hist + 34 * nthr);
   } else {
     keys = p.ws_keys + (int64_t)li * p.pad_max;
     bitmap = reinterpret_cast<uint32_t*>(smem_raw);
@@ -167,7 +154,6 @@ __global__ void sample_kernel(SampleParams p) {
           kf = __fadd_rn(kf, 0.0f);                       // -0 -> +0
           if (kRadix) {
             img[i - P] = float_image(kf);
-            idx_a[i - P] = (uint16_t)(i - P);
           } else {
             keys[i - P] = ((unsigned long long)float_image(kf) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
           }
@@ -187,37 +173,42 @@ __global__ void sample_kernel(SampleParams p) {
     return;
   }
 
+  int order_per_log = 0, order_per = 1;        // how the sorted order is laid out (radix path)
   if (kRadix) {
-    // ---- stable LSD radix sort of the candidate order, descending image ----
-    // warp w owns candidates [w*seg, (w+1)*seg), seg a multiple of 32
-    const int seg = (((n_cand + n_warps - 1) / n_warps) + 31) & ~31;
-    const int seg_lo = min(n_cand, warp * seg), seg_hi = min(n_cand, seg_lo + seg);
-    const uint32_t lt_mask = (1u << lane) - 1u;
+    // ---- stable LSD radix sort of the candidate order, descending image: 7 passes of 5 bits ----
+    // Thread t owns the consecutive candidates [t*per, (t+1)*per) and a private counter per digit,
+    // cnt[digit][t]; in (digit, thread) order the counters' prefix sums are the stable output
+    // offsets.  No atomics, no inter-thread traffic inside the counting and scattering walks.
+    // Thread t owns the `per` consecutive positions [t*per, (t+1)*per) of the order (per a power of
+    // two); position i is STORED at (i % per) * nthr + i / per, so that the lanes of a warp walking
+    // their runs in step touch consecutive shared-memory words.
+    int per_log = 0;
+    while ((nthr << per_log) < n_cand) ++per_log;
+    const int per = 1 << per_log;
     uint16_t* src = idx_a;
     uint16_t* dst = idx_b;
-    for (int shift = 0; shift < 32 && Kp > 0; shift += 8) {
-      for (int i = tid; i < 256 * n_warps; i += nthr) hist[i] = 0;
+    for (int k = 0; k < per; ++k) {
+      const int i = tid * per + k;
+      if (i < n_cand) src[k * nthr + tid] = (uint16_t)i;
+    }
+    // counter x = digit * nthr + thread sits at cnt[x + 2 * (x >> 5)]: one pad word per 32 counters, so that
+    // the 32 consecutive counters a thread scans start in a different bank for every lane
+    uint32_t* cnt_words = reinterpret_cast<uint32_t*>(hist);
+    for (int shift = 0; shift < 32 && Kp > 0; shift += 5) {
+      for (int i = tid; i < 17 * nthr; i += nthr) cnt_words[i] = 0u;
       __syncthreads();
-      // count: the lowest lane of each group of equal digits adds the group's size
-      for (int i0 = seg_lo; i0 < seg_hi; i0 += 32) {
-        const int i = i0 + lane;
-        const bool live = i < seg_hi;
-        const uint32_t d = live ? 255u - ((img[src[i]] >> shift) & 255u) : 0u;
-        const uint32_t peers = same_digit_lanes(d, live);
-        if (live && (peers & lt_mask) == 0) hist[warp * 256 + d] += (uint16_t)__popc(peers);
-        __syncwarp();
+      for (int k = 0; k < per && tid * per + k < n_cand; ++k) {
+        const uint32_t d = 31u - ((img[src[k * nthr + tid]] >> shift) & 31u);
+        const uint32_t x = d * nthr + tid;
+        hist[x + 2 * (x >> 5)] += 1;
       }
       __syncthreads();
-      // exclusive scan in (digit, warp) order, 8 consecutive entries of that order per thread
-      // (the counters are stored [warp][digit] so that the walks above and below spread over the banks)
       {
-        int c[8], sum = 0;
+        uint32_t* mine = cnt_words + 17 * tid;          // counters 32*tid .. 32*tid + 31 of the scan order
+        uint32_t wv[16];
+        int sum = 0;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int q = 8 * tid + e;
-          c[e] = hist[(q % n_warps) * 256 + q / n_warps];
-          sum += c[e];
-        }
+        for (int e = 0; e < 16; ++e) { wv[e] = mine[e]; sum += (int)(wv[e] & 0xFFFFu) + (int)(wv[e] >> 16); }
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -229,29 +220,25 @@ __global__ void sample_kernel(SampleParams p) {
         int run = incl - sum;
         for (int w2 = 0; w2 < warp; ++w2) run += s_warp_tot[w2];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int q = 8 * tid + e;
-          hist[(q % n_warps) * 256 + q / n_warps] = (uint16_t)run;
-          run += c[e];
+        for (int e = 0; e < 16; ++e) {
+          const int c0 = (int)(wv[e] & 0xFFFFu), c1 = (int)(wv[e] >> 16);
+          mine[e] = (uint32_t)run | ((uint32_t)(run + c0) << 16);
+          run += c0 + c1;
         }
       }
       __syncthreads();
-      // scatter: rank = offset of (digit, warp) + position inside the group
-      for (int i0 = seg_lo; i0 < seg_hi; i0 += 32) {
-        const int i = i0 + lane;
-        const bool live = i < seg_hi;
-        const uint16_t cand = live ? src[i] : (uint16_t)0;
-        const uint32_t d = live ? 255u - ((img[cand] >> shift) & 255u) : 0u;
-        const uint32_t peers = same_digit_lanes(d, live);
-        if (live) dst[hist[warp * 256 + d] + __popc(peers & lt_mask)] = cand;
-        __syncwarp();
-        if (live && (peers & lt_mask) == 0) hist[warp * 256 + d] += (uint16_t)__popc(peers);
-        __syncwarp();
+      for (int k = 0; k < per && tid * per + k < n_cand; ++k) {
+        const uint16_t cand = src[k * nthr + tid];
+        const uint32_t d = 31u - ((img[cand] >> shift) & 31u);
+        const uint32_t x = d * nthr + tid;
+        const uint32_t pos = hist[x + 2 * (x >> 5)]++;
+        dst[(pos & (per - 1)) * nthr + (pos >> per_log)] = cand;
       }
       __syncthreads();
       uint16_t* t = src; src = dst; dst = t;
     }
     idx_a = src;        // the sorted order
+    order_per_log = per_log; order_per = per;
   } else {
     // ---- bitonic sort, descending ----
     for (int k = 2; k <= pad; k <<= 1) {
@@ -282,7 +269,8 @@ __global__ void sample_kernel(SampleParams p) {
   for (int j = tid; j < p.k_max; j += nthr) {
     int idx = -1;
     if (j < Kp) {
-      idx = kRadix ? P + (int)idx_a[j] : (int)(0xFFFFFFFFu - (uint32_t)(keys[j] & 0xFFFFFFFFull));
+      idx = kRadix ? P + (int)idx_a[(j & (order_per - 1)) * nthr + (j >> order_per_log)]
+                   : (int)(0xFFFFFFFFu - (uint32_t)(keys[j] & 0xFFFFFFFFull));
       atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
     }
     ko[j] = idx;
@@ -425,7 +413,8 @@ extern "C" int ngc_sample_evict(const float* logits, const int32_t* n, const int
     sample_tiny_kernel<<<(grid + kTinyWarps - 1) / kTinyWarps, kTinyWarps * 32, 0, (cudaStream_t)stream>>>(p, (int)grid);
   } else if (n_max <= kSampleSmemMaxUnits) {
     const size_t n_al = (size_t)((n_max + 7) & ~7);
-    const size_t smem = n_al * 4 + 2 * n_al * 2 + (size_t)256 * (threads / 32) * 2 + bitmap_bytes;
+    const size_t n_slots = (size_t)(p.pad_max > threads ? p.pad_max : threads);
+    const size_t smem = n_al * 4 + 2 * n_slots * 2 + (size_t)34 * threads * 2 + bitmap_bytes;
     if (smem > 48 * 1024)
       NGC_CUDA_TRY(cudaFuncSetAttribute(sample_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     sample_kernel<true><<<grid, threads, smem, (cudaStream_t)stream>>>(p);
