@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(kThreads, 3) replay_attn_kernel(ReplayAttnPara
   extern __shared__ uint8_t smem_dyn[];
   // key sources of this query tile: the kept lists of the rounds it straddles, then the contiguous run
   __shared__ int s_seg_rho[kMaxSeg], s_seg_n[kMaxSeg], s_seg_first[kMaxSeg + 1];
-  __shared__ int s_nseg, s_clo;
+  __shared__ int s_nseg, s_clo, s_uniform;
 
   uint8_t* stage = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -96,9 +96,11 @@ __global__ void __launch_bounds__(kThreads, 3) replay_attn_kernel(ReplayAttnPara
     ++nseg;
     s_seg_first[nseg] = first;
     s_nseg = nseg;
+    s_uniform = r_lo == r_hi;                     // every query of the tile lies in the same block
   }
   __syncthreads();
   const int nseg = s_nseg, c_lo = s_clo, n_tiles = s_seg_first[nseg];
+  const bool uniform = s_uniform != 0;
 
   // this thread's two query rows: position, round index, first position of its own block
   const int t_row[2] = {q0 + 16 * warp + gid, q0 + 16 * warp + gid + 8};
@@ -194,23 +196,36 @@ __global__ void __launch_bounds__(kThreads, 3) replay_attn_kernel(ReplayAttnPara
       }
     }
     // ---- visibility and online softmax (log2 domain) ----
+    // a tile needs no mask when every query of the CTA lies in one block and the tile is a full
+    // tile of that block's kept list, or lies entirely before the first query
+    const bool need_mask = !uniform || (rho >= 1 ? n_here < kKTile : c_lo + kt * kKTile + kKTile - 1 > q0);
     float mx[2] = {-INFINITY, -INFINITY};
+    if (need_mask) {
 #pragma unroll
-    for (int n8 = 0; n8 < 8; ++n8)
+      for (int n8 = 0; n8 < 8; ++n8)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int jj = 8 * n8 + 2 * tig + (e & 1), r = e >> 1;
-        bool vis;
-        if (rho >= 1) {
-          vis = jj < n_here && blk[r] == rho;                       // a kept entry of the round before this row's block
-        } else {
-          const int j = c_lo + kt * kKTile + jj;                    // a token of the row's own block, causal
-          vis = j >= lo_row[r] && j <= t_row[r];
+        for (int e = 0; e < 4; ++e) {
+          const int jj = 8 * n8 + 2 * tig + (e & 1), r = e >> 1;
+          bool vis;
+          if (rho >= 1) {
+            vis = jj < n_here && blk[r] == rho;                       // a kept entry of the round before this row's block
+          } else {
+            const int j = c_lo + kt * kKTile + jj;                    // a token of the row's own block, causal
+            vis = j >= lo_row[r] && j <= t_row[r];
+          }
+          const float z = vis ? sc[n8][e] * p.scale_log2 : -INFINITY;
+          sc[n8][e] = z;
+          mx[r] = fmaxf(mx[r], z);
         }
-        const float z = vis ? sc[n8][e] * p.scale_log2 : -INFINITY;
-        sc[n8][e] = z;
-        mx[r] = fmaxf(mx[r], z);
-      }
+    } else {
+#pragma unroll
+      for (int n8 = 0; n8 < 8; ++n8)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          sc[n8][e] *= p.scale_log2;
+          mx[e >> 1] = fmaxf(mx[e >> 1], sc[n8][e]);
+        }
+    }
     float alpha[2], m_use[2];
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
