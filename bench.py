@@ -37,8 +37,9 @@ from paper_2604_18002_b200 import synth
 
 CFG = dict(synth.CONFIGS[2])
 WORKLOAD = "config2: 1.5B-shaped GQA rollout step (L28, 12q/2kv, d128, bf16, B64, 4096->2048 tokens, 256 decode steps)"
-# the other workloads (--config 3|4|5) are measurement aids; the default line is always config 2
+# the other workloads (--config 1, 3..7) are measurement aids; the default line is always config 2
 OTHER_WORKLOADS = {
+    1: "config1: tiny single-layer check (L1, 4q/4kv, d64, fp32, B4, 512 tokens of which 64 protected -> 256, 64 decode steps)",
     3: "config3: 7B-shaped ragged batch (L28, 28q/4kv, d128, bf16, B256, lengths 1024..8192 -> ceil(len/3), 128 decode steps)",
     4: "config4: per-(layer, KV head) eviction (L28, 12q/2kv, d128, bf16, B128, 16384 -> 8192 tokens, 7168 lists, 64 decode steps)",
     5: "config5: rollout loop (L28, 12q/2kv, d128, bf16, B64, 256 prompt + 8192 generated, a round every 512 tokens 768 -> 256, "
@@ -312,7 +313,7 @@ def run_other(args):
     cid = args.config
     cfg = synth.CONFIGS[cid]
     L, B, Hq, Hkv, d, steps = cfg["L"], args.batch or cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["d"], args.decode_steps or cfg["steps"]
-    dtype = torch.bfloat16
+    dtype = torch.float32 if cfg["dtype"] == "f32" else torch.bfloat16
     lists = cfg["lists"]
     loop = cid >= 5                      # grow-then-evict loop (rounds) instead of one round + decode
     block = cfg.get("block", 1)
@@ -342,12 +343,13 @@ def run_other(args):
     lens0 = lens.to(dev)
     logits = ro.score_logits if from_score else synth.make_logits(B, G, n_max, seed=cfg["data_seed"] + 7, std=cfg["logit_std"], device=dev)
     n_t, k_t = n_evict.to(dev), budget.to(dev)
-    ring = min(steps, args.ring)
+    p_t = torch.full((B,), cfg["n_protect"], dtype=torch.int32, device=dev) if cfg["n_protect"] else None
+    ring = ((cadence if loop else steps) if args.graph else min(steps, args.ring))
     q = synth.make_queries(L, B, Hq, d, dtype, seed=11, steps=ring, device=dev)
     nk, nv = synth.make_new_kv(L, B, Hkv, d, dtype, seed=13, steps=ring, device=dev)
     q_recent = synth.normal((L, B, Hq, W_RECENT, d), 17, dtype, device=dev)
     out = torch.empty((ring, L, B, Hq, d), dtype=torch.float32, device=dev)
-    row_bytes = L * Hkv * 2 * d * 2
+    row_bytes = L * Hkv * 2 * d * (4 if dtype == torch.float32 else 2)
     names = ["score", "sample", "logprob", "compact", "decode", "recompute"]
     acc = {n: [] for n in names}
 
@@ -372,9 +374,9 @@ def run_other(args):
         else:
             ngc.ngc_score_evict(ro.cache, q_recent, ro.block, lists, ro.score_logits, ws=ro.ws_score, status=ro.status)
         e[1].record()
-        ngc.ngc_sample_evict(logits, n_t, None, k_t, cfg["noise_seed"], rnd, ro.kept_order, ro.kept_sorted, None, ws=ro.ws_sample, status=ro.status)
+        ngc.ngc_sample_evict(logits, n_t, p_t, k_t, cfg["noise_seed"], rnd, ro.kept_order, ro.kept_sorted, None, ws=ro.ws_sample, status=ro.status)
         e[2].record()
-        ngc.ngc_evict_logprob(logits, n_t, None, k_t, ro.kept_order, ro.logp, status=ro.status)
+        ngc.ngc_evict_logprob(logits, n_t, p_t, k_t, ro.kept_order, ro.logp, status=ro.status)
         e[3].record()
         if paged is not None:
             ngc.ngc_evict_pages(paged, ro.kept_sorted, k_t, status=ro.status)
@@ -384,9 +386,17 @@ def run_other(args):
         ro.launches += 7          # score 3, sample 1, log-prob 1, compaction 2
         t.append(e)
 
+    graph = None
+
     def decode(n, t):
         e0, e1 = ev(), ev()
         e0.record()
+        if graph is not None:
+            graph.replay()          # all decode steps of the round with one launch from the host
+            ro.launches += 2 * n
+            e1.record()
+            t.append((e0, e1))
+            return
         for s in range(n):
             if paged is not None:
                 ngc.ngc_decode_attn_paged(paged, q[s % ring], out[s % ring], nk[s % ring], nv[s % ring], ws=ro.ws_decode, status=ro.status)
@@ -430,6 +440,11 @@ def run_other(args):
         one_step(w, [])
     torch.cuda.synchronize()
     ro.check_status()
+    if args.graph:
+        assert paged is None, "--graph and --paged are separate measurements"
+        graph = ro.capture_decode_steps(q[: (cadence if loop else steps)], out, nk, nv)
+        one_step(args.warmup, [])
+        torch.cuda.synchronize()
     rec = []
     launches0 = ro.launches
     t0, t1 = ev(), ev()
@@ -467,9 +482,10 @@ def run_other(args):
     dec_gbs = vis * row_bytes / (dec_ms * 1e-3) / 1e9
     cmp_gbs = compact_bytes / (med["compact"] * 1e-3) / 1e9
     result = {"metric": "evict+compact+decode tokens/sec", "value": round(tokens / (ms_per_step * 1e-3), 1), "unit": "tokens/s", "n_gpus": 1,
-              "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "dtype": "bf16", "data": "synthetic",
+              "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "dtype": cfg["dtype"], "data": "synthetic",
               "config": {"workload": OTHER_WORKLOADS[cid], "batch": B, "decode_steps": steps, "input_ring": ring,
-                         "layout": "paged (eviction edits page tables, no K/V movement)" if paged is not None else "contiguous strips, in-place compaction"},
+                         "layout": "paged (eviction edits page tables, no K/V movement)" if paged is not None else "contiguous strips, in-place compaction",
+                         "decode_loop": "one CUDA graph per round" if args.graph else "eager launches"},
               "per_call_ms": med,
               "roofline": {"bound": "hbm", "kernel": "decode_stream_t_kernel (all decode calls of a step, launch gaps included)",
                            "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
@@ -639,11 +655,12 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seqs", type=int, default=4)
     ap.add_argument("--cpu-decode-steps", type=int, default=48)
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5, 6, 7],
-                    help="2 = the benchmark workload (default); 3..7 = the other workloads, one GPU, per-phase timing only")
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7],
+                    help="2 = the benchmark workload (default); 1, 3..7 = the other workloads, one GPU, per-phase timing only")
     ap.add_argument("--kernel", default=None, choices=["score_backward", "replay_attn"],
                     help="time one training-side call instead of the benchmark step (one GPU)")
     ap.add_argument("--layers", type=int, default=4, help="--kernel replay_attn: layers of the history to run")
+    ap.add_argument("--graph", action="store_true", help="--config 1|3..7: replay the decode calls of a round as one CUDA graph")
     ap.add_argument("--paged", action="store_true", help="--config 6|7 only: paged cache, one eviction unit = one page")
     ap.add_argument("--ring", type=int, default=8, help="distinct decode-input steps kept on the device for --config 3|4|5")
     ap.add_argument("--traffic", type=float, default=None, help="dram bytes per decode launch from an ncu capture (profiles/)")

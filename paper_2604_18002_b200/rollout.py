@@ -74,6 +74,19 @@ class NgcRollout:
         split = ngc.decode_splits(self.cache, append=new_k is not None) > 1
         self.launches += 1 + (1 if new_k is not None else 0) + (1 if split else 0)
 
+    def capture_decode_steps(self, q: torch.Tensor, out: torch.Tensor, new_k: torch.Tensor, new_v: torch.Tensor):
+        """Records the decode calls of ``q.shape[0]`` consecutive steps (step s reads ``q[s]``, ``new_k[s]``,
+        ``new_v[s]`` and writes ``out[s]``) into one CUDA graph and returns it; ``graph.replay()`` then runs all
+        of them with a single launch from the host.  For short caches and small batches a decode step is a few
+        microseconds of GPU work, less than the host needs to enqueue its kernels, so the loop is launch-bound
+        unless it is replayed as a graph.  Call ``decode_step`` once before capturing (the first call of a
+        process configures the kernels); the tensors must stay alive and in place while the graph is used."""
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for s in range(q.shape[0]):
+                self.decode_step(q[s], out[s], new_k[s], new_v[s])
+        return graph
+
     def check_status(self):
         code = int(self.status.item())
         if code != 0:
