@@ -7,11 +7,13 @@
 //    streaming kernel.  A producer warp feeds a ring of shared-memory stages
 //    with TMA tensor loads (64 tokens x 128 channels of K and of V per stage,
 //    128-byte swizzle, completion on mbarriers).  Four consumer warps each own
-//    16 tokens of a stage: S = Q K^T and O += P V run on the tensor cores
-//    (mma.sync m16n8k16, the group's query heads on the M axis, so the g heads
-//    that share a K/V row reuse it straight from shared memory), with a
-//    single-pass online softmax in fp32.  Per-warp partial states are merged
-//    through shared memory at the end of the item.
+//    16 tokens of a stage and compute the TRANSPOSED products on the tensor
+//    cores (mma.sync m16n8k16): S^T = K Q^T with the tokens on M and the
+//    group's heads on N = 8 (no padded head rows; the g heads that share a K/V
+//    row reuse it straight from shared memory), and O^T = V^T P^T with the
+//    channels on M; P^T moves from accumulator to operand layout with two
+//    movmatrix transposes.  Single-pass online softmax in fp32.  Per-warp
+//    partial states are merged through shared memory at the end of the item.
 //  * everything else (fp32 caches, d = 64, large groups): one query head per
 //    CTA, a warp per token row, fp32 FMA and warp-shuffle reductions.
 //
@@ -236,9 +238,8 @@ constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
 constexpr int kBoxBytes = kTileT * 128;       // one 64 x 64 bf16 box
 constexpr int kTileBytes = 2 * kBoxBytes;     // K (or V) tile: two boxes (channels 0-63, 64-127)
 constexpr int kStageBytes = 2 * kTileBytes;   // K + V
-constexpr int kStages = 3;
-constexpr int kTStages = 2;                   // ring depth and CTAs per SM of the variant for groups of <= 8 heads
-constexpr int kTMinCtas = 3;
+constexpr int kStages1 = 2, kMinCtas1 = 3;    // groups of <= 8 heads: 128 registers, 2-stage ring, 3 CTAs per SM
+constexpr int kStages2 = 3, kMinCtas2 = 2;    // groups of 9..16 heads: two head tiles, 3-stage ring, 2 CTAs per SM
 constexpr int kORowStride = 132;              // floats; merge buffer row stride (bank spread)
 
 // Tensor maps of a launch: K and V with the full-tile box (64 rows, or one page) and with a
@@ -280,274 +281,14 @@ __device__ __forceinline__ void issue_tile(const DecodeParams& p, const KvMaps& 
   }
 }
 
-__global__ void __launch_bounds__(kStreamThreads, 2)
-decode_stream_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
-  extern __shared__ uint8_t smem_dyn[];
-  __shared__ uint64_t bar_full[kStages], bar_empty[kStages];
-  __shared__ float sm_m[kConsumerWarps][16], sm_l[kConsumerWarps][16];
-
-  uint8_t* stage_base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int gid = lane >> 2, tig = lane & 3;
-
-  int item = blockIdx.x;
-  const int split = item % p.n_split; item /= p.n_split;
-  const int h = item % p.Hkv;
-  const int b = (item / p.Hkv) % p.B;
-  const int lr = item / (p.Hkv * p.B);
-  const int l = p.layer_begin + lr;
-  const int g = p.g;
-  const int32_t* table = p.page_table
-      ? p.page_table + ((int64_t)b * p.G + list_of(p.lists, l, h, p.Hkv)) * p.pages_cap : nullptr;
-
-  if (tid == 0) {
-#pragma unroll
-    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&bar_full[s], 1); ptx::mbar_init(&bar_empty[s], kConsumerWarps); }
-    ptx::fence_barrier_init();
-    ptx::prefetch_tensormap(&maps.k);
-    ptx::prefetch_tensormap(&maps.v);
-  }
-  ptx::grid_dep_wait();           // lens and the cache rows of earlier calls are final from here on
-  ptx::grid_dep_launch();
-
-  int len = visible_len(p, b);
-  if (len < 0) {
-    if (tid == 0) set_dev_status(p.dev_status, NGC_DEV_STRIP_FULL);
-    len = 0;
-  }
-  const int t_new = (p.append && len > 0) ? len - 1 : -1;      // position of the appended row
-  const int nt = (len + kTileT - 1) / kTileT;
-  const int tps = (nt + p.n_split - 1) / p.n_split;
-  const int tile_lo = min(nt, split * tps);
-  const int tile_hi = min(nt, tile_lo + tps);
-  const int n_tiles = tile_hi - tile_lo;
-  __syncthreads();
-
-  float o_acc[16][4];
-  float m_run[2] = {-INFINITY, -INFINITY};
-  float l_run[2] = {0.f, 0.f};
-#pragma unroll
-  for (int i = 0; i < 16; ++i) { o_acc[i][0] = 0.f; o_acc[i][1] = 0.f; o_acc[i][2] = 0.f; o_acc[i][3] = 0.f; }
-
-  if (warp == kConsumerWarps) {
-    // ------------------------------------------------ producer
-    if (lane == 0 && n_tiles > 0) {
-      const int plane = l * p.Hkv + h;
-      const int row0 = table ? 0 : (int)p.seq_off[b];
-      for (int it = 0; it < n_tiles; ++it) {
-        const int s = it % kStages;
-        if (it >= kStages) {
-          if (!ptx::mbar_wait_bounded(&bar_empty[s], ((it / kStages) - 1) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
-        }
-        issue_tile(p, maps, table, row0, b, plane, tile_lo + it, len, stage_base + s * kStageBytes, &bar_full[s]);
-      }
-    }
-    __syncwarp();
-  } else {
-    // ------------------------------------------------ consumers
-    // Q fragments (A operand): rows = heads of the group (gid, gid+8), zero beyond g.
-    uint32_t qa[8][4];
-    {
-      const uint32_t* q0 = (const uint32_t*)((const __nv_bfloat16*)p.q + (((int64_t)l * p.B + b) * p.Hq + h * g + gid) * 128);
-      const uint32_t* q1 = q0 + 8 * 64;   // 8 heads further (128 bf16 = 64 words per head)
-      const bool v0 = gid < g, v1 = gid + 8 < g;
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const int w0 = (16 * ks + 2 * tig) >> 1;
-        qa[ks][0] = v0 ? q0[w0] : 0u;
-        qa[ks][1] = v1 ? q1[w0] : 0u;
-        qa[ks][2] = v0 ? q0[w0 + 4] : 0u;
-        qa[ks][3] = v1 ? q1[w0 + 4] : 0u;
-      }
-    }
-    // lane-dependent parts of the swizzled shared-memory addresses
-    const uint32_t k_lane_off = (uint32_t)((16 * warp + (lane & 7)) * 128);
-    const uint32_t v_lane_off = (uint32_t)((16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * 128);
-    const uint32_t x7 = (uint32_t)(lane & 7);
-
-    // The appended row sits in the strip's last tile.  The warp whose slice holds it fetches the row
-    // from the caller's buffer now, long before the tile arrives: lanes 0-15 take the sixteen
-    // 16-byte pieces of the K row, lanes 16-31 those of the V row.
-    const bool own_new = t_new >= 0 && tile_hi == nt && n_tiles > 0 && ((t_new % kTileT) >> 4) == warp;
-    uint4 piece = make_uint4(0, 0, 0, 0);
-    if (own_new)
-      piece = ((const uint4*)((lane >> 4) ? p.new_v : p.new_k))[(((int64_t)l * p.B + b) * p.Hkv + h) * 16 + (lane & 15)];
-
-    for (int it = 0; it < n_tiles; ++it) {
-      const int s = it % kStages;
-      if (!ptx::mbar_wait_bounded(&bar_full[s], (it / kStages) & 1)) set_dev_status(p.dev_status, NGC_DEV_TIMEOUT);
-      uint8_t* st = stage_base + s * kStageBytes;
-      const uint32_t k_st = ptx::smem_u32(st);
-      const uint32_t v_st = k_st + kTileBytes;
-      const int tile_t0 = (tile_lo + it) * kTileT;
-      const int valid = len - tile_t0 - 16 * warp;      // live tokens in this warp's slice (may exceed 16)
-
-      if (own_new && it == n_tiles - 1) {
-        // The appended row lives in this warp's slice: take it from the caller's buffer (the tile
-        // holds whatever the cache row held before) and store it into the cache for later steps.
-        const int isv = lane >> 4, c = lane & 15, r = t_new - tile_t0;
-        uint8_t* dst = st + isv * kTileBytes + (c >> 3) * kBoxBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-        *reinterpret_cast<uint4*>(dst) = piece;
-        const int64_t row = table ? ((int64_t)b * p.pages_cap + table[t_new / p.page]) * p.page + t_new % p.page
-                                  : p.seq_off[b] + t_new;
-        ((uint4*)(isv ? p.v : p.k))[((int64_t)(l * p.Hkv + h) * p.rows + row) * 16 + c] = piece;
-        ptx::fence_proxy_async();      // the stage is refilled by TMA later: order this generic write before it
-        __syncwarp();
-      }
-      if (valid > 0) {
-        if (valid < 16) {
-          // dead V rows may hold anything (NaN x 0 would poison the sum): zero them
-          for (int i = lane; i < 16 * 16; i += 32) {
-            const int r = i >> 4, c = i & 15;
-            if (r >= valid) {
-              uint8_t* rowp = st + kTileBytes + (c >> 3) * kBoxBytes + (16 * warp + r) * 128 + (c & 7) * 16;
-              *reinterpret_cast<uint4*>(rowp) = make_uint4(0, 0, 0, 0);
-            }
-          }
-          __syncwarp();
-        }
-        // ---- S = Q K^T for 16 tokens (two n-tiles of 8) ----
-        float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-#pragma unroll
-          for (int n8 = 0; n8 < 2; ++n8) {
-            const uint32_t chunk = (uint32_t)(4 * (j & 1) + (lane >> 3));
-            const uint32_t addr = k_st + (j >> 1) * kBoxBytes + k_lane_off + n8 * (8 * 128) + ((chunk ^ x7) << 4);
-            uint32_t r0, r1, r2, r3;
-            ptx::ldmatrix_x4(addr, r0, r1, r2, r3);
-            ptx::mma_bf16_16816(sc[n8], qa[2 * j], r0, r1);
-            ptx::mma_bf16_16816(sc[n8], qa[2 * j + 1], r2, r3);
-          }
-        }
-        // ---- online softmax (log2 domain) ----
-        float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-        for (int n8 = 0; n8 < 2; ++n8) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int tok = 8 * n8 + 2 * tig + (e & 1);
-            const float z = tok < valid ? sc[n8][e] * p.scale_log2 : -INFINITY;
-            sc[n8][e] = z;
-            mx[e >> 1] = fmaxf(mx[e >> 1], z);
-          }
-        }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-        }
-        float m_new[2], alpha[2];
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          m_new[r] = fmaxf(m_run[r], mx[r]);          // finite: token 0 of the slice is live
-          alpha[r] = ptx::ex2_approx(m_run[r] - m_new[r]);
-        }
-        const bool changed = (m_new[0] != m_run[0]) || (m_new[1] != m_run[1]);
-        if (__any_sync(0xffffffffu, changed)) {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            o_acc[i][0] *= alpha[0]; o_acc[i][1] *= alpha[0];
-            o_acc[i][2] *= alpha[1]; o_acc[i][3] *= alpha[1];
-          }
-          l_run[0] *= alpha[0];
-          l_run[1] *= alpha[1];
-          m_run[0] = m_new[0];
-          m_run[1] = m_new[1];
-        }
-        uint32_t pa[4];
-        {
-          float pr[2][4];
-#pragma unroll
-          for (int n8 = 0; n8 < 2; ++n8)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              pr[n8][e] = ptx::ex2_approx(sc[n8][e] - m_run[e >> 1]);
-              l_run[e >> 1] += pr[n8][e];
-            }
-          pa[0] = ptx::pack_bf16x2(pr[0][0], pr[0][1]);
-          pa[1] = ptx::pack_bf16x2(pr[0][2], pr[0][3]);
-          pa[2] = ptx::pack_bf16x2(pr[1][0], pr[1][1]);
-          pa[3] = ptx::pack_bf16x2(pr[1][2], pr[1][3]);
-        }
-        // ---- O += P V (16 tokens x 128 channels) ----
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj) {
-          const uint32_t chunk = (uint32_t)(2 * (jj & 3) + (lane >> 4));
-          const uint32_t addr = v_st + (jj >> 2) * kBoxBytes + v_lane_off + ((chunk ^ x7) << 4);
-          uint32_t r0, r1, r2, r3;
-          ptx::ldmatrix_x4_trans(addr, r0, r1, r2, r3);
-          ptx::mma_bf16_16816(o_acc[2 * jj], pa, r0, r1);
-          ptx::mma_bf16_16816(o_acc[2 * jj + 1], pa, r2, r3);
-        }
-      }
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&bar_empty[s]);
-    }
-    // quad-reduce the row sums and publish this warp's state
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-    }
-    if (tig == 0) {
-      sm_m[warp][gid] = m_run[0]; sm_m[warp][gid + 8] = m_run[1];
-      sm_l[warp][gid] = l_run[0]; sm_l[warp][gid + 8] = l_run[1];
-    }
-  }
-  __syncthreads();   // every stage has been consumed; the ring is free for the merge buffer
-
-  float* obuf = reinterpret_cast<float*>(stage_base);      // [warp][16][kORowStride]
-  if (warp < kConsumerWarps) {
-    float f[2];
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      const int row = gid + 8 * r;
-      float mg = sm_m[0][row];
-#pragma unroll
-      for (int w = 1; w < kConsumerWarps; ++w) mg = fmaxf(mg, sm_m[w][row]);
-      f[r] = m_run[r] == -INFINITY ? 0.f : ptx::ex2_approx(m_run[r] - mg);
-    }
-    float* ob = obuf + warp * 16 * kORowStride;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      *reinterpret_cast<float2*>(ob + gid * kORowStride + 8 * i + 2 * tig) = make_float2(o_acc[i][0] * f[0], o_acc[i][1] * f[0]);
-      *reinterpret_cast<float2*>(ob + (gid + 8) * kORowStride + 8 * i + 2 * tig) = make_float2(o_acc[i][2] * f[1], o_acc[i][3] * f[1]);
-    }
-  }
-  __syncthreads();
-  if (tid < 128) {
-    const int c = tid;
-    for (int row = 0; row < g; ++row) {
-      float mg = sm_m[0][row];
-#pragma unroll
-      for (int w = 1; w < kConsumerWarps; ++w) mg = fmaxf(mg, sm_m[w][row]);
-      float o = 0.f, ls = 0.f;
-#pragma unroll
-      for (int w = 0; w < kConsumerWarps; ++w) {
-        o += obuf[(w * 16 + row) * kORowStride + c];
-        const float mw = sm_m[w][row];
-        ls += mw == -INFINITY ? 0.f : sm_l[w][row] * ptx::ex2_approx(mw - mg);
-      }
-      const int hq = h * g + row;
-      if (p.n_split == 1) {
-        store_out(p, (((int64_t)l * p.B + b) * p.Hq + hq) * 128 + c, ls > 0.f ? o / ls : 0.f);
-      } else {
-        const int64_t pit = (((int64_t)lr * p.B + b) * p.Hq + hq) * p.n_split + split;
-        p.part_o[pit * 128 + c] = o;
-        if (c == 0) p.part_ml[pit] = make_float2(mg, ls);
-      }
-    }
-  }
-}
-
-// Variant for groups of at most 8 query heads (every GQA shape in the paper's model family).
-template <int kNStages, int kMinCtas>
+// The streaming kernel.  NH = 8-head tiles of the group (1: groups of at most 8 heads, every GQA shape of
+// the paper's model family; 2: groups of 9..16 heads).
+template <int NH, int kNStages, int kMinCtas>
 __global__ void __launch_bounds__(kStreamThreads, kMinCtas)
 decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ uint64_t bar_full[kNStages], bar_empty[kNStages];
-  __shared__ float sm_m[kConsumerWarps][8], sm_l[kConsumerWarps][8];
+  __shared__ float sm_m[kConsumerWarps][8 * NH], sm_l[kConsumerWarps][8 * NH];
 
   uint8_t* stage_base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -586,12 +327,15 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
   const int n_tiles = tile_hi - tile_lo;
   __syncthreads();
 
-  // O^T accumulators: o_acc[mt] = channels 16*mt + {gid, gid+8} x heads {2*tig, 2*tig+1}
-  float o_acc[8][4];
-  float m_run[2] = {-INFINITY, -INFINITY};      // running max / sum of heads 2*tig, 2*tig+1 (log2 domain)
-  float l_run[2] = {0.f, 0.f};
+  // O^T accumulators: o_acc[t][mt] = channels 16*mt + {gid, gid+8} x heads 8*t + {2*tig, 2*tig+1}
+  float o_acc[NH][8][4];
+  float m_run[NH][2], l_run[NH][2];             // running max / sum of heads 8*t + 2*tig, + 1 (log2 domain)
 #pragma unroll
-  for (int i = 0; i < 8; ++i) { o_acc[i][0] = 0.f; o_acc[i][1] = 0.f; o_acc[i][2] = 0.f; o_acc[i][3] = 0.f; }
+  for (int t = 0; t < NH; ++t) {
+    m_run[t][0] = -INFINITY; m_run[t][1] = -INFINITY; l_run[t][0] = 0.f; l_run[t][1] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { o_acc[t][i][0] = 0.f; o_acc[t][i][1] = 0.f; o_acc[t][i][2] = 0.f; o_acc[t][i][3] = 0.f; }
+  }
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------ producer
@@ -610,16 +354,17 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
   } else {
     // ------------------------------------------------ consumers
     // Transposed products: S^T = K Q^T (16 tokens x 8 heads) and O^T = V^T P^T (128 channels x 8
-    // heads), so the at most 8 heads of the group sit on the N = 8 axis of the MMA with no padding.
+    // heads) per tile of 8 heads, so the heads of the group sit on the N = 8 axis of the MMA.
     // Q^T fragments (B operand, column n = head gid): zero beyond g.
-    uint32_t qb[8][2];
-    {
-      const uint32_t* q0 = (const uint32_t*)((const __nv_bfloat16*)p.q + (((int64_t)l * p.B + b) * p.Hq + h * g + gid) * 128);
-      const bool live = gid < g;
+    uint32_t qb[NH][8][2];
+#pragma unroll
+    for (int t = 0; t < NH; ++t) {
+      const uint32_t* q0 = (const uint32_t*)((const __nv_bfloat16*)p.q + (((int64_t)l * p.B + b) * p.Hq + h * g + 8 * t + gid) * 128);
+      const bool live = 8 * t + gid < g;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
-        qb[ks][0] = live ? q0[8 * ks + tig] : 0u;
-        qb[ks][1] = live ? q0[8 * ks + tig + 4] : 0u;
+        qb[t][ks][0] = live ? q0[8 * ks + tig] : 0u;
+        qb[t][ks][1] = live ? q0[8 * ks + tig + 4] : 0u;
       }
     }
     // lane-dependent parts of the swizzled shared-memory addresses
@@ -665,62 +410,73 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
           __syncwarp();
         }
         // ---- S^T = K Q^T: 16 tokens x 8 heads ----
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};     // (tok gid, head 2tig), (gid, 2tig+1), (gid+8, 2tig), (gid+8, 2tig+1)
+        float sc[NH][4];                        // (tok gid, head 2tig), (gid, 2tig+1), (gid+8, 2tig), (gid+8, 2tig+1)
+#pragma unroll
+        for (int t = 0; t < NH; ++t) { sc[t][0] = 0.f; sc[t][1] = 0.f; sc[t][2] = 0.f; sc[t][3] = 0.f; }
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
           const uint32_t chunk = (uint32_t)(2 * (ks & 3) + (lane >> 4));
           const uint32_t addr = k_st + (ks >> 2) * kBoxBytes + k_lane_off + ((chunk ^ x7) << 4);
           uint32_t a[4];
           ptx::ldmatrix_x4(addr, a[0], a[1], a[2], a[3]);
-          ptx::mma_bf16_16816(sc, a, qb[ks][0], qb[ks][1]);
+#pragma unroll
+          for (int t = 0; t < NH; ++t) ptx::mma_bf16_16816(sc[t], a, qb[t][ks][0], qb[t][ks][1]);
         }
         // ---- online softmax per head (log2 domain) ----
-        sc[0] = gid < valid ? sc[0] * p.scale_log2 : -INFINITY;
-        sc[1] = gid < valid ? sc[1] * p.scale_log2 : -INFINITY;
-        sc[2] = gid + 8 < valid ? sc[2] * p.scale_log2 : -INFINITY;
-        sc[3] = gid + 8 < valid ? sc[3] * p.scale_log2 : -INFINITY;
-        float mx[2] = {fmaxf(sc[0], sc[2]), fmaxf(sc[1], sc[3])};
+        uint32_t pb[NH][2];
+        bool changed = false;
+        float alpha[NH][2];
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 4));
-          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 8));
-          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 16));
-        }
-        float m_new[2], alpha[2];
+        for (int t = 0; t < NH; ++t) {
+          sc[t][0] = gid < valid ? sc[t][0] * p.scale_log2 : -INFINITY;
+          sc[t][1] = gid < valid ? sc[t][1] * p.scale_log2 : -INFINITY;
+          sc[t][2] = gid + 8 < valid ? sc[t][2] * p.scale_log2 : -INFINITY;
+          sc[t][3] = gid + 8 < valid ? sc[t][3] * p.scale_log2 : -INFINITY;
+          float mx[2] = {fmaxf(sc[t][0], sc[t][2]), fmaxf(sc[t][1], sc[t][3])};
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          m_new[r] = fmaxf(m_run[r], mx[r]);          // finite: token 0 of the slice is live
-          alpha[r] = ptx::ex2_approx(m_run[r] - m_new[r]);
+          for (int r = 0; r < 2; ++r) {
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 4));
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 8));
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 16));
+            const float m_new = fmaxf(m_run[t][r], mx[r]);          // finite: token 0 of the slice is live
+            alpha[t][r] = ptx::ex2_approx(m_run[t][r] - m_new);
+            changed = changed || m_new != m_run[t][r];
+            m_run[t][r] = m_new;
+          }
         }
-        const bool changed = (m_new[0] != m_run[0]) || (m_new[1] != m_run[1]);
         if (__any_sync(0xffffffffu, changed)) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            o_acc[i][0] *= alpha[0]; o_acc[i][1] *= alpha[1];
-            o_acc[i][2] *= alpha[0]; o_acc[i][3] *= alpha[1];
-          }
-          l_run[0] *= alpha[0];
-          l_run[1] *= alpha[1];
-          m_run[0] = m_new[0];
-          m_run[1] = m_new[1];
-        }
-        float pr[4];
+          for (int t = 0; t < NH; ++t) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          pr[e] = ptx::ex2_approx(sc[e] - m_run[e & 1]);
-          l_run[e & 1] += pr[e];
+            for (int i = 0; i < 8; ++i) {
+              o_acc[t][i][0] *= alpha[t][0]; o_acc[t][i][1] *= alpha[t][1];
+              o_acc[t][i][2] *= alpha[t][0]; o_acc[t][i][3] *= alpha[t][1];
+            }
+            l_run[t][0] *= alpha[t][0];
+            l_run[t][1] *= alpha[t][1];
+          }
         }
-        // P^T as B operand (k = token, n = head): transpose the two 8 x 8 (token x head) blocks
-        const uint32_t pb0 = ptx::movmatrix_trans(ptx::pack_bf16x2(pr[0], pr[1]));
-        const uint32_t pb1 = ptx::movmatrix_trans(ptx::pack_bf16x2(pr[2], pr[3]));
-        // ---- O^T += V^T P^T (128 channels x 8 heads) ----
+#pragma unroll
+        for (int t = 0; t < NH; ++t) {
+          float pr[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            pr[e] = ptx::ex2_approx(sc[t][e] - m_run[t][e & 1]);
+            l_run[t][e & 1] += pr[e];
+          }
+          // P^T as B operand (k = token, n = head): transpose the two 8 x 8 (token x head) blocks
+          pb[t][0] = ptx::movmatrix_trans(ptx::pack_bf16x2(pr[0], pr[1]));
+          pb[t][1] = ptx::movmatrix_trans(ptx::pack_bf16x2(pr[2], pr[3]));
+        }
+        // ---- O^T += V^T P^T (128 channels x 8 heads per tile of heads) ----
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) {
           const uint32_t chunk = (uint32_t)(2 * (mt & 3) + ((lane >> 3) & 1));
           const uint32_t addr = v_st + (mt >> 2) * kBoxBytes + v_lane_off + ((chunk ^ x7) << 4);
           uint32_t a[4];
           ptx::ldmatrix_x4_trans(addr, a[0], a[1], a[2], a[3]);
-          ptx::mma_bf16_16816(o_acc[mt], a, pb0, pb1);
+#pragma unroll
+          for (int t = 0; t < NH; ++t) ptx::mma_bf16_16816(o_acc[t][mt], a, pb[t][0], pb[t][1]);
         }
       }
       __syncwarp();
@@ -728,36 +484,42 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
     }
     // row sums over the tokens of the slice (spread over gid), then publish this warp's state
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 4);
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 8);
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 16);
-    }
-    if (gid == 0) {
-      sm_m[warp][2 * tig] = m_run[0]; sm_m[warp][2 * tig + 1] = m_run[1];
-      sm_l[warp][2 * tig] = l_run[0]; sm_l[warp][2 * tig + 1] = l_run[1];
+    for (int t = 0; t < NH; ++t) {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        l_run[t][r] += __shfl_xor_sync(0xffffffffu, l_run[t][r], 4);
+        l_run[t][r] += __shfl_xor_sync(0xffffffffu, l_run[t][r], 8);
+        l_run[t][r] += __shfl_xor_sync(0xffffffffu, l_run[t][r], 16);
+      }
+      if (gid == 0) {
+        sm_m[warp][8 * t + 2 * tig] = m_run[t][0]; sm_m[warp][8 * t + 2 * tig + 1] = m_run[t][1];
+        sm_l[warp][8 * t + 2 * tig] = l_run[t][0]; sm_l[warp][8 * t + 2 * tig + 1] = l_run[t][1];
+      }
     }
   }
   __syncthreads();   // every stage has been consumed; the ring is free for the merge buffer
 
-  float* obuf = reinterpret_cast<float*>(stage_base);      // [warp][8 heads][kORowStride]
+  float* obuf = reinterpret_cast<float*>(stage_base);      // [warp][8 * NH heads][kORowStride]
   if (warp < kConsumerWarps) {
-    float f[2];
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      const int row = 2 * tig + r;
-      float mg = sm_m[0][row];
+    for (int t = 0; t < NH; ++t) {
+      float f[2];
 #pragma unroll
-      for (int w = 1; w < kConsumerWarps; ++w) mg = fmaxf(mg, sm_m[w][row]);
-      f[r] = m_run[r] == -INFINITY ? 0.f : ptx::ex2_approx(m_run[r] - mg);
-    }
-    float* ob = obuf + warp * 8 * kORowStride;
+      for (int r = 0; r < 2; ++r) {
+        const int row = 8 * t + 2 * tig + r;
+        float mg = sm_m[0][row];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      ob[(2 * tig) * kORowStride + 16 * i + gid] = o_acc[i][0] * f[0];
-      ob[(2 * tig + 1) * kORowStride + 16 * i + gid] = o_acc[i][1] * f[1];
-      ob[(2 * tig) * kORowStride + 16 * i + gid + 8] = o_acc[i][2] * f[0];
-      ob[(2 * tig + 1) * kORowStride + 16 * i + gid + 8] = o_acc[i][3] * f[1];
+        for (int w = 1; w < kConsumerWarps; ++w) mg = fmaxf(mg, sm_m[w][row]);
+        f[r] = m_run[t][r] == -INFINITY ? 0.f : ptx::ex2_approx(m_run[t][r] - mg);
+      }
+      float* ob = obuf + (warp * 8 * NH + 8 * t) * kORowStride;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        ob[(2 * tig) * kORowStride + 16 * i + gid] = o_acc[t][i][0] * f[0];
+        ob[(2 * tig + 1) * kORowStride + 16 * i + gid] = o_acc[t][i][1] * f[1];
+        ob[(2 * tig) * kORowStride + 16 * i + gid + 8] = o_acc[t][i][2] * f[0];
+        ob[(2 * tig + 1) * kORowStride + 16 * i + gid + 8] = o_acc[t][i][3] * f[1];
+      }
     }
   }
   __syncthreads();
@@ -770,7 +532,7 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
       float o = 0.f, ls = 0.f;
 #pragma unroll
       for (int w = 0; w < kConsumerWarps; ++w) {
-        o += obuf[(w * 8 + row) * kORowStride + c];
+        o += obuf[(w * 8 * NH + row) * kORowStride + c];
         const float mw = sm_m[w][row];
         ls += mw == -INFINITY ? 0.f : sm_l[w][row] * ptx::ex2_approx(mw - mg);
       }
@@ -870,19 +632,19 @@ int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* ne
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(attr_once, [&] {
-      attr_err = cudaFuncSetAttribute(decode_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      kStages * kStageBytes + 1024);
+      attr_err = cudaFuncSetAttribute(decode_stream_t_kernel<1, kStages1, kMinCtas1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      kStages1 * kStageBytes + 1024);
       if (attr_err == cudaSuccess)
-        attr_err = cudaFuncSetAttribute(decode_stream_t_kernel<kTStages, kTMinCtas>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kTStages * kStageBytes + 1024);
+        attr_err = cudaFuncSetAttribute(decode_stream_t_kernel<2, kStages2, kMinCtas2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        kStages2 * kStageBytes + 1024);
     });
     if (attr_err != cudaSuccess) return cuda_fail(attr_err);
-    if (p.g <= 8)      // heads on the N axis of the MMA: no padded rows
-      NGC_CUDA_TRY(launch_pdl(decode_stream_t_kernel<kTStages, kTMinCtas>, dim3((unsigned)items), dim3(kStreamThreads),
-                              kTStages * kStageBytes + 1024, stream, maps, p));
+    if (p.g <= 8)
+      NGC_CUDA_TRY(launch_pdl(decode_stream_t_kernel<1, kStages1, kMinCtas1>, dim3((unsigned)items), dim3(kStreamThreads),
+                              kStages1 * kStageBytes + 1024, stream, maps, p));
     else
-      NGC_CUDA_TRY(launch_pdl(decode_stream_kernel, dim3((unsigned)items), dim3(kStreamThreads), kStages * kStageBytes + 1024,
-                              stream, maps, p));
+      NGC_CUDA_TRY(launch_pdl(decode_stream_t_kernel<2, kStages2, kMinCtas2>, dim3((unsigned)items), dim3(kStreamThreads),
+                              kStages2 * kStageBytes + 1024, stream, maps, p));
   } else {
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hq * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
