@@ -90,3 +90,34 @@ def test_binding_refuses_cpu_tensors(ngc):
     t = torch.zeros(4)
     with pytest.raises(ngc.NgcError):
         ngc._ptr(t)
+
+
+def test_added_entry_points_refuse_bad_arguments(ngc):
+    """Gradient, paged and replay entries: null pointers, inconsistent shapes and unsupported layouts are
+    turned away on the host (nothing is launched, so this runs without a GPU)."""
+    lib = ngc.lib
+    bf = ngc.CacheDesc(16, 16, 16, 16, 64, 1, 1, 12, 2, 128, ngc.BF16, 64)      # 16-byte aligned dummy pointers
+    f32 = ngc.CacheDesc(16, 16, 16, 16, 16, 1, 1, 2, 1, 64, ngc.F32, 16)
+    # log-prob gradient
+    assert lib.ngc_evict_logprob_backward(1, 1, None, 1, 1, None, 1, 1, 1, 8, 4, None, None, 0, None, None) == -1   # no output
+    assert lib.ngc_evict_logprob_backward(1, 1, None, 1, 1, None, 0, 1, 1, 8, 4, 1, None, 0, None, None) == -1     # no rounds
+    # score gradient: fp32 / d = 64 caches are not built; the log variant needs the forward logits; workspace is mandatory
+    assert lib.ngc_score_evict_backward(C.byref(f32), 16, 5, 1, 0, 0, None, 16, 16, 16, 16, None, 0, None, None) == -2
+    assert lib.ngc_score_evict_backward(C.byref(bf), 16, 5, 1, 0, 1, None, 16, 64, 16, 16, None, 0, None, None) == -1
+    assert lib.ngc_score_evict_backward(C.byref(bf), 16, 9, 1, 0, 0, None, 16, 64, 16, 16, None, 0, None, None) == -2  # 6 * 9 rows > 40
+    assert lib.ngc_score_evict_backward(C.byref(bf), 16, 5, 1, 0, 0, None, 16, 64, 16, 16, None, 0, None, None) == -3
+    # paged cache: page size 32 or 64, bf16 / d = 128 only
+    pg = ngc.PagedCacheDesc(16, 16, 16, 16, 1, 1, 12, 2, 128, ngc.BF16, 48, 4, 0)
+    assert lib.ngc_decode_attn_paged(C.byref(pg), 16, None, None, 0, 1, 1.0, 16, 0, None, 0, None, None) == -1
+    pg = ngc.PagedCacheDesc(16, 16, 16, 16, 1, 1, 4, 4, 64, ngc.F32, 32, 4, 0)
+    assert lib.ngc_decode_attn_paged(C.byref(pg), 16, None, None, 0, 1, 1.0, 16, 0, None, 0, None, None) == -2
+    assert lib.ngc_score_evict_paged(C.byref(pg), 16, 5, 0, 16, 4, None, 0, None, None) == -2
+    assert lib.ngc_evict_pages(None, 1, 1, 4, None, None) == -1
+    # replay
+    assert lib.ngc_replay_visibility(None, 1, 1, 1, 1, 1, 1, 4, 1, 8, 1, 1, None, None) == -1
+    assert lib.ngc_replay_visibility(1, 1, 1, 1, 0, 1, 1, 4, 1, 8, 1, 1, None, None) == -1                 # no rounds
+    assert lib.ngc_replay_visibility(1, 1, 1, 1, 1, 1, 1, 4, 1, 40000, 1, 1, None, None) == -2             # alive set beyond shared memory
+    assert lib.ngc_replay_attn(C.byref(f32), 16, 8, None, None, None, 0, 0, 0, 1.0, 16, 0, None, None) == -2
+    assert lib.ngc_replay_attn(C.byref(bf), 16, 8, None, None, None, 2, 4, 0, 1.0, 16, 0, None, None) == -1   # rounds without lists
+    assert lib.ngc_replay_attn(C.byref(bf), None, 8, None, None, None, 0, 0, 0, 1.0, 16, 0, None, None) == -1
+    assert ngc.lib.ngc_workspace_bytes(ngc.OP_SCORE_BACKWARD, C.byref(bf), 1, 0, 0) > 0
