@@ -266,14 +266,15 @@ __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" 
 
 template <int NT>
 __global__ void __launch_bounds__(kThreads, 2)
-score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
+score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_gk, BwdParams p) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ uint64_t bar_full[kStagesB], bar_empty[kStagesB];
   __shared__ float sm_negM[kMaxRows], sm_inv[kMaxRows], sm_c[kMaxRows];
 
   uint8_t* stage_base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  uint8_t* q_s = stage_base + kStagesB * kStageBytes;          // [48][kQRowBytes] bf16 query rows, zero padded
+  uint8_t* q_s = stage_base + kStagesB * kStageBytes + kStageBytes;   // [48][kQRowBytes] bf16 query rows, zero padded
   uint8_t* dz_s = q_s + kQBytes;                               // [2][64][kDzRowBytes] bf16 dz of a tile
+  uint8_t* dk_s = stage_base + kStagesB * kStageBytes;         // [64][128] bf16 dK of a tile, swizzled like a K tile
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gid = lane >> 2, tig = lane & 3;
   const Item it = decode_item(p);
@@ -400,6 +401,11 @@ score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
       asm volatile("st.shared.b32 [%0], %1;" ::"r"(dz_buf + off + 8 * kDzRowBytes), "r"(hi[t8]) : "memory");
     }
     // ---- dK = dZ Q (16 tokens x 128 channels, 64 at a time): A operand straight from the packed dz ----
+    // A tile that lies wholly inside the sequence leaves through shared memory and one TMA store per
+    // 64-channel box; the sequence's last, partial tile is written row by row (rows beyond T_b stay untouched).
+    const bool full_tile = (it.tile_lo + i) * kTileT + kTileT <= T_b;
+    if (tid == 0) ptx::bulk_wait_read<0>();          // the previous tile's store has read the dK buffer
+    consumer_bar();
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       float dk[8][4];
@@ -418,14 +424,30 @@ score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
           }
         }
       }
+      if (full_tile) {
+        const int ra = 16 * warp + gid, rb = ra + 8;
 #pragma unroll
-      for (int n = 0; n < 8; ++n) {
-        const int ch = 64 * half + 8 * n + 2 * tig;
-        if (t0 < T_b) *reinterpret_cast<uint32_t*>(gk_strip + (int64_t)t0 * 128 + ch) = ptx::pack_bf16x2(dk[n][0], dk[n][1]);
-        if (t1 < T_b) *reinterpret_cast<uint32_t*>(gk_strip + (int64_t)t1 * 128 + ch) = ptx::pack_bf16x2(dk[n][2], dk[n][3]);
+        for (int n = 0; n < 8; ++n) {
+          *reinterpret_cast<uint32_t*>(dk_s + half * kBoxBytes + ra * 128 + ((n ^ (ra & 7)) << 4) + 4 * tig) = ptx::pack_bf16x2(dk[n][0], dk[n][1]);
+          *reinterpret_cast<uint32_t*>(dk_s + half * kBoxBytes + rb * 128 + ((n ^ (rb & 7)) << 4) + 4 * tig) = ptx::pack_bf16x2(dk[n][2], dk[n][3]);
+        }
+      } else {
+#pragma unroll
+        for (int n = 0; n < 8; ++n) {
+          const int ch = 64 * half + 8 * n + 2 * tig;
+          if (t0 < T_b) *reinterpret_cast<uint32_t*>(gk_strip + (int64_t)t0 * 128 + ch) = ptx::pack_bf16x2(dk[n][0], dk[n][1]);
+          if (t1 < T_b) *reinterpret_cast<uint32_t*>(gk_strip + (int64_t)t1 * 128 + ch) = ptx::pack_bf16x2(dk[n][2], dk[n][3]);
+        }
       }
     }
-    consumer_bar();              // the tile's dz is complete and dead K rows are zero
+    ptx::fence_proxy_async();    // the dK tile was written through the generic proxy, the TMA store reads it
+    consumer_bar();              // the tile's dz and dK are complete and dead K rows are zero
+    if (tid == 0 && full_tile) {
+      const int y = (int)p.seq_off[it.b] + (it.tile_lo + i) * kTileT;
+      ptx::tma_store_3d(&map_gk, 0, y, it.l * p.Hkv + it.h, dk_s);
+      ptx::tma_store_3d(&map_gk, 64, y, it.l * p.Hkv + it.h, dk_s + kBoxBytes);
+      ptx::bulk_commit();
+    }
     // ---- dQ[:, 32*warp .. +32] += dZ^T K over the 64 tokens of the tile ----
 #pragma unroll
     for (int kt = 0; kt < 4; ++kt) {
@@ -452,6 +474,7 @@ score_bwd_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p) {
     __syncwarp();
     if (lane == 0) ptx::mbar_arrive(&bar_empty[s]);
   }
+  if (tid == 0) ptx::bulk_wait<0>();       // the last dK tile has left shared memory and reached global memory
   // ---- this range's dQ partial: rows x 128 channels, fp32 ----
   float* part = p.dq_part + ((int64_t)it.strip * p.n_split + it.split) * kMaxRows * 128;
 #pragma unroll
@@ -489,9 +512,9 @@ int bwd_n_split(const ngc_cache* c) {
 }
 
 template <int NT>
-int launch_bwd(const CUtensorMap& map_k, const BwdParams& p, unsigned grid, cudaStream_t stream) {
+int launch_bwd(const CUtensorMap& map_k, const CUtensorMap& map_gk, const BwdParams& p, unsigned grid, cudaStream_t stream) {
   const int smem_a = kStagesA * kStageBytes + 1024;
-  const int smem_b = kStagesB * kStageBytes + 1024 + kQBytes + 2 * kDzBytes;
+  const int smem_b = kStagesB * kStageBytes + 1024 + kStageBytes + kQBytes + 2 * kDzBytes;
   static std::once_flag attr_once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(attr_once, [&] {
@@ -501,7 +524,7 @@ int launch_bwd(const CUtensorMap& map_k, const BwdParams& p, unsigned grid, cuda
   });
   if (attr_err != cudaSuccess) return cuda_fail(attr_err);
   score_bwd_stats_kernel<NT><<<grid, kThreads, smem_a, stream>>>(map_k, p);
-  score_bwd_kernel<NT><<<grid, kThreads, smem_b, stream>>>(map_k, p);
+  score_bwd_kernel<NT><<<grid, kThreads, smem_b, stream>>>(map_k, map_gk, p);
   return launch_status();
 }
 
@@ -549,16 +572,17 @@ extern "C" int ngc_score_evict_backward(const ngc_cache* c, const void* q_recent
   p.inv_sqrt_d = 1.0f / sqrtf((float)c->d);
   p.scale_log2 = p.inv_sqrt_d * 1.4426950408889634f;
   if (items > 0x7fffffffULL) return NGC_ERR_UNSUPPORTED;
-  CUtensorMap map_k;
-  if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, kTileT)) return NGC_ERR_UNSUPPORTED;
+  CUtensorMap map_k, map_gk;
+  if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, kTileT) || !make_kv_map(&map_gk, grad_k, c->rows, c->L * c->Hkv, kTileT))
+    return NGC_ERR_UNSUPPORTED;
   const unsigned grid = (unsigned)items;
   int rc;
   switch ((p.n_rows + 7) / 8) {
-    case 1: rc = launch_bwd<1>(map_k, p, grid, stream); break;
-    case 2: rc = launch_bwd<2>(map_k, p, grid, stream); break;
-    case 3: rc = launch_bwd<3>(map_k, p, grid, stream); break;
-    case 4: rc = launch_bwd<4>(map_k, p, grid, stream); break;
-    default: rc = launch_bwd<5>(map_k, p, grid, stream); break;
+    case 1: rc = launch_bwd<1>(map_k, map_gk, p, grid, stream); break;
+    case 2: rc = launch_bwd<2>(map_k, map_gk, p, grid, stream); break;
+    case 3: rc = launch_bwd<3>(map_k, map_gk, p, grid, stream); break;
+    case 4: rc = launch_bwd<4>(map_k, map_gk, p, grid, stream); break;
+    default: rc = launch_bwd<5>(map_k, map_gk, p, grid, stream); break;
   }
   if (rc != NGC_OK) return rc;
   score_bwd_reduce_kernel<<<(unsigned)(c->L * c->B * c->Hkv * p.n_rows), 128, 0, stream>>>(p);
