@@ -341,3 +341,70 @@ def test_config6_paper_setting_block_eviction_scored_from_k():
             sl = slice(i * peak, i * peak + K * block)
             assert np.array_equal(after.k[:, :, sl], kc[:, :, sl]) and np.array_equal(after.v[:, :, sl], vc[:, :, sl])
     assert np.array_equal(ro.cache.lens.cpu().numpy(), np.full(B, K * block, np.int32))     # steady state: delta / epsilon / 2
+
+
+def test_score_backward_config2_shape_sampled_sequences():
+    """Gradient of the scores at the benchmark's cache shape (B = 64, T = 4096, 12/2 heads, shared list; 4 of the 28
+    layers to keep the oracle to seconds): two sampled sequences against the oracle, 2e-2 of the largest entry."""
+    need_gpu_gb(6)
+    b = ngc()
+    cfg = synth.CONFIGS[2]
+    L, Hq, Hkv, d, B, T, w = 4, cfg["Hq"], cfg["Hkv"], cfg["d"], cfg["B"], cfg["T"], 5
+    dev, dtype = "cuda", torch.bfloat16
+    c = synth.make_cache(L, B, Hq, Hkv, d, dtype, [T] * B, capacity=T, seed=8, outlier_channels=4, device=dev)
+    dc = b.NgcCache(c.k, c.v, c.seq_off, c.lens, Hq, T)
+    qr = synth.normal((L, B, Hq, w, d), 9, dtype, device=dev)
+    up = synth.make_logits(B, 1, T, seed=10, device=dev)
+    gq = torch.empty(qr.shape, dtype=torch.float32, device=dev)
+    gk = torch.zeros_like(c.k)
+    ws = b.alloc_workspace(b.workspace_bytes(b.OP_SCORE_BACKWARD, dc))
+    st = b.new_status()
+    b.ngc_score_evict_backward(dc, qr, 1, b.LISTS_SHARED, up, gq, gk, ws=ws, status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    for bb in (0, 63):
+        k1 = synth.to_numpy(c.k[:, :, bb * T:(bb + 1) * T])
+        ref_q, ref_k = oracle.score_evict_grad(k1, np.array([0, T], np.int64), np.array([T], np.int32), synth.to_numpy(qr[:, bb:bb + 1]), 1, 0,
+                                               up[bb:bb + 1].cpu().numpy().astype(np.float64))
+        got_q = gq[:, bb:bb + 1].cpu().numpy().astype(np.float64)
+        got_k = synth.as_f64(synth.to_numpy(gk[:, :, bb * T:(bb + 1) * T]))
+        assert np.max(np.abs(got_q - ref_q)) <= 2e-2 * np.abs(ref_q).max() + 1e-6
+        assert np.max(np.abs(got_k - ref_k)) <= 2e-2 * np.abs(ref_k).max() + 1e-6
+
+
+def test_replay_attn_rollout_loop_history_sampled_sequence():
+    """Replay attention over the rollout-loop history (T = 8448, 16 rounds, 768 -> 256 per round, per-layer lists),
+    one layer, B = 8: sequence 5 against the dense-mask oracle at all of its 8448 positions."""
+    need_gpu_gb(4)
+    b = ngc()
+    from oracle import replay
+    cfg = synth.CONFIGS[5]
+    L, Hq, Hkv, d, B = 1, cfg["Hq"], cfg["Hkv"], cfg["d"], 8
+    K, delta, prompt = cfg["budget"], cfg["cadence"], cfg["T"]
+    R, alive = cfg["steps"] // delta, prompt + delta
+    T = prompt + R * delta
+    dev, dtype = "cuda", torch.bfloat16
+    rng = np.random.default_rng(4)
+    ks = np.sort(np.argsort(rng.random((R, B, L, alive)), -1)[..., :K], -1).astype(np.int32)
+    budget = np.full((R, B), K, np.int32)
+    alive_before = np.full((R, B), alive, np.int32)
+    total_before = (alive + delta * np.arange(R))[:, None].repeat(B, 1).astype(np.int32)
+    t = lambda a: torch.as_tensor(a).to(dev)
+    pos = torch.empty((R, B, L, K), dtype=torch.int32, device=dev)
+    cnt = torch.empty((R, B, L), dtype=torch.int32, device=dev)
+    st = b.new_status()
+    b.ngc_replay_visibility(t(ks), t(budget), t(alive_before), t(total_before), 1, alive, pos, cnt, status=st)
+    c = synth.make_cache(L, B, Hq, Hkv, d, dtype, [T] * B, capacity=T, seed=6, device=dev)
+    dc = b.NgcCache(c.k, c.v, c.seq_off, c.lens, Hq, T)
+    q = synth.normal((L, B, Hq, T, d), 7, dtype, device=dev)
+    out = torch.empty((L, B, Hq, T, d), dtype=torch.float32, device=dev)
+    b.ngc_replay_attn(dc, q, out, pos, cnt, t(total_before), lists=b.LISTS_PER_LAYER, status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    bb = 5
+    ref_pos, ref_cnt, rc = replay.alive_positions(ks[:, bb:bb + 1], budget[:, bb:bb + 1], alive_before[:, bb:bb + 1], total_before[:, bb:bb + 1])
+    assert rc == 0 and np.array_equal(pos[:, bb:bb + 1].cpu().numpy(), ref_pos)
+    M = replay.dense_mask(T, [int(x) for x in total_before[:, bb]], [ref_pos[r, 0, 0, : ref_cnt[r, 0, 0]] for r in range(R)])
+    ref = replay.replay_attention(synth.as_f64(synth.to_numpy(q[0, bb])), synth.as_f64(synth.to_numpy(c.k[0, :, bb * T:(bb + 1) * T])),
+                                  synth.as_f64(synth.to_numpy(c.v[0, :, bb * T:(bb + 1) * T])), M[None])
+    assert max_rel_err_per_vector(out[0, bb].cpu().numpy().astype(np.float64), ref) <= 2e-2
