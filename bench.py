@@ -14,6 +14,10 @@ HBM; `e2e` is the same step driven from pinned host buffers through the public
 host entry (copies inside the timed region); `roofline` is the decode kernel's
 achieved HBM bandwidth; `cpu_baseline` is the CPU oracle timed on a bounded
 sample of the same workload.
+
+Measurement aids on one GPU (not the benchmark line):
+    python bench.py --config 1|3|4|5|6|7 [--paged] [--graph]   per-phase timing of the other workloads
+    python bench.py --kernel score_backward|replay_attn        one training-side call
 """
 from __future__ import annotations
 
