@@ -35,7 +35,12 @@
  *   k, v    : [L][Hkv][R][d] elements; R rows per (layer, KV head) plane.
  *   seq_off : int64 [B+1]; sequence b owns rows seq_off[b] .. seq_off[b+1] of
  *             every plane (its capacity); seq_off[0] = 0, seq_off[B] = R.
- *   lens    : int32 [B]; the first lens[b] rows of a strip are alive.
+ *   lens    : int32 [B]; the first lens[b] rows of a strip are alive.  With
+ *             lens_lists != 0 the cache holds one length per (sequence, list) instead:
+ *             int32 [B][G] for that ngc_lists mode, and the strips of list gi of
+ *             sequence b have lens[b*G + gi] alive rows.  The paper evicts per layer
+ *             in units of several tokens, and a short last unit that one layer keeps
+ *             and another evicts leaves the layers with different lengths.
  * A (layer, head, sequence) strip is therefore T x d contiguous rows, which
  * decode streams linearly and compaction moves row by row.  Rows at or beyond
  * lens[b] hold unspecified bytes.
@@ -78,7 +83,7 @@ typedef enum { NGC_OP_SCORE = 0, NGC_OP_SAMPLE = 1, NGC_OP_LOGPROB = 2, NGC_OP_C
                NGC_OP_SCORE_BACKWARD = 5 } ngc_op;
 
 /* Describes the cache; owns nothing.  `rows` and `max_len` are host copies the
- * launch geometry needs: rows = seq_off[B]; max_len >= every lens[b] at the
+ * launch geometry needs: rows = seq_off[B]; max_len >= every length at the
  * time of the call (a loose bound such as the largest capacity is fine; it
  * only sizes grids and workspaces). */
 typedef struct {
@@ -90,6 +95,8 @@ typedef struct {
   int32_t L, B, Hq, Hkv, d;   /* Hq % Hkv == 0; d in {64, 128} */
   int32_t dtype;              /* ngc_dtype of k, v, queries and new rows */
   int32_t max_len;
+  int32_t lens_lists;         /* 0: lens[B]; NGC_LISTS_PER_LAYER / _KVHEAD: lens[B][G] of that mode.  Calls that
+                                 take an eviction `lists` mode need lens_lists == 0 or == lists. */
 } ngc_cache;
 
 /* Library version (major*10000 + minor*100 + patch). */

@@ -38,7 +38,7 @@ class CacheDesc(C.Structure):
     """Mirror of ``ngc_cache``."""
     _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("seq_off", C.c_void_p), ("lens", C.c_void_p),
                 ("rows", C.c_int64), ("L", C.c_int32), ("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
-                ("d", C.c_int32), ("dtype", C.c_int32), ("max_len", C.c_int32)]
+                ("d", C.c_int32), ("dtype", C.c_int32), ("max_len", C.c_int32), ("lens_lists", C.c_int32)]
 
 
 class PagedCacheDesc(C.Structure):
@@ -135,14 +135,18 @@ class NgcCache:
     k: torch.Tensor        # [L][Hkv][R][d]
     v: torch.Tensor
     seq_off: torch.Tensor  # int64 [B+1], device
-    lens: torch.Tensor     # int32 [B], device
+    lens: torch.Tensor     # int32 [B] (or [B][G] with lens_lists != 0), device
     Hq: int
     max_len: int           # host bound on lens (any value >= max(lens) at call time)
+    lens_lists: int = 0    # 0: one length per sequence; LISTS_PER_LAYER / _KVHEAD: one per (sequence, list)
 
     def desc(self, extra_len: int = 0) -> CacheDesc:
         L, Hkv, R, d = self.k.shape
+        if self.lens_lists:
+            assert tuple(self.lens.shape) == (self.seq_off.shape[0] - 1, lists_G(self.lens_lists, L, Hkv))
         return CacheDesc(_ptr(self.k), _ptr(self.v), _ptr(self.seq_off), _ptr(self.lens), R, L,
-                         self.lens.shape[0], self.Hq, Hkv, d, _dtype_code(self.k), self.max_len + extra_len)
+                         self.seq_off.shape[0] - 1, self.Hq, Hkv, d, _dtype_code(self.k), self.max_len + extra_len,
+                         self.lens_lists)
 
     @property
     def L(self):
@@ -150,7 +154,7 @@ class NgcCache:
 
     @property
     def B(self):
-        return self.lens.shape[0]
+        return self.seq_off.shape[0] - 1
 
     @property
     def Hkv(self):
@@ -305,7 +309,7 @@ class NgcPagedCache:
         L, Hkv, n_pages, page, d = self.k.shape
         B, _, pages_cap = self.page_table.shape
         flat = self.k.view(L, Hkv, n_pages * page, d)
-        return NgcCache(flat, flat, torch.zeros(1, dtype=torch.int64, device=self.k.device), self.lens, self.Hq, pages_cap * page)
+        return NgcCache(flat, flat, torch.zeros(B + 1, dtype=torch.int64, device=self.k.device), self.lens, self.Hq, pages_cap * page)
 
 
 def ngc_evict_pages(cache: NgcPagedCache, kept_sorted: torch.Tensor, budget: torch.Tensor, status: Optional[torch.Tensor] = None):

@@ -33,6 +33,7 @@ struct CompactParams {
   int64_t plane_vecs;   // R * row_vecs
   int L, B, Hkv, G, lists, block, k_max;
   int row_vecs;         // 16-byte vectors per row
+  int lens_lists;       // 0: lens[B]; else == lists: lens[B][G]
 };
 
 // Validates one kept list with the whole CTA.  Returns (to every thread) the
@@ -90,7 +91,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
   const int h = s % p.Hkv;
   const int l = s / p.Hkv;
   const int gi = list_of(p.lists, l, h, p.Hkv);
-  const int len = p.lens[b];
+  const int len = p.lens[len_index(p.lens_lists, p.L, p.Hkv, b, l, h)];
   const int K = p.budget[b];
   const int32_t* kept = p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max;
 
@@ -171,25 +172,28 @@ __device__ int validate_list_warp(const int32_t* kept, int K, int k_max, int len
   return tokens;
 }
 
-// After all strips moved: lens[b] <- kept token count (one CTA per sequence, a warp per list;
-// every list of the sequence is re-validated and they must agree).
+// After all strips moved: the lengths become the kept token counts (one CTA per sequence, a warp per
+// list; every list is re-validated).  With one length per sequence the lists must agree; with a
+// length per list each list gets its own count.
 __global__ void compact_lens_kernel(CompactParams p) {
   __shared__ int s_bad, s_min, s_max;
   const int b = blockIdx.x;
-  const int len = p.lens[b];
   const int K = p.budget[b];
+  const bool per_list = p.lens_lists != 0;          // then lens_lists == lists: every list has its own length
   if (threadIdx.x == 0) { s_bad = 0; s_min = 0x7fffffff; s_max = -1; }
   __syncthreads();
   const int warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   for (int gi = warp; gi < p.G; gi += n_warps) {
-    const int t = validate_list_warp(p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max, K, p.k_max, len, p.block);
+    int32_t* len_p = const_cast<int32_t*>(p.lens) + (per_list ? (int64_t)b * p.G + gi : b);
+    const int t = validate_list_warp(p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max, K, p.k_max, *len_p, p.block);
     if ((threadIdx.x & 31) == 0) {
       if (t < 0) atomicOr(&s_bad, 1);            // already reported by the strip kernel
+      else if (per_list) *len_p = t;             // lists may keep different token counts (a short last unit)
       else { atomicMin(&s_min, t); atomicMax(&s_max, t); }
     }
   }
   __syncthreads();
-  if (threadIdx.x == 0 && !s_bad) {
+  if (threadIdx.x == 0 && !per_list && !s_bad) {
     if (s_min != s_max) set_dev_status(p.dev_status, NGC_DEV_LISTS_DISAGREE);
     else const_cast<int32_t*>(p.lens)[b] = s_min;
   }
@@ -268,6 +272,7 @@ extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const in
   using namespace ngc;
   if (!valid_cache(c) || !kept_sorted || !budget || k_max <= 0 || block <= 0 || lists < 0 || lists > 2)
     return NGC_ERR_INVALID_ARG;
+  if (c->lens_lists != 0 && c->lens_lists != lists) return NGC_ERR_INVALID_ARG;   // a length per eviction list, or one per sequence
   const int row_bytes = c->d * elt_bytes(c->dtype);
   CompactParams p;
   p.k = (uint4*)c->k;
@@ -281,7 +286,7 @@ extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const in
   p.plane_vecs = c->rows * p.row_vecs;
   p.L = c->L; p.B = c->B; p.Hkv = c->Hkv;
   p.G = lists_G(lists, c->L, c->Hkv);
-  p.lists = lists; p.block = block; p.k_max = k_max;
+  p.lists = lists; p.block = block; p.k_max = k_max; p.lens_lists = c->lens_lists;
   const int64_t strips = (int64_t)c->L * c->Hkv * c->B * 2;
   if (strips > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
   if ((((uintptr_t)c->k | (uintptr_t)c->v) & 15) != 0) return NGC_ERR_INVALID_ARG;      // rows move as 16-byte vectors

@@ -58,14 +58,16 @@ struct DecodeParams {
   // paged layout (page_table != null): rows of a plane = B * pages_cap * page, seq_off unused
   const int32_t* page_table;   // [B][G][pages_cap]
   int page, pages_cap, lists, G;
+  int lens_lists;              // 0: lens[B]; else lens[B][G'] of that lists mode
 };
 
 // Visible length of sequence b for this call; -1 if the appended row does not fit.
 __device__ __forceinline__ int64_t seq_capacity(const DecodeParams& p, int b) {
   return p.page_table ? (int64_t)p.pages_cap * p.page : p.seq_off[b + 1] - p.seq_off[b];
 }
-__device__ __forceinline__ int visible_len(const DecodeParams& p, int b) {
-  const int len = p.lens[b];
+// Visible length of strip (b, l, h) in this call; -1 if the appended row does not fit.
+__device__ __forceinline__ int visible_len(const DecodeParams& p, int b, int l, int h) {
+  const int len = p.lens[len_index(p.lens_lists, p.L, p.Hkv, b, l, h)];
   if (!p.append) return len;
   return (len + 1 > seq_capacity(p, b)) ? -1 : len + 1;
 }
@@ -75,10 +77,11 @@ __device__ __forceinline__ int visible_len(const DecodeParams& p, int b) {
 __global__ void bump_lens_kernel(DecodeParams p) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();          // every CTA of the attention (and combine) kernel has read lens
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= p.B) return;
-  const int len = p.lens[b];
-  if (len + 1 <= seq_capacity(p, b)) p.lens[b] = len + 1;
+  const int per_seq = lists_G(p.lens_lists, p.L, p.Hkv);      // length entries per sequence
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= p.B * per_seq) return;
+  const int len = p.lens[idx];
+  if (len + 1 <= seq_capacity(p, idx / per_seq)) p.lens[idx] = len + 1;
 }
 
 // ---------------------------------------------------------------- output helpers
@@ -136,7 +139,7 @@ __global__ void __launch_bounds__(kGenWarps * 32) decode_generic_kernel(DecodePa
 
   ptx::grid_dep_wait();
   ptx::grid_dep_launch();
-  int len = visible_len(p, b);
+  int len = visible_len(p, b, l, h);
   if (len < 0) {
     if (tid == 0) set_dev_status(p.dev_status, NGC_DEV_STRIP_FULL);
     len = 0;
@@ -314,7 +317,7 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
   ptx::grid_dep_wait();           // lens and the cache rows of earlier calls are final from here on
   ptx::grid_dep_launch();
 
-  int len = visible_len(p, b);
+  int len = visible_len(p, b, l, h);
   if (len < 0) {
     if (tid == 0) set_dev_status(p.dev_status, NGC_DEV_STRIP_FULL);
     len = 0;
@@ -609,6 +612,7 @@ int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* ne
   p.n_split = decode_n_split(c, p.n_layers);
   p.part_o = nullptr; p.part_ml = nullptr;
   p.page_table = pv.table; p.page = pv.page; p.pages_cap = pv.pages_cap; p.lists = pv.lists;
+  p.lens_lists = c->lens_lists;
   p.G = lists_G(pv.lists, c->L, c->Hkv);
   if (p.n_split > 1) {
     const size_t items = (size_t)p.n_layers * c->B * c->Hq * p.n_split;
@@ -658,7 +662,7 @@ int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* ne
   if (p.n_split > 1)
     NGC_CUDA_TRY(launch_pdl(combine_kernel, dim3((unsigned)(p.n_layers * c->B * c->Hq)), dim3(c->d), 0, stream, p));
   if (p.append && layer_end == c->L)
-    NGC_CUDA_TRY(launch_pdl(bump_lens_kernel, dim3((c->B + 255) / 256), dim3(256), 0, stream, p));
+    NGC_CUDA_TRY(launch_pdl(bump_lens_kernel, dim3((c->B * lists_G(c->lens_lists, c->L, c->Hkv) + 255) / 256), dim3(256), 0, stream, p));
   return NGC_OK;
 }
 
@@ -691,6 +695,7 @@ extern "C" int ngc_decode_attn_paged(ngc_paged_cache* pc, const void* q, const v
   c.rows = (int64_t)pc->B * pc->pages_cap * pc->page;
   c.L = pc->L; c.B = pc->B; c.Hq = pc->Hq; c.Hkv = pc->Hkv; c.d = pc->d; c.dtype = pc->dtype;
   c.max_len = pc->pages_cap * pc->page;
+  c.lens_lists = 0;
   const PagedView pv = {pc->page_table, pc->page, pc->pages_cap, pc->lists};
   return decode_impl(&c, pv, q, new_k, new_v, layer_begin, layer_end, scale, out, out_dtype, ws, ws_bytes, dev_status,
                      (cudaStream_t)stream);

@@ -40,7 +40,12 @@ inline int elt_bytes(int dtype) { return dtype == NGC_F32 ? 4 : 2; }
 inline bool valid_cache(const ngc_cache* c) {
   return c && c->k && c->v && c->seq_off && c->lens && c->L > 0 && c->B > 0 && c->Hq > 0 && c->Hkv > 0 &&
          c->Hq % c->Hkv == 0 && (c->d == 64 || c->d == 128) && c->rows >= 0 && c->max_len >= 0 &&
-         (c->dtype == NGC_F32 || c->dtype == NGC_BF16);
+         (c->dtype == NGC_F32 || c->dtype == NGC_BF16) && c->lens_lists >= 0 && c->lens_lists <= 2;
+}
+
+// Index of the length entry of strip (b, l, h): lens[B] when lens_lists == 0, else lens[B][G] of that mode.
+__host__ __device__ inline int64_t len_index(int lens_lists, int L, int Hkv, int b, int l, int h) {
+  return (int64_t)b * lists_G(lens_lists, L, Hkv) + list_of(lens_lists, l, h, Hkv);
 }
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }

@@ -301,6 +301,7 @@ extern "C" int ngc_replay_attn(const ngc_cache* c, const void* q, int t_max,
     return NGC_ERR_INVALID_ARG;
   if (out_dtype != NGC_F32 && out_dtype != NGC_BF16) return NGC_ERR_INVALID_ARG;
   if (c->dtype != NGC_BF16 || c->d != 128) return NGC_ERR_UNSUPPORTED;
+  if (c->lens_lists != 0) return NGC_ERR_INVALID_ARG;      // the full sequences have one length each
   if ((((uintptr_t)c->k | (uintptr_t)c->v | (uintptr_t)q | (uintptr_t)out) & 15) != 0) return NGC_ERR_INVALID_ARG;
   if (c->rows == 0) return NGC_OK;
   ReplayAttnParams p;

@@ -56,7 +56,7 @@ struct BwdParams {
   void* grad_k;                // [L][Hkv][R][128] bf16
   int32_t* dev_status;
   int64_t rows_R;
-  int L, B, Hq, Hkv, g, w, n_rows, block, lists, G, n_max, log_transform, n_split;
+  int L, B, Hq, Hkv, g, w, n_rows, block, lists, G, n_max, log_transform, n_split, lens_lists;
   float scale_log2, inv_sqrt_d;
 };
 
@@ -98,7 +98,7 @@ __device__ __forceinline__ Item decode_item(const BwdParams& p) {
   it.h = it.strip % p.Hkv;
   it.b = (it.strip / p.Hkv) % p.B;
   it.l = it.strip / (p.Hkv * p.B);
-  it.T_b = p.lens[it.b];
+  it.T_b = p.lens[len_index(p.lens_lists, p.L, p.Hkv, it.b, it.l, it.h)];
   const int nt = (it.T_b + kTileT - 1) / kTileT;
   const int tps = (nt + p.n_split - 1) / p.n_split;
   it.tile_lo = min(nt, it.split * tps);
@@ -549,6 +549,7 @@ extern "C" int ngc_score_evict_backward(const ngc_cache* c, const void* q_recent
   const int g = c->Hq / c->Hkv;
   if (c->dtype != NGC_BF16 || c->d != 128 || g * w > kMaxRows || c->rows >= 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
   if ((((uintptr_t)c->k | (uintptr_t)q_recent | (uintptr_t)grad_k) & 15) != 0) return NGC_ERR_INVALID_ARG;
+  if (c->lens_lists != 0 && c->lens_lists != lists) return NGC_ERR_INVALID_ARG;
   if ((int64_t)n_max * block < c->max_len) return NGC_ERR_INVALID_ARG;
   const size_t q_elems = (size_t)c->L * c->B * c->Hq * w * 128;
   if (c->rows == 0 || c->max_len == 0) {
@@ -569,6 +570,7 @@ extern "C" int ngc_score_evict_backward(const ngc_cache* c, const void* q_recent
   p.rows_R = c->rows;
   p.L = c->L; p.B = c->B; p.Hq = c->Hq; p.Hkv = c->Hkv; p.g = g; p.w = w; p.n_rows = g * w;
   p.block = block; p.lists = lists; p.G = lists_G(lists, c->L, c->Hkv); p.n_max = n_max; p.log_transform = log_transform;
+  p.lens_lists = c->lens_lists;
   p.inv_sqrt_d = 1.0f / sqrtf((float)c->d);
   p.scale_log2 = p.inv_sqrt_d * 1.4426950408889634f;
   if (items > 0x7fffffffULL) return NGC_ERR_UNSUPPORTED;

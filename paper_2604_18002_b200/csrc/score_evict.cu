@@ -51,6 +51,7 @@ struct ScoreParams {
   // psi is indexed by logical token: sequence b starts at b * pages_cap * page
   const int32_t* page_table;   // [B][G_tab][pages_cap]
   int page, pages_cap, tab_lists, tab_G;
+  int lens_lists;              // 0: lens[B]; else == lists: lens[B][G]
 };
 
 __device__ __forceinline__ int64_t psi_row0(const ScoreParams& p, int b) {
@@ -86,7 +87,7 @@ __global__ void __launch_bounds__(kChunk) score_kernel(ScoreParams p) {
   const int h = strip % p.Hkv;
   const int b = (strip / p.Hkv) % p.B;
   const int l = strip / (p.Hkv * p.B);
-  const int T_b = p.lens[b];
+  const int T_b = p.lens[len_index(p.lens_lists, p.L, p.Hkv, b, l, h)];
   if (chunk * kChunk >= T_b) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t = chunk * kChunk + tid;
@@ -231,7 +232,7 @@ score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, fl
   const int h = strip % p.Hkv;
   const int b = (strip / p.Hkv) % p.B;
   const int l = strip / (p.Hkv * p.B);
-  const int T_b = p.lens[b];
+  const int T_b = p.lens[len_index(p.lens_lists, p.L, p.Hkv, b, l, h)];
   const int n_rows = p.n_rows;
   const int w_eff = min(p.w, T_b);
 
@@ -440,7 +441,7 @@ score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, fl
 __global__ void __launch_bounds__(256) score_finish_kernel(ScoreParams p) {
   const int li = blockIdx.x;                    // b * G + gi
   const int b = li / p.G, gi = li - b * p.G;
-  const int T_b = p.lens[b];
+  const int T_b = p.lens[p.lens_lists ? li : b];      // a length per list means lens_lists == lists
   const int n_units = (T_b + p.block - 1) / p.block;
   const int u = blockIdx.y * blockDim.x + threadIdx.x;
   if (u >= n_units || u >= p.n_max) return;
@@ -525,6 +526,7 @@ int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, in
     return NGC_ERR_INVALID_ARG;
   const int g = c->Hq / c->Hkv;
   if (g * w > 128) return NGC_ERR_UNSUPPORTED;
+  if (c->lens_lists != 0 && c->lens_lists != lists) return NGC_ERR_INVALID_ARG;   // a length per scored list, or one per sequence
   if ((int64_t)n_max * block < c->max_len) return NGC_ERR_INVALID_ARG;
   if (c->rows == 0 || c->max_len == 0) return NGC_OK;
   const size_t need = score_workspace_bytes(c, 0, n_max);
@@ -541,6 +543,7 @@ int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, in
   p.log_transform = log_transform;
   p.inv_sqrt_d = 1.0f / sqrtf((float)c->d);
   p.page_table = pv.table; p.page = pv.page; p.pages_cap = pv.pages_cap; p.tab_lists = pv.lists;
+  p.lens_lists = c->lens_lists;
   p.tab_G = lists_G(pv.lists, c->L, c->Hkv);
 
   p.n_split = 1;
@@ -618,6 +621,7 @@ extern "C" int ngc_score_evict_paged(const ngc_paged_cache* pc, const void* q_re
   c.rows = (int64_t)pc->B * pc->pages_cap * pc->page;
   c.L = pc->L; c.B = pc->B; c.Hq = pc->Hq; c.Hkv = pc->Hkv; c.d = pc->d; c.dtype = pc->dtype;
   c.max_len = pc->pages_cap * pc->page;
+  c.lens_lists = 0;
   const PagedView pv = {pc->page_table, pc->page, pc->pages_cap, pc->lists};
   return score_impl(&c, pv, q_recent, w, pc->page, pc->lists, log_transform, logits, n_max, ws, ws_bytes, dev_status,
                     (cudaStream_t)stream);

@@ -19,9 +19,11 @@ from . import binding as ngc
 
 class NgcRollout:
     def __init__(self, L, B, Hq, Hkv, d, dtype, capacity, n_max, k_max, lists=ngc.LISTS_SHARED, block=1,
-                 w=5, device="cuda", list_base=0, with_score=True, kv=None):
+                 w=5, device="cuda", list_base=0, with_score=True, kv=None, per_list_lens=False):
         """``kv``: optional (k, v) device tensors of shape [L][Hkv][sum(capacity)][d] to adopt
-        instead of allocating fresh ones."""
+        instead of allocating fresh ones.  ``per_list_lens``: keep one cache length per (sequence,
+        eviction list) instead of one per sequence, so that lists may keep different token counts
+        (units of several tokens with a short last unit); needs ``lists`` != shared."""
         self.L, self.B, self.Hq, self.Hkv, self.d = L, B, Hq, Hkv, d
         self.dtype, self.lists, self.block, self.w = dtype, lists, block, w
         self.device = device
@@ -35,8 +37,9 @@ class NgcRollout:
             kv = (torch.empty((L, Hkv, R, d), dtype=dtype, device=device),
                   torch.empty((L, Hkv, R, d), dtype=dtype, device=device))
         assert tuple(kv[0].shape) == (L, Hkv, R, d) and tuple(kv[1].shape) == (L, Hkv, R, d)
-        self.cache = ngc.NgcCache(kv[0], kv[1], seq_off.to(device), torch.zeros(B, dtype=torch.int32, device=device),
-                                  Hq, int(cap.max()))
+        lens_shape = (B, self.G) if per_list_lens else (B,)
+        self.cache = ngc.NgcCache(kv[0], kv[1], seq_off.to(device), torch.zeros(lens_shape, dtype=torch.int32, device=device),
+                                  Hq, int(cap.max()), lists if per_list_lens else 0)
         self.n_max, self.k_max = n_max, k_max
         self.logits = torch.empty((B, self.G, n_max), dtype=torch.float32, device=device)
         self.score_logits = torch.empty_like(self.logits) if with_score else None

@@ -39,9 +39,10 @@ def test_version_and_strerror(ngc):
 
 
 def test_struct_layout_matches_header(ngc):
-    # 4 pointers, int64, 7 int32 (+4 bytes tail padding)
-    assert C.sizeof(ngc.CacheDesc) == 4 * 8 + 8 + 7 * 4 + 4
+    # 4 pointers, int64, 8 int32
+    assert C.sizeof(ngc.CacheDesc) == 4 * 8 + 8 + 8 * 4
     assert ngc.CacheDesc.rows.offset == 32 and ngc.CacheDesc.L.offset == 40 and ngc.CacheDesc.max_len.offset == 64
+    assert ngc.CacheDesc.lens_lists.offset == 68
 
 
 def test_workspace_sizes_on_host(ngc):
@@ -83,6 +84,12 @@ def test_bad_arguments_are_refused_before_launch(ngc):
     assert lib.ngc_score_evict(C.byref(good), 1, 0, 1, 0, 0, 1, 16, None, 0, None, None) == -1
     assert lib.ngc_score_evict(C.byref(good), 1, 5, 1, 0, 0, 1, 8, None, 0, None, None) == -1     # n_max too small
     assert lib.ngc_score_evict(C.byref(good), 1, 5, 1, 0, 0, 1, 16, None, 0, None, None) == -3    # no workspace
+    # a length per layer cannot serve a shared or a per-head eviction list
+    per_layer = ngc.CacheDesc(1, 1, 1, 1, 16, 1, 1, 2, 1, 64, ngc.F32, 16, 1)
+    assert lib.ngc_compact_kv(C.byref(per_layer), 1, 1, 4, 0, 1, None, None) == -1
+    assert lib.ngc_score_evict(C.byref(per_layer), 1, 5, 1, 2, 0, 1, 16, None, 0, None, None) == -1
+    bad_mode = ngc.CacheDesc(1, 1, 1, 1, 16, 1, 1, 2, 1, 64, ngc.F32, 16, 3)
+    assert lib.ngc_compact_kv(C.byref(bad_mode), 1, 1, 4, 0, 1, None, None) == -1
 
 
 def test_binding_refuses_cpu_tensors(ngc):

@@ -68,3 +68,34 @@ def test_score_backward_token_ranges_and_unsupported_shapes():
     qr = synth.normal((1, 1, 4, 2, 64), 2, torch.float32).cuda()
     with pytest.raises(b.NgcError, match="not supported"):
         b.ngc_score_evict_backward(dc, qr, 1, 1, torch.zeros((1, 1, 10), device="cuda"), torch.zeros_like(qr), torch.zeros_like(dc.k))
+
+
+def test_score_backward_with_a_length_per_layer():
+    """Per-layer lists whose layers hold different numbers of tokens: every layer against the oracle run on it alone."""
+    b = ngc()
+    L, B, Hq, Hkv, d, w, block, dtype = 3, 2, 12, 2, 128, 5, 32, torch.bfloat16
+    cap = 400
+    lens = np.array([[300, 268, 290], [65, 97, 33]], np.int32)               # [B][L]
+    c = synth.make_cache(L, B, Hq, Hkv, d, dtype, [cap, cap], capacity=cap, seed=3, outlier_channels=4)
+    qr = synth.normal((L, B, Hq, w, d), 4, dtype)
+    n_max = (cap + block - 1) // block
+    up = synth.make_logits(B, L, n_max, seed=5).numpy().astype(np.float64)
+    dc = b.NgcCache(c.k.cuda(), c.v.cuda(), c.seq_off.cuda(), torch.as_tensor(lens).cuda(), Hq, cap, b.LISTS_PER_LAYER)
+    gq = torch.zeros(qr.shape, dtype=torch.float32, device="cuda")
+    gk = torch.zeros_like(dc.k)
+    ws = b.alloc_workspace(b.workspace_bytes(b.OP_SCORE_BACKWARD, dc))
+    st = b.new_status()
+    b.ngc_score_evict_backward(dc, qr.cuda(), block, b.LISTS_PER_LAYER, torch.as_tensor(up, dtype=torch.float32).cuda(), gq, gk, ws=ws, status=st)
+    torch.cuda.synchronize()
+    assert status_value(st) == 0
+    so = c.seq_off.numpy()
+    for l in range(L):
+        ref_q, ref_k = oracle.score_evict_grad(np.ascontiguousarray(synth.to_numpy(c.k)[l:l + 1]), so, np.ascontiguousarray(lens[:, l]),
+                                               np.ascontiguousarray(synth.to_numpy(qr)[l:l + 1]), block, 0, np.ascontiguousarray(up[:, l:l + 1]))
+        got_q = gq[l:l + 1].cpu().numpy().astype(np.float64)
+        got_k = synth.as_f64(synth.to_numpy(gk[l:l + 1]))
+        for bb in range(B):
+            sl = slice(so[bb], so[bb] + lens[bb, l])
+            assert np.max(np.abs(got_q[:, bb] - ref_q[:, bb])) <= TOL * np.abs(ref_q[:, bb]).max() + FLOOR
+            assert np.max(np.abs(got_k[:, :, sl] - ref_k[:, :, sl])) <= TOL * np.abs(ref_k[:, :, sl]).max() + FLOOR
+            assert np.all(got_k[:, :, so[bb] + lens[bb, l]:so[bb + 1]] == 0.0)
