@@ -228,7 +228,8 @@ int ngc_evict_logprob_backward(const float* logits, const int32_t* n, const int3
  * list), instead of the paper's dense B x T x T masks.
  *   kept_sorted  [R][B][G][k_max] as written by ngc_sample_evict at round r
  *   budget       [R][B] kept units;  alive_before [R][B] tokens alive when round
- *                r fired (lens[b] at that time);  total_before [R][B] sequence
+ *                r fired (lens[b] at that time), or [R][B][G] with per_list != 0 (caches
+ *                with a length per list);  total_before [R][B] sequence
  *                length when round r fired (the tokens appended since the last
  *                round are the positions just below it)
  *   block        tokens per unit;  alive_max (host) >= every alive_before
@@ -239,7 +240,7 @@ int ngc_evict_logprob_backward(const float* logits, const int32_t* n, const int3
  */
 int ngc_replay_visibility(const int32_t* kept_sorted, const int32_t* budget, const int32_t* alive_before,
                           const int32_t* total_before, int R, int B, int G, int k_max, int block, int alive_max,
-                          int32_t* alive_pos, int32_t* alive_count, int32_t* dev_status, ngc_stream stream);
+                          int per_list, int32_t* alive_pos, int32_t* alive_count, int32_t* dev_status, ngc_stream stream);
 
 /*
  * Replay attention -- Section 4.5: one pass over ALL tokens of a rollout in
@@ -307,7 +308,9 @@ int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* new_k, const
  *                of every (layer, KV head) plane the list covers.  Each row of the
  *                table is a permutation of 0 .. pages_cap-1: entries at and beyond
  *                ceil(lens[b] / page) name the sequence's free pages.
- *   lens       : int32 [B] alive tokens (same for every list of b)
+ *   lens       : int32 [B] alive tokens (same for every list of b), or int32 [B][G] with
+ *                lens_per_list != 0 (a partly filled last page that one list keeps and
+ *                another evicts leaves them with different lengths)
  *   lists      : ngc_lists, fixes G and which planes a list covers
  *   page       : tokens per page, 32 or 64
  */
@@ -319,6 +322,7 @@ typedef struct {
   int32_t L, B, Hq, Hkv, d;
   int32_t dtype;
   int32_t page, pages_cap, lists;
+  int32_t lens_per_list;
 } ngc_paged_cache;
 
 /*

@@ -28,7 +28,8 @@ def alive_positions(kept_sorted, budget, alive_before, total_before, block=1):
 
     kept_sorted  [R][B][G][k_max] int32  kept units of round r, ascending, -1 padded
     budget       [R][B]           int32  number of kept units
-    alive_before [R][B]           int32  |A_r|: tokens alive when round r fires
+    alive_before [R][B]           int32  |A_r|: tokens alive when round r fires ([R][B][G] when the lists of a
+                                         sequence hold different numbers of tokens)
     total_before [R][B]           int32  sequence length when round r fires (block_r ends there)
     Returns (pos [R][B][G][k_max*block] int32 ascending, -1 padded; count [R][B][G]; rc) with
     rc = 0, 1 (inconsistent counts) or 3 (bad kept list); a failing list gets count -1 from
@@ -37,7 +38,9 @@ def alive_positions(kept_sorted, budget, alive_before, total_before, block=1):
     kept_sorted = np.asarray(kept_sorted, np.int32)
     R, B, G, k_max = kept_sorted.shape
     budget = np.asarray(budget, np.int32).reshape(R, B)
-    alive_before = np.asarray(alive_before, np.int32).reshape(R, B)
+    alive_before = np.asarray(alive_before, np.int32)
+    alive_before = alive_before.reshape(R, B, G) if alive_before.size == R * B * G and G > 1 else \
+        np.repeat(alive_before.reshape(R, B, 1), G, 2)
     total_before = np.asarray(total_before, np.int32).reshape(R, B)
     pos = np.full((R, B, G, k_max * block), -1, np.int32)
     count = np.full((R, B, G), -1, np.int32)
@@ -46,7 +49,7 @@ def alive_positions(kept_sorted, budget, alive_before, total_before, block=1):
         for g in range(G):
             kept_prev = np.zeros(0, np.int64)          # kept_{r-1}, original positions
             for r in range(R):
-                n_alive, total, K = int(alive_before[r, b]), int(total_before[r, b]), int(budget[r, b])
+                n_alive, total, K = int(alive_before[r, b, g]), int(total_before[r, b]), int(budget[r, b])
                 grow = n_alive - len(kept_prev)        # |block_r|: tokens appended since the last round
                 if grow < 0 or grow > total or K < 0 or K > k_max:
                     rc = max(rc, 1)

@@ -45,7 +45,8 @@ class PagedCacheDesc(C.Structure):
     """Mirror of ``ngc_paged_cache``."""
     _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("page_table", C.c_void_p), ("lens", C.c_void_p),
                 ("L", C.c_int32), ("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("d", C.c_int32),
-                ("dtype", C.c_int32), ("page", C.c_int32), ("pages_cap", C.c_int32), ("lists", C.c_int32)]
+                ("dtype", C.c_int32), ("page", C.c_int32), ("pages_cap", C.c_int32), ("lists", C.c_int32),
+                ("lens_per_list", C.c_int32)]
 
 
 def _load():
@@ -84,7 +85,7 @@ def _load():
     lib.ngc_replay_attn.restype = i32
     lib.ngc_replay_attn.argtypes = [C.POINTER(CacheDesc), vp, i32, vp, vp, vp, i32, i32, i32, C.c_float, vp, i32, vp, vp]
     lib.ngc_replay_visibility.restype = i32
-    lib.ngc_replay_visibility.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.ngc_replay_visibility.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.ngc_evict_pages.restype = i32
     lib.ngc_evict_pages.argtypes = [C.POINTER(PagedCacheDesc), vp, vp, i32, vp, vp]
     lib.ngc_decode_attn_paged.restype = i32
@@ -293,7 +294,7 @@ class NgcPagedCache:
     k: torch.Tensor           # [L][Hkv][B * pages_cap][page][d] bf16
     v: torch.Tensor
     page_table: torch.Tensor  # int32 [B][G][pages_cap], each row a permutation of 0..pages_cap-1
-    lens: torch.Tensor        # int32 [B]
+    lens: torch.Tensor        # int32 [B], or [B][G] (a length per list)
     Hq: int
     lists: int
 
@@ -302,7 +303,7 @@ class NgcPagedCache:
         B, G, pages_cap = self.page_table.shape
         assert n_pages == B * pages_cap and G == lists_G(self.lists, L, Hkv)
         return PagedCacheDesc(_ptr(self.k), _ptr(self.v), _ptr(self.page_table), _ptr(self.lens), L, B, self.Hq, Hkv, d,
-                              _dtype_code(self.k), page, pages_cap, self.lists)
+                              _dtype_code(self.k), page, pages_cap, self.lists, 1 if self.lens.dim() == 2 else 0)
 
     def as_contiguous_desc(self) -> "NgcCache":
         """Shape-only view for workspace sizing (same L, B, Hq, Hkv)."""
@@ -348,7 +349,8 @@ def ngc_replay_visibility(kept_sorted: torch.Tensor, budget: torch.Tensor, alive
     """kept_sorted [R][B][G][k_max] -> alive_pos [R][B][G][k_max*block], alive_count [R][B][G] (int32)."""
     R, B, G, k_max = kept_sorted.shape
     rc = lib.ngc_replay_visibility(_ptr(kept_sorted), _ptr(budget), _ptr(alive_before), _ptr(total_before), R, B, G, k_max, block,
-                                   alive_max, _ptr(alive_pos), _ptr(alive_count), _ptr(status), _stream())
+                                   alive_max, 1 if alive_before.dim() == 3 else 0, _ptr(alive_pos), _ptr(alive_count), _ptr(status),
+                                   _stream())
     _check(rc, "ngc_replay_visibility")
 
 

@@ -213,7 +213,7 @@ struct PageEvictParams {
   const int32_t* kept_sorted;
   const int32_t* budget;
   int32_t* dev_status;
-  int B, G, k_max, page, pages_cap;
+  int B, G, k_max, page, pages_cap, per_list;
 };
 
 __global__ void evict_pages_kernel(PageEvictParams p) {
@@ -221,13 +221,14 @@ __global__ void evict_pages_kernel(PageEvictParams p) {
   __shared__ int s_bad, s_min, s_max;
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-  const int len = p.lens[b];
   const int K = p.budget[b];
   if (threadIdx.x == 0) { s_bad = 0; s_min = 0x7fffffff; s_max = -1; }
   __syncthreads();
   int32_t* old_row = s_rows + warp * p.pages_cap;
-  const int n_units = (len + p.page - 1) / p.page;
   for (int gi = warp; gi < p.G; gi += n_warps) {
+    int32_t* len_p = p.lens + (p.per_list ? (int64_t)b * p.G + gi : b);
+    const int len = *len_p;
+    const int n_units = (len + p.page - 1) / p.page;
     const int32_t* kept = p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max;
     int32_t* row = p.page_table + ((int64_t)b * p.G + gi) * p.pages_cap;
     const int t = n_units <= p.pages_cap ? validate_list_warp(kept, K, p.k_max, len, p.page) : -1;
@@ -235,7 +236,10 @@ __global__ void evict_pages_kernel(PageEvictParams p) {
       if (lane == 0) { atomicOr(&s_bad, 1); set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); }
       continue;
     }
-    if (lane == 0) { atomicMin(&s_min, t); atomicMax(&s_max, t); }
+    if (lane == 0) {
+      if (p.per_list) *len_p = t;                  // every list has its own length
+      else { atomicMin(&s_min, t); atomicMax(&s_max, t); }
+    }
     for (int j = lane; j < p.pages_cap; j += 32) old_row[j] = row[j];
     __syncwarp();
     // kept pages to the front
@@ -258,7 +262,7 @@ __global__ void evict_pages_kernel(PageEvictParams p) {
     __syncwarp();
   }
   __syncthreads();
-  if (threadIdx.x == 0 && !s_bad) {
+  if (threadIdx.x == 0 && !p.per_list && !s_bad) {
     if (s_min != s_max) set_dev_status(p.dev_status, NGC_DEV_LISTS_DISAGREE);
     else p.lens[b] = s_min;
   }
@@ -309,6 +313,7 @@ extern "C" int ngc_evict_pages(ngc_paged_cache* c, const int32_t* kept_sorted, c
   PageEvictParams p;
   p.page_table = c->page_table; p.lens = c->lens; p.kept_sorted = kept_sorted; p.budget = budget; p.dev_status = dev_status;
   p.B = c->B; p.G = lists_G(c->lists, c->L, c->Hkv); p.k_max = k_max; p.page = c->page; p.pages_cap = c->pages_cap;
+  p.per_list = c->lens_per_list != 0;
   const int threads = p.G > 4 ? 256 : 32 * (p.G < 1 ? 1 : p.G);
   const size_t smem = (size_t)(threads / 32) * c->pages_cap * 4;
   if (smem > 96 * 1024) return NGC_ERR_UNSUPPORTED;

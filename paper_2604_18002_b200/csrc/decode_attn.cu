@@ -695,7 +695,7 @@ extern "C" int ngc_decode_attn_paged(ngc_paged_cache* pc, const void* q, const v
   c.rows = (int64_t)pc->B * pc->pages_cap * pc->page;
   c.L = pc->L; c.B = pc->B; c.Hq = pc->Hq; c.Hkv = pc->Hkv; c.d = pc->d; c.dtype = pc->dtype;
   c.max_len = pc->pages_cap * pc->page;
-  c.lens_lists = 0;
+  c.lens_lists = pc->lens_per_list ? pc->lists : 0;
   const PagedView pv = {pc->page_table, pc->page, pc->pages_cap, pc->lists};
   return decode_impl(&c, pv, q, new_k, new_v, layer_begin, layer_end, scale, out, out_dtype, ws, ws_bytes, dev_status,
                      (cudaStream_t)stream);

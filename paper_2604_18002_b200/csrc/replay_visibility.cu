@@ -20,12 +20,12 @@ constexpr int kThreads = 256;
 struct ReplayParams {
   const int32_t* kept_sorted;    // [R][B][G][k_max]
   const int32_t* budget;         // [R][B]
-  const int32_t* alive_before;   // [R][B]
+  const int32_t* alive_before;   // [R][B], or [R][B][G] when per_list
   const int32_t* total_before;   // [R][B]
   int32_t* alive_pos;            // [R][B][G][k_max * block]
   int32_t* alive_count;          // [R][B][G]
   int32_t* dev_status;
-  int R, B, G, k_max, block, alive_max;
+  int R, B, G, k_max, block, alive_max, per_list;
 };
 
 __global__ void __launch_bounds__(kThreads) replay_visibility_kernel(ReplayParams p) {
@@ -42,7 +42,7 @@ __global__ void __launch_bounds__(kThreads) replay_visibility_kernel(ReplayParam
     const int64_t li = ((int64_t)r * p.B + b) * p.G + gi;
     int32_t* out = p.alive_pos + li * out_stride;
     if (!fail) {
-      const int n_alive = p.alive_before[r * p.B + b];
+      const int n_alive = p.per_list ? p.alive_before[li] : p.alive_before[r * p.B + b];
       const int total = p.total_before[r * p.B + b];
       const int K = p.budget[r * p.B + b];
       const int grow = n_alive - n_prev;          // tokens appended since the last round (block_r)
@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(kThreads) replay_visibility_kernel(ReplayParam
 
 extern "C" int ngc_replay_visibility(const int32_t* kept_sorted, const int32_t* budget, const int32_t* alive_before,
                                      const int32_t* total_before, int R, int B, int G, int k_max, int block, int alive_max,
-                                     int32_t* alive_pos, int32_t* alive_count, int32_t* dev_status, ngc_stream stream) {
+                                     int per_list, int32_t* alive_pos, int32_t* alive_count, int32_t* dev_status, ngc_stream stream) {
   using namespace ngc;
   if (!kept_sorted || !budget || !alive_before || !total_before || !alive_pos || !alive_count || R <= 0 || B <= 0 || G <= 0 ||
       k_max <= 0 || block <= 0 || alive_max <= 0)
@@ -110,7 +110,7 @@ extern "C" int ngc_replay_visibility(const int32_t* kept_sorted, const int32_t* 
   ReplayParams p;
   p.kept_sorted = kept_sorted; p.budget = budget; p.alive_before = alive_before; p.total_before = total_before;
   p.alive_pos = alive_pos; p.alive_count = alive_count; p.dev_status = dev_status;
-  p.R = R; p.B = B; p.G = G; p.k_max = k_max; p.block = block; p.alive_max = alive_max;
+  p.R = R; p.B = B; p.G = G; p.k_max = k_max; p.block = block; p.alive_max = alive_max; p.per_list = per_list;
   replay_visibility_kernel<<<(unsigned)(B * G), kThreads, smem, (cudaStream_t)stream>>>(p);
   return launch_status();
 }

@@ -621,7 +621,7 @@ extern "C" int ngc_score_evict_paged(const ngc_paged_cache* pc, const void* q_re
   c.rows = (int64_t)pc->B * pc->pages_cap * pc->page;
   c.L = pc->L; c.B = pc->B; c.Hq = pc->Hq; c.Hkv = pc->Hkv; c.d = pc->d; c.dtype = pc->dtype;
   c.max_len = pc->pages_cap * pc->page;
-  c.lens_lists = 0;
+  c.lens_lists = pc->lens_per_list ? pc->lists : 0;
   const PagedView pv = {pc->page_table, pc->page, pc->pages_cap, pc->lists};
   return score_impl(&c, pv, q_recent, w, pc->page, pc->lists, log_transform, logits, n_max, ws, ws_bytes, dev_status,
                     (cudaStream_t)stream);

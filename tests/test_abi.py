@@ -121,9 +121,9 @@ def test_added_entry_points_refuse_bad_arguments(ngc):
     assert lib.ngc_score_evict_paged(C.byref(pg), 16, 5, 0, 16, 4, None, 0, None, None) == -2
     assert lib.ngc_evict_pages(None, 1, 1, 4, None, None) == -1
     # replay
-    assert lib.ngc_replay_visibility(None, 1, 1, 1, 1, 1, 1, 4, 1, 8, 1, 1, None, None) == -1
-    assert lib.ngc_replay_visibility(1, 1, 1, 1, 0, 1, 1, 4, 1, 8, 1, 1, None, None) == -1                 # no rounds
-    assert lib.ngc_replay_visibility(1, 1, 1, 1, 1, 1, 1, 4, 1, 40000, 1, 1, None, None) == -2             # alive set beyond shared memory
+    assert lib.ngc_replay_visibility(None, 1, 1, 1, 1, 1, 1, 4, 1, 8, 0, 1, 1, None, None) == -1
+    assert lib.ngc_replay_visibility(1, 1, 1, 1, 0, 1, 1, 4, 1, 8, 0, 1, 1, None, None) == -1              # no rounds
+    assert lib.ngc_replay_visibility(1, 1, 1, 1, 1, 1, 1, 4, 1, 40000, 0, 1, 1, None, None) == -2          # alive set beyond shared memory
     assert lib.ngc_replay_attn(C.byref(f32), 16, 8, None, None, None, 0, 0, 0, 1.0, 16, 0, None, None) == -2
     assert lib.ngc_replay_attn(C.byref(bf), 16, 8, None, None, None, 2, 4, 0, 1.0, 16, 0, None, None) == -1   # rounds without lists
     assert lib.ngc_replay_attn(C.byref(bf), None, 8, None, None, None, 0, 0, 0, 1.0, 16, 0, None, None) == -1

@@ -170,3 +170,55 @@ def test_paged_full_sequence_and_bad_list_are_reported():
     table = pc.page_table.cpu().numpy()
     assert np.array_equal(table[1], table_before[1]) and np.array_equal(pc.lens.cpu().numpy(), [64, 41])
     assert np.array_equal(table[0, 0, :2], table_before[0, 0][[0, 2]])
+
+
+def test_paged_lists_with_their_own_lengths():
+    """Per-layer lists on a paged cache with a partly filled last page: layers that keep it and layers
+    that evict it end at different lengths (lens [B][G]); decode and a second round follow, every layer
+    checked against the oracle run on that layer alone."""
+    b = ngc()
+    L, B, Hq, Hkv, d, dtype, page, pages_cap, lists = 3, 2, 12, 2, 128, torch.bfloat16, 32, 16, 1
+    cap = pages_cap * page
+    lens0 = [205, 77]
+    c = synth.make_cache(L, B, Hq, Hkv, d, dtype, lens0, capacity=cap, seed=21, outlier_channels=4)
+    pc = to_paged(c, page, pages_cap, lists, seed=22)
+    pc.lens = torch.as_tensor(np.repeat(np.array(lens0, np.int32)[:, None], L, 1)).cuda().contiguous()
+    so = c.seq_off.numpy()
+    kh, vh = synth.to_numpy(c.k), synth.to_numpy(c.v)
+    k_ref = [np.ascontiguousarray(kh[l:l + 1]) for l in range(L)]
+    v_ref = [np.ascontiguousarray(vh[l:l + 1]) for l in range(L)]
+    o_lens = [np.array(lens0, np.int32) for _ in range(L)]
+    st = b.new_status()
+    ws = b.alloc_workspace(b.workspace_bytes(b.OP_DECODE, pc.as_contiguous_desc()))
+    out = torch.zeros((L, B, Hq, d), dtype=torch.float32, device="cuda")
+    step = 0
+    for rnd in range(2):
+        units = np.stack([(o + page - 1) // page for o in o_lens], 1)
+        n_b, budget = units.max(1).astype(np.int32), np.maximum(1, units.min(1) // 2).astype(np.int32)
+        lg = synth.make_logits(B, L, pages_cap, seed=30 + rnd).numpy()
+        for bb in range(B):
+            for l in range(L):
+                lg[bb, l, units[bb, l]:] = -np.inf
+        r_ko, r_ks, _, rst = oracle.sample_evict(lg, n_b, None, budget, int(budget.max()), seed=3, rnd=rnd)
+        assert not rst.any()
+        b.ngc_evict_pages(pc, torch.as_tensor(r_ks).cuda(), torch.as_tensor(budget).cuda(), status=st)
+        for l in range(L):
+            k_ref[l], v_ref[l], nl, rc = oracle.compact_kv(k_ref[l], v_ref[l], so, o_lens[l], r_ks[:, l:l + 1], budget, 0, page)
+            assert rc == 0
+            o_lens[l] = nl.copy()
+        torch.cuda.synchronize()
+        assert status_value(st) == 0 and np.array_equal(pc.lens.cpu().numpy(), np.stack(o_lens, 1))
+        for _ in range(5):
+            q = synth.make_queries(L, B, Hq, d, dtype, seed=40 + step)
+            nk, nv = synth.make_new_kv(L, B, Hkv, d, dtype, seed=60 + 2 * step)
+            b.ngc_decode_attn_paged(pc, q.cuda(), out, nk.cuda(), nv.cuda(), ws=ws, status=st)
+            got = out.cpu().numpy().astype(np.float64)
+            for l in range(L):
+                ref, rc = oracle.decode_attn(k_ref[l], v_ref[l], so, o_lens[l], synth.to_numpy(q[l:l + 1]), synth.to_numpy(nk[l:l + 1]),
+                                             synth.to_numpy(nv[l:l + 1]))
+                assert rc == 0 and max_rel_err_per_vector(got[l:l + 1], ref) <= 2e-2
+            step += 1
+        torch.cuda.synchronize()
+        assert status_value(st) == 0 and np.array_equal(pc.lens.cpu().numpy(), np.stack(o_lens, 1))
+    got_lens = pc.lens.cpu().numpy()
+    assert (got_lens.max(1) != got_lens.min(1)).any()

@@ -109,3 +109,40 @@ def test_replay_visibility_rollout_loop_size():
     for r in range(1, R):
         old = got_pos[r] < total_before[r - 1][:, None, None]
         assert np.all(old.sum(-1) == (ks[r] < K).sum(-1))
+
+
+def test_replay_visibility_with_a_length_per_list():
+    """Units of 32 tokens, per-layer lists, rounds at lengths that are no multiple of 32: the layers of a sequence
+    hold different numbers of tokens, so the alive count is given per (round, sequence, list)."""
+    rng = np.random.default_rng(9)
+    R, B, G, block = 4, 3, 5, 32
+    grows = rng.integers(40, 200, (R, B))
+    total_before = np.cumsum(grows, 0).astype(np.int32)
+    alive_before = np.zeros((R, B, G), np.int32)
+    kept_n = np.zeros((B, G), np.int64)
+    budget = np.zeros((R, B), np.int32)
+    lists = []
+    for r in range(R):
+        alive_before[r] = kept_n + grows[r][:, None]
+        units = (alive_before[r] + block - 1) // block                      # [B][G]
+        budget[r] = np.maximum(1, units.min(1) // 2)
+        row = []
+        for b in range(B):
+            per_g = []
+            for g in range(G):
+                u = np.sort(rng.choice(units[b, g], budget[r, b], replace=False))
+                per_g.append(u)
+                short = units[b, g] * block - alive_before[r, b, g]
+                kept_n[b, g] = budget[r, b] * block - (short if u[-1] == units[b, g] - 1 else 0)
+            row.append(per_g)
+        lists.append(row)
+    k_max = int(budget.max())
+    ks = np.full((R, B, G, k_max), -1, np.int32)
+    for r in range(R):
+        for b in range(B):
+            for g in range(G):
+                ks[r, b, g, : budget[r, b]] = lists[r][b][g]
+    assert (alive_before.max(2) != alive_before.min(2)).any()              # the lists really differ
+    ref_pos, ref_cnt, rc = replay.alive_positions(ks, budget, alive_before, total_before, block)
+    got_pos, got_cnt, st = gpu_replay(ks, budget, alive_before, total_before, block, int(alive_before.max()))
+    assert rc == 0 and st == 0 and np.array_equal(got_cnt, ref_cnt) and np.array_equal(got_pos, ref_pos)
