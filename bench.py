@@ -50,6 +50,9 @@ OTHER_WORKLOADS = {
        "per-layer lists) + log-prob recompute of all 16 rounds",
     6: "config6: the paper's Countdown setting (L28, 12q/2kv, d128, bf16, B512 = 32 prompts x 16 rollouts, 256 prompt + 1024 generated, "
        "a round every 256 tokens 512 -> 256, units of 32 tokens, per-layer lists scored from K with 5 recent queries)",
+    8: "config8: the paper's math setting with its own cadence (L28, 12q/2kv, d128, bf16, B2048, 337 prompt + 1050 generated, a round every "
+       "350 tokens keeping 10 units of 32, per-layer lists scored from K, rounds at lengths with a short last unit: one cache length per "
+       "(rollout, layer))",
     7: "config7: the paper's math setting (L28, 12q/2kv, d128, bf16, B2048 = 256 prompts x 8 rollouts, 352 prompt + 1056 generated, "
        "a round every 352 tokens 704 -> 352, units of 32 tokens, per-layer lists scored from K with 5 recent queries)",
 }
@@ -328,8 +331,8 @@ def run_other(args):
         steps = rounds * cadence
         lens = torch.full((B,), prompt, dtype=torch.int32)
         budget = torch.full((B,), K, dtype=torch.int32)              # in units
-        cap = torch.full((B,), prompt + cadence, dtype=torch.int64)
-        n_evict = torch.full((B,), (prompt + cadence) // block, dtype=torch.int32)
+        cap = torch.full((B,), prompt + cadence + block, dtype=torch.int64)
+        n_evict = torch.full((B,), (prompt + cadence + block - 1) // block, dtype=torch.int32)
     else:
         if isinstance(cfg["T"], tuple):
             lens = synth.ragged_lens(B, cfg["T"][0], cfg["T"][1], cfg["len_seed"])
@@ -338,13 +341,16 @@ def run_other(args):
         budget = torch.ceil(lens.double() / 3).to(torch.int32) if cfg["budget"] == "third" else torch.full((B,), cfg["budget"], dtype=torch.int32)
         cap = torch.maximum(lens.long(), budget.long() + steps)
         n_evict = lens
-    n_max, k_max = int(n_evict.max()), int(budget.max())
+    n_max, k_max = max(int(n_evict.max()), (int(cap.max()) + block - 1) // block), int(budget.max())
     src = synth.make_cache(L, B, Hq, Hkv, d, dtype, lens, capacity=cap, seed=cfg["data_seed"], outlier_channels=cfg["outliers"], device=dev)
+    per_list = bool(cfg.get("per_list_lens"))
     ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=cap, n_max=n_max, k_max=k_max, lists=lists, block=block, device=dev, w=W_RECENT,
-                    kv=(src.k, src.v))
+                    kv=(src.k, src.v), per_list_lens=per_list)
     del src
     G = ro.G
     lens0 = lens.to(dev)
+    if per_list:
+        lens0 = lens0[:, None].repeat(1, G).contiguous()
     logits = ro.score_logits if from_score else synth.make_logits(B, G, n_max, seed=cfg["data_seed"] + 7, std=cfg["logit_std"], device=dev)
     n_t, k_t = n_evict.to(dev), budget.to(dev)
     p_t = torch.full((B,), cfg["n_protect"], dtype=torch.int32, device=dev) if cfg["n_protect"] else None
@@ -361,7 +367,7 @@ def run_other(args):
     if args.paged:
         # same memory viewed as page pools (one eviction unit = one page): eviction edits the tables only
         assert loop and block in (32, 64), "--paged needs a block-eviction workload (--config 6 or 7)"
-        pages_cap = (prompt + cadence) // block
+        pages_cap = (prompt + cadence + block) // block
         table = torch.arange(pages_cap, dtype=torch.int32, device=dev).repeat(B, G, 1).contiguous()
         table0 = table.clone()
         paged = ngc.NgcPagedCache(ro.cache.k.view(L, Hkv, B * pages_cap, block, d), ro.cache.v.view(L, Hkv, B * pages_cap, block, d),
@@ -373,6 +379,10 @@ def run_other(args):
     def eviction(rnd, t):
         e = [ev() for _ in range(5)]
         e[0].record()
+        if per_list:
+            # units per rollout = those of its longest layer; units a shorter layer lacks keep logit -inf
+            n_t.copy_((ro.cache.lens.max(1).values + (block - 1)) // block)
+            ro.score_logits.fill_(float("-inf"))
         if paged is not None:
             ngc.ngc_score_evict_paged(paged, q_recent, ro.score_logits, ws=ro.ws_score, status=ro.status)
         else:
@@ -474,7 +484,8 @@ def run_other(args):
     kept = float(budget.sum())
     if loop:
         kept *= block
-        vis = B * rounds * sum(prompt + s + 1 for s in range(cadence))
+        # after the first round the cache restarts from the kept units (a short last unit can cost up to block - 1 tokens less)
+        vis = B * (sum(prompt + s + 1 for s in range(cadence)) + (rounds - 1) * sum(K * block + s + 1 for s in range(cadence)))
         score_bytes = float(n_evict.sum()) * block * row_bytes / 2
     else:
         vis = sum(kept + B * (s + 1) for s in range(steps))
@@ -659,7 +670,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seqs", type=int, default=4)
     ap.add_argument("--cpu-decode-steps", type=int, default=48)
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7],
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8],
                     help="2 = the benchmark workload (default); 1, 3..7 = the other workloads, one GPU, per-phase timing only")
     ap.add_argument("--kernel", default=None, choices=["score_backward", "replay_attn"],
                     help="time one training-side call instead of the benchmark step (one GPU)")

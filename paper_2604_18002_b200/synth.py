@@ -153,4 +153,9 @@ CONFIGS = {
             budget=8, block=32, lists=1, logit_std=1.0, steps=1024, cadence=256, outliers=0, data_seed=0, noise_seed=1),
     7: dict(name="paper-math-B2048", L=28, Hq=12, Hkv=2, d=128, dtype="bf16", B=2048, T=352, n_protect=0,
             budget=11, block=32, lists=1, logit_std=1.0, steps=1056, cadence=352, outliers=0, data_seed=0, noise_seed=1),
+    # the same with the paper's own cadence of 350 tokens and a prompt that is no multiple of the unit: rounds fire at
+    # lengths with a short last unit, so the layers of a rollout keep different token counts (a length per list)
+    8: dict(name="paper-math-ragged-B2048", L=28, Hq=12, Hkv=2, d=128, dtype="bf16", B=2048, T=337, n_protect=0,
+            budget=10, block=32, lists=1, logit_std=1.0, steps=1050, cadence=350, outliers=0, data_seed=0, noise_seed=1,
+            per_list_lens=True),
 }
