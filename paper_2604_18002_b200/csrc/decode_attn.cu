@@ -587,9 +587,6 @@ size_t decode_workspace_bytes(const ngc_cache* c, int layers) {
 namespace ngc {
 namespace {
 
-// Paged layout of a call (table == nullptr: contiguous strips addressed through seq_off).
-struct PagedView { const int32_t* table; int page, pages_cap, lists; };
-
 int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* new_k, const void* new_v,
                 int layer_begin, int layer_end, float scale, void* out, int out_dtype,
                 void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {

@@ -50,6 +50,9 @@ __host__ __device__ inline int64_t len_index(int lens_lists, int L, int Hkv, int
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// Paged layout of a call (table == nullptr: contiguous strips addressed through seq_off).
+struct PagedView { const int32_t* table; int page, pages_cap, lists; };
+
 #ifdef __CUDACC__
 // Launch with programmatic stream serialisation: the kernel may begin while
 // the previous kernel of the stream drains, and waits for it on the device

@@ -517,8 +517,6 @@ size_t score_workspace_bytes(const ngc_cache* c, int G, int n_max) {
 namespace ngc {
 namespace {
 
-struct PagedView { const int32_t* table; int page, pages_cap, lists; };
-
 int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, int w, int block, int lists,
                int log_transform, float* logits, int n_max,
                void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {
