@@ -151,3 +151,109 @@ def test_replay_attention_pins():
     M = replay.dense_mask(T, total_before, [pos[i, 0, 0, : cnt[i, 0, 0]] for i in range(2)])
     rep = replay.replay_attention(qf[0, 0].astype(np.float64), kf[0].astype(np.float64), vf[0].astype(np.float64), M[None])
     assert np.abs(rep - rollout_out).max() < 1e-10
+
+
+def _random_list_history(rng, R, block, boundaries, grows):
+    """One list's rollout: random unit decisions at every boundary.  Returns the kept units per round, the alive
+    count when each round fired, and the evicted ORIGINAL positions per round (for the set simulation)."""
+    alive, kept_lists, alive_before, evicted_sets = list(range(grows[0])), [], [], []
+    for r in range(R):
+        n_units = (len(alive) + block - 1) // block
+        K = int(rng.integers(1, n_units + 1))
+        units = sorted(rng.choice(n_units, K, replace=False).tolist())
+        keep_idx = [i for u in units for i in range(u * block, min((u + 1) * block, len(alive)))]
+        alive_before.append(len(alive))
+        kept_lists.append(units)
+        evicted_sets.append(set(alive) - {alive[i] for i in keep_idx})
+        alive = [alive[i] for i in keep_idx] + list(range(boundaries[r], boundaries[r] + grows[r + 1]))
+    return kept_lists, alive_before, evicted_sets
+
+
+def test_per_list_alive_counts_match_independent_lists_and_set_simulation():
+    """Several lists per sequence whose alive counts differ (Section 4.1: every layer evicts the same fraction but not
+    the same entries, so with units of several tokens a short last unit kept by one layer and evicted by another
+    leaves the layers with different lengths).  The [R][B][G] form of `alive_before` must give, list by list, what G
+    separate single-list calls give, and each list must agree with the token-by-token set simulation."""
+    rng = np.random.default_rng(11)
+    for trial in range(12):
+        block = int(rng.choice([4, 32]))
+        R, B, G = int(rng.integers(2, 5)), 2, 3
+        # growth that is NOT a multiple of the unit, so that the last unit of a round is short
+        grows = [[int(rng.integers(block + 1, 3 * block + 2)) | 1 for _ in range(R + 1)] for _ in range(B)]
+        hist = [[None] * G for _ in range(B)]
+        bounds = [[int(x) for x in np.cumsum(grows[b][:-1])] for b in range(B)]
+        # every list of a sequence keeps the same number of UNITS per round (one budget per sequence), drawn per
+        # sequence; which units -- and therefore whether the short last one survives -- differs per list
+        for b in range(B):
+            alive = [list(range(grows[b][0])) for _ in range(G)]
+            kept_l = [[] for _ in range(G)]
+            ab_l = [[] for _ in range(G)]
+            ev_l = [[] for _ in range(G)]
+            for r in range(R):
+                n_units = [(len(a) + block - 1) // block for a in alive]
+                K = int(rng.integers(1, min(n_units) + 1))
+                for g in range(G):
+                    units = sorted(rng.choice(n_units[g], K, replace=False).tolist())
+                    if g == 0 and n_units[g] - 1 not in units:          # list 0 always keeps the (short) last unit
+                        units[-1] = n_units[g] - 1
+                    if g == 1 and K < n_units[g] and n_units[g] - 1 in units:   # list 1 drops it when it can
+                        free = sorted(set(range(n_units[g] - 1)) - set(units))
+                        units = sorted(units[:-1] + [free[0]])
+                    keep_idx = [i for u in units for i in range(u * block, min((u + 1) * block, len(alive[g])))]
+                    ab_l[g].append(len(alive[g]))
+                    kept_l[g].append(units)
+                    ev_l[g].append(set(alive[g]) - {alive[g][i] for i in keep_idx})
+                    alive[g] = [alive[g][i] for i in keep_idx] + list(range(bounds[b][r], bounds[b][r] + grows[b][r + 1]))
+            for g in range(G):
+                hist[b][g] = (kept_l[g], ab_l[g], ev_l[g])
+        k_max = max(len(k) for b in range(B) for g in range(G) for k in hist[b][g][0])
+        ks = np.full((R, B, G, k_max), -1, np.int32)
+        budget = np.zeros((R, B), np.int32)
+        ab = np.zeros((R, B, G), np.int32)
+        tb = np.zeros((R, B), np.int32)
+        for b in range(B):
+            for g in range(G):
+                for r in range(R):
+                    u = hist[b][g][0][r]
+                    ks[r, b, g, : len(u)] = u
+                    budget[r, b] = len(u)
+                    ab[r, b, g] = hist[b][g][1][r]
+                    tb[r, b] = bounds[b][r]
+        assert any(len(set(ab[r, b])) > 1 for r in range(R) for b in range(B)), "the lists never disagreed"
+        pos, count, rc = replay.alive_positions(ks, budget, ab, tb, block)
+        assert rc == 0
+        for b in range(B):
+            T = int(sum(grows[b]))
+            for g in range(G):
+                # (i) the per-list call equals a single-list call on that list alone
+                p1, c1, rc1 = replay.alive_positions(ks[:, b:b + 1, g:g + 1], budget[:, b:b + 1], ab[:, b:b + 1, g],
+                                                     tb[:, b:b + 1], block)
+                assert rc1 == 0
+                assert np.array_equal(c1[:, 0, 0], count[:, b, g])
+                assert np.array_equal(p1[:, 0, 0], pos[:, b, g])
+                # (ii) and the token-by-token simulation of that list's cache
+                M = replay.dense_mask(T, bounds[b], [pos[r, b, g, : count[r, b, g]] for r in range(R)])
+                vis = simulate_with_sets(T, bounds[b], hist[b][g][2])
+                for t in range(T):
+                    assert set(np.nonzero(M[t])[0].tolist()) == vis[t], (trial, b, g, t)
+
+
+def test_per_list_form_is_not_confused_with_the_per_sequence_form():
+    """[R][B] alive counts are broadcast over the lists; [R][B][G] counts are taken list by list in that index order
+    (a transposed reshape would hand list g of sequence b the count of another list)."""
+    R, B, G, block = 1, 2, 2, 1
+    ks = np.full((R, B, G, 3), -1, np.int32)
+    ab = np.array([[[3, 5], [4, 6]]], np.int32)                  # [R][B][G]: all different
+    for b in range(B):
+        for g in range(G):
+            ks[0, b, g, :2] = [0, ab[0, b, g] - 1]               # keep the first and the last alive entry
+    tb = np.full((R, B), 6, np.int32)
+    pos, count, rc = replay.alive_positions(ks, np.full((R, B), 2), ab, tb, block)
+    assert rc == 0 and np.all(count == 2)
+    for b in range(B):
+        for g in range(G):
+            n = int(ab[0, b, g])                                 # A_0 = the last n positions before 6
+            assert list(pos[0, b, g, :2]) == [6 - n, 5]
+    # broadcast form: one count per sequence
+    pos2, count2, rc = replay.alive_positions(ks[:, :, :1], np.full((R, B), 2), ab[:, :, 0], tb, block)
+    assert rc == 0 and list(pos2[0, 1, 0, :2]) == [6 - 4, 5]
