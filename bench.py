@@ -379,14 +379,13 @@ def run_other(args):
     def eviction(rnd, t):
         e = [ev() for _ in range(5)]
         e[0].record()
-        if per_list:
-            # units per rollout = those of its longest layer; units a shorter layer lacks keep logit -inf
-            n_t.copy_((ro.cache.lens.max(1).values + (block - 1)) // block)
-            ro.score_logits.fill_(float("-inf"))
+        # with a length per list the scoring call itself reports the units of each rollout's longest layer (n_t) and
+        # writes -inf into the units a shorter layer lacks
         if paged is not None:
             ngc.ngc_score_evict_paged(paged, q_recent, ro.score_logits, ws=ro.ws_score, status=ro.status)
         else:
-            ngc.ngc_score_evict(ro.cache, q_recent, ro.block, lists, ro.score_logits, ws=ro.ws_score, status=ro.status)
+            ngc.ngc_score_evict(ro.cache, q_recent, ro.block, lists, ro.score_logits, ws=ro.ws_score, status=ro.status,
+                                n_units_out=n_t if per_list else None)
         e[1].record()
         ngc.ngc_sample_evict(logits, n_t, p_t, k_t, cfg["noise_seed"], rnd, ro.kept_order, ro.kept_sorted, None, ws=ro.ws_sample, status=ro.status)
         e[2].record()

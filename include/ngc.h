@@ -4,17 +4,23 @@
  *
  * One eviction round is   ngc_score_evict -> ngc_sample_evict -> ngc_evict_logprob
  * -> ngc_compact_kv,   after which generation continues with
- * ngc_decode_attn_ragged over the surviving entries (paper Section 4.1,
- * "grow-then-evict").
+ * ngc_decode_attn_ragged over the surviving entries (paper Section 4.1: the
+ * cache grows during generation and is pruned at each round).
  *
  * Conventions
  * -----------
- * - Plain C.  No global state except the last CUDA error code.
+ * - Plain C.  Host-side state: the last CUDA error code (per thread) and one
+ *   flag per device recording that a kernel family has been configured there
+ *   (the first call of a kernel family on each device sets its shared-memory
+ *   limit, which CUDA stores per device; make that first call outside any
+ *   stream capture).  Device-side state: none, except the built-in scratch
+ *   array of ngc_decode_attn_ragged_static (see there).
  * - Every data pointer is a DEVICE pointer owned by the caller unless the
  *   comment says "host".  The library never allocates, frees or synchronises;
  *   scratch comes from a caller-supplied workspace sized by
- *   ngc_workspace_bytes().  Every call only enqueues work on `stream`
- *   (a cudaStream_t) and returns.
+ *   ngc_workspace_bytes() (ngc_decode_attn_ragged_static alone uses its own
+ *   array instead).  Every call only enqueues work on `stream` (a
+ *   cudaStream_t, which must belong to the current device) and returns.
  * - Return value: NGC_OK or a negative ngc_status.  Invalid host-visible
  *   arguments are refused before anything is launched.  Problems only visible
  *   on the device (a budget larger than the list, a NaN logit, a corrupt kept
@@ -23,9 +29,9 @@
  *   sequence is skipped.  Kernels never trap and every wait inside them is
  *   bounded.
  * - "Lists": a sequence has G eviction lists; G = 1 (one decision shared by all
- *   layers and heads), L (one per layer, the paper's setting: Section 4.1,
- *   "the same fraction (though not the same entries) in each of the L
- *   layers"), or L*Hkv (one per layer and KV head).  List gi of sequence b is
+ *   layers and heads), L (one per layer, the paper's setting: Section 4.1 has
+ *   every layer evict an equal share of its entries but choose them on its
+ *   own), or L*Hkv (one per layer and KV head).  List gi of sequence b is
  *   row b*G + gi of every [B][G][...] array.
  * - "Units": eviction acts on units of `block` consecutive tokens (Section 4.2,
  *   block-level evictions); the last unit of a sequence may be short.
@@ -130,18 +136,26 @@ int ngc_decode_splits(const ngc_cache* c, int layers);
  *   lists    which heads are averaged: SHARED = all layers and heads,
  *            PER_LAYER = the Hq heads of the layer (the paper), PER_LAYER_KVHEAD
  *            = the Hq/Hkv heads of one KV group.
- *   logits   [B][G][n_max] fp32 out; units >= ceil(lens[b]/block) untouched.
+ *   logits   [B][G][n_max] fp32 out.  With one length per sequence, units >=
+ *            ceil(lens[b]/block) are untouched.  With a length per list
+ *            (lens_lists == lists) the sequence is scored on the units of its
+ *            LONGEST list, n_b = max over its lists of ceil(len/block): a shorter
+ *            list gets -inf in the units it lacks (never drawn by
+ *            ngc_sample_evict, no mass in Eq. (1)); units >= n_b are untouched.
+ *   n_units_out  int32 [B] out, may be NULL: n_b, the unit count per sequence to
+ *            pass to ngc_sample_evict / ngc_evict_logprob as `n` (for one length
+ *            per sequence simply ceil(lens[b]/block)).
  *   log_transform  0: logit = s_j (the paper's literal reading); 1: logit = log s_j.
  * Requires n_max >= ceil(max_len/block).  Reads K only.
  */
 int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, int lists,
-                    int log_transform, float* logits, int n_max,
+                    int log_transform, float* logits, int n_max, int32_t* n_units_out,
                     void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
 
 /*
  * Gradient of the eviction scores with respect to the recent queries and the
  * keys -- Sections 4.4 and 4.5: the eviction loss reaches the model through
- * the scores, whose inputs are recomputed "on the autograd graph".  The chain
+ * the scores, which the replay pass recomputes with gradients enabled.  The chain
  * rule through the block mean, the average over attention rows and the
  * softmax of ngc_score_evict:
  *   grad_logits   [B][G][n_max] fp32 upstream gradient (e.g. from ngc_evict_logprob_backward)
@@ -266,21 +280,29 @@ int ngc_replay_attn(const ngc_cache* c, const void* q, int t_max,
                     int32_t* dev_status, ngc_stream stream);
 
 /*
- * Physical eviction -- Section 4.1 ("permanently evicts the rest").  In place:
+ * Physical eviction -- Section 4.1 (entries that are not kept are gone for good).  In place:
  * in every (layer, KV head, sequence) strip of K and V the tokens of the kept
  * units move to the front in ascending original order, and lens[b] becomes
  * the number of kept tokens.  Bit-exact row moves; rows beyond the new length
  * are unspecified afterwards.
  *   kept_sorted [B][G][k_max] ascending unit indices (as written by
  *   ngc_sample_evict); budget int32 [B]; lists says how G maps to (layer, head).
- * A strip whose list is corrupt is left untouched and reported.
+ * Errors leave whole sequences alone: with one length per sequence (lens_lists
+ * == 0), a sequence that has a corrupt list (NGC_DEV_BAD_KEPT), or whose lists
+ * would keep different token counts (NGC_DEV_LISTS_DISAGREE: units of several
+ * tokens with a short last unit that some lists keep and others evict), is
+ * reported and none of its strips moves; its lens[b] and every row are as
+ * before the call.  With a length per list (lens_lists == lists) the lists are
+ * independent: a corrupt list leaves its own strips and length untouched.
+ * (While the call runs, lens[b] of such a sequence briefly holds a negative
+ * marker; it is restored before the call's last kernel ends.)
  */
 int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const int32_t* budget, int k_max,
                    int lists, int block, int32_t* dev_status, ngc_stream stream);
 
 /*
- * Decode attention over the surviving entries -- Section 4.1 (generation
- * continues "conditioned on the surviving entries").  For layers
+ * Decode attention over the surviving entries -- Section 4.1 (after a round,
+ * generation goes on with only what was kept).  For layers
  * [layer_begin, layer_end): if new_k/new_v are given, the new token's K/V row
  * is first written at position lens[b] of each strip and is visible to its
  * own query; then out = softmax(scale * q K^T) V over the alive rows, one
@@ -298,8 +320,8 @@ int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* new_k, const
                            void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
 
 /*
- * Paged variant -- Section 4.2 notes that block-level eviction "maps naturally
- * onto paged KV cache systems": with one eviction unit = one page, evicting is
+ * Paged variant -- Section 4.2 remarks that evicting whole blocks fits paged
+ * KV caches: with one eviction unit = one page, evicting is
  * an edit of a page table and no K/V row moves.
  *
  *   k, v       : [L][Hkv][B * pages_cap][page][d] elements (bf16, d = 128)
@@ -328,13 +350,14 @@ typedef struct {
 /*
  * ngc_score_evict over a paged cache: units are pages (block = page), the
  * lists are the cache's own (c->lists); K is read page by page through the
- * table.  logits [B][G][n_max], n_max >= pages_cap.  Workspace as for
+ * table.  logits [B][G][n_max], n_max >= pages_cap; n_units_out as in
+ * ngc_score_evict (may be NULL).  Workspace as for
  * NGC_OP_SCORE of a contiguous cache with rows = B * pages_cap * page and
  * max_len = pages_cap * page.
  */
 int ngc_score_evict_paged(const ngc_paged_cache* c, const void* q_recent, int w, int log_transform,
-                          float* logits, int n_max, void* ws, size_t ws_bytes, int32_t* dev_status,
-                          ngc_stream stream);
+                          float* logits, int n_max, int32_t* n_units_out, void* ws, size_t ws_bytes,
+                          int32_t* dev_status, ngc_stream stream);
 
 /*
  * Eviction on a paged cache: for every list the pages named by kept_sorted
@@ -380,6 +403,8 @@ int ngc_decode_attn_paged(ngc_paged_cache* c, const void* q, const void* new_k, 
  * - The first call on each device looks up the device address of the array
  *   (a one-off host-side set-up on the current device, serialised by a
  *   mutex); make that first call before starting any stream capture.
+ * - The array used is the CURRENT device's; a `stream` that belongs to another
+ *   device is refused with NGC_ERR_INVALID_ARG.
  * - All calls on a device share the one array, which keeps whatever the last
  *   call left in it.  Nothing in it needs to start at zero (every slot is
  *   written before it is read within a call), but two calls that overlap on

@@ -84,7 +84,7 @@ int ngc_oracle_evict_logprob_scan(const float* logits, const int32_t* n, const i
                                   const int32_t* budget, const int32_t* kept_order,
                                   int n_batches, int B, int G, int n_max, int k_max, double* logp);
 
-/* Section 4.1 "permanently evicts the rest": out-of-place definition.  For
+/* Section 4.1, physical eviction (what is not kept is gone): out-of-place definition.  For
  * every (layer, head, sequence) strip, row j of k_out/v_out is the j-th kept
  * token in ascending original position.  Units are `block` tokens wide (last
  * unit may be short).  new_lens[b] = number of kept tokens.  k_out/v_out have

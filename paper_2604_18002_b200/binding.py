@@ -65,7 +65,7 @@ def _load():
     lib.ngc_decode_splits.restype = i32
     lib.ngc_decode_splits.argtypes = [C.POINTER(CacheDesc), i32]
     lib.ngc_score_evict.restype = i32
-    lib.ngc_score_evict.argtypes = [C.POINTER(CacheDesc), vp, i32, i32, i32, i32, vp, i32, vp, sz, vp, vp]
+    lib.ngc_score_evict.argtypes = [C.POINTER(CacheDesc), vp, i32, i32, i32, i32, vp, i32, vp, vp, sz, vp, vp]
     lib.ngc_sample_evict.restype = i32
     lib.ngc_sample_evict.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, u64, u64, u32, i32, vp, vp, vp, vp, sz, vp, vp]
     lib.ngc_evict_logprob.restype = i32
@@ -79,7 +79,7 @@ def _load():
     lib.ngc_decode_attn_ragged_static.restype = i32
     lib.ngc_decode_attn_ragged_static.argtypes = [C.POINTER(CacheDesc), vp, vp, vp, i32, i32, C.c_float, vp, i32, vp, vp]
     lib.ngc_score_evict_paged.restype = i32
-    lib.ngc_score_evict_paged.argtypes = [C.POINTER(PagedCacheDesc), vp, i32, i32, vp, i32, vp, sz, vp, vp]
+    lib.ngc_score_evict_paged.argtypes = [C.POINTER(PagedCacheDesc), vp, i32, i32, vp, i32, vp, vp, sz, vp, vp]
     lib.ngc_score_evict_backward.restype = i32
     lib.ngc_score_evict_backward.argtypes = [C.POINTER(CacheDesc), vp, i32, i32, i32, i32, vp, vp, i32, vp, vp, vp, sz, vp, vp]
     lib.ngc_replay_attn.restype = i32
@@ -195,13 +195,15 @@ def new_status(device="cuda") -> torch.Tensor:
 
 
 def ngc_score_evict(cache: NgcCache, q_recent: torch.Tensor, block: int, lists: int, logits: torch.Tensor,
-                    log_transform: int = 0, ws: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
-    """q_recent [L][B][Hq][w][d] -> logits [B][G][n_max] fp32 (in place)."""
+                    log_transform: int = 0, ws: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+                    n_units_out: Optional[torch.Tensor] = None):
+    """q_recent [L][B][Hq][w][d] -> logits [B][G][n_max] fp32 (in place); n_units_out int32 [B] (optional):
+    the unit count per sequence to hand to the sampler."""
     w = q_recent.shape[3]
     n_max = logits.shape[2]
     d = cache.desc()
     rc = lib.ngc_score_evict(C.byref(d), _ptr(q_recent), w, block, lists, log_transform, _ptr(logits), n_max,
-                             _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
+                             _ptr(n_units_out), _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
     _check(rc, "ngc_score_evict")
 
 
@@ -335,11 +337,12 @@ def ngc_decode_attn_paged(cache: NgcPagedCache, q: torch.Tensor, out: torch.Tens
 
 
 def ngc_score_evict_paged(cache: NgcPagedCache, q_recent: torch.Tensor, logits: torch.Tensor, log_transform: int = 0,
-                          ws: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None):
+                          ws: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+                          n_units_out: Optional[torch.Tensor] = None):
     """q_recent [L][B][Hq][w][d] -> logits [B][G][n_max] fp32 (units = pages)."""
     d = cache.desc()
     rc = lib.ngc_score_evict_paged(C.byref(d), _ptr(q_recent), q_recent.shape[3], log_transform, _ptr(logits), logits.shape[2],
-                                   _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
+                                   _ptr(n_units_out), _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream())
     _check(rc, "ngc_score_evict_paged")
 
 

@@ -8,7 +8,12 @@
 // before the first store of tile i (one __syncthreads per tile).  The leading
 // run of tokens that already sit in place is skipped.  HBM-bound: 16-byte
 // vector loads/stores, five CTAs per SM, next tile prefetched into registers
-// before the current one is stored.  The row width is a template parameter:
+// before the current one is stored.  With several lists per sequence and one
+// length per sequence, a check kernel runs first: a sequence with a corrupt list,
+// or whose lists would keep different token counts, is reported and marked
+// (its length entry is complemented for the duration of the call) so that NONE
+// of its strips moves; the length kernel behind restores the entry.
+// The row width is a template parameter:
 // with run-time divisions in the per-vector index arithmetic the kernel was
 // issue-bound (ncu: 61 % issue slots busy at 60 % of DRAM throughput).
 // (Measured alternatives that were slower on B200: per-row bulk async copies,
@@ -92,6 +97,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
   const int l = s / p.Hkv;
   const int gi = list_of(p.lists, l, h, p.Hkv);
   const int len = p.lens[len_index(p.lens_lists, p.L, p.Hkv, b, l, h)];
+  if (len < 0) return;          // marked by the check kernel: the sequence stays as it is (already reported)
   const int K = p.budget[b];
   const int32_t* kept = p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max;
 
@@ -172,6 +178,35 @@ __device__ int validate_list_warp(const int32_t* kept, int K, int k_max, int len
   return tokens;
 }
 
+// Before any strip moves (several lists per sequence, one length per sequence): one CTA per sequence, a
+// warp per list, checks every list of the sequence.  If one is corrupt, or the lists would keep different
+// token counts (a short last unit that some keep and some evict), the sequence is reported and its length
+// entry is replaced by its complement (a negative number) for the rest of the call: the strip kernel
+// skips such a sequence entirely and the length kernel restores the entry, so the sequence is left
+// exactly as it was.
+__global__ void compact_check_kernel(CompactParams p) {
+  __shared__ int s_bad, s_min, s_max;
+  const int b = blockIdx.x;
+  const int K = p.budget[b];
+  const int len = p.lens[b];
+  if (threadIdx.x == 0) { s_bad = 0; s_min = 0x7fffffff; s_max = -1; }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  for (int gi = warp; gi < p.G; gi += n_warps) {
+    const int t = len < 0 ? -1 : validate_list_warp(p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max, K, p.k_max, len, p.block);
+    if ((threadIdx.x & 31) == 0) {
+      if (t < 0) atomicOr(&s_bad, 1);
+      else { atomicMin(&s_min, t); atomicMax(&s_max, t); }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (s_bad) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
+    else if (s_min != s_max) set_dev_status(p.dev_status, NGC_DEV_LISTS_DISAGREE);
+    if ((s_bad || s_min != s_max) && len >= 0) const_cast<int32_t*>(p.lens)[b] = ~len;
+  }
+}
+
 // After all strips moved: the lengths become the kept token counts (one CTA per sequence, a warp per
 // list; every list is re-validated).  With one length per sequence the lists must agree; with a
 // length per list each list gets its own count.
@@ -180,6 +215,11 @@ __global__ void compact_lens_kernel(CompactParams p) {
   const int b = blockIdx.x;
   const int K = p.budget[b];
   const bool per_list = p.lens_lists != 0;          // then lens_lists == lists: every list has its own length
+  if (!per_list && p.lens[b] < 0) {                 // marked by the check kernel: put the length back, nothing moved
+    __syncthreads();                                // (every thread has read the entry)
+    if (threadIdx.x == 0) const_cast<int32_t*>(p.lens)[b] = ~p.lens[b];
+    return;
+  }
   if (threadIdx.x == 0) { s_bad = 0; s_min = 0x7fffffff; s_max = -1; }
   __syncthreads();
   const int warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
@@ -294,13 +334,20 @@ extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const in
   const int64_t strips = (int64_t)c->L * c->Hkv * c->B * 2;
   if (strips > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
   if ((((uintptr_t)c->k | (uintptr_t)c->v) & 15) != 0) return NGC_ERR_INVALID_ARG;      // rows move as 16-byte vectors
+  if (p.row_vecs != 8 && p.row_vecs != 16 && p.row_vecs != 32) return NGC_ERR_UNSUPPORTED;
+  const int lens_threads = p.G > 4 ? 1024 : 128;
+  if (p.G > 1 && p.lens_lists == 0) {
+    // the strips of a sequence must move together or not at all
+    compact_check_kernel<<<c->B, lens_threads, 0, (cudaStream_t)stream>>>(p);
+    const int rc0 = launch_status();
+    if (rc0 != NGC_OK) return rc0;
+  }
   if (p.row_vecs == 8) compact_kernel<8><<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
   else if (p.row_vecs == 16) compact_kernel<16><<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
-  else if (p.row_vecs == 32) compact_kernel<32><<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
-  else return NGC_ERR_UNSUPPORTED;
+  else compact_kernel<32><<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
   int rc = launch_status();
   if (rc != NGC_OK) return rc;
-  compact_lens_kernel<<<c->B, p.G > 4 ? 1024 : 128, 0, (cudaStream_t)stream>>>(p);
+  compact_lens_kernel<<<c->B, lens_threads, 0, (cudaStream_t)stream>>>(p);
   return launch_status();
 }
 

@@ -29,8 +29,6 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include <mutex>
-
 #include "kv_map.cuh"
 #include "ngc_common.cuh"
 #include "ngc_plan.h"
@@ -570,13 +568,23 @@ int decode_n_split(const ngc_cache* c, int layers) {
   return ns < 1 ? 1 : ns;
 }
 
+// Scratch of ONE call over `n_layers` layers: the split partials, o [items][d] fp32 then (m, l) [items]
+// (0 when the call does not split).  *ml_offset (if given) gets the byte offset of the (m, l) array.
+size_t decode_call_scratch_bytes(const ngc_cache* c, int n_layers, size_t* ml_offset) {
+  const int ns = decode_n_split(c, n_layers);
+  if (ml_offset) *ml_offset = 0;
+  if (ns <= 1) return 0;
+  const size_t items = (size_t)n_layers * c->B * c->Hq * ns;
+  const size_t o_bytes = align256(items * c->d * 4);
+  if (ml_offset) *ml_offset = o_bytes;
+  return o_bytes + align256(items * 8);
+}
+
+// Workspace that serves a call over any layer range of up to `layers` layers.
 size_t decode_workspace_bytes(const ngc_cache* c, int layers) {
   size_t worst = 0;
   for (int n = 1; n <= layers; ++n) {
-    const int ns = decode_n_split(c, n);
-    if (ns <= 1) continue;
-    const size_t items = (size_t)n * c->B * c->Hq * ns;
-    const size_t bytes = align256(items * c->d * 4) + align256(items * 8);
+    const size_t bytes = decode_call_scratch_bytes(c, n, nullptr);
     if (bytes > worst) worst = bytes;
   }
   return worst;
@@ -612,11 +620,11 @@ int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* ne
   p.lens_lists = c->lens_lists;
   p.G = lists_G(pv.lists, c->L, c->Hkv);
   if (p.n_split > 1) {
-    const size_t items = (size_t)p.n_layers * c->B * c->Hq * p.n_split;
-    const size_t need = align256(items * c->d * 4) + align256(items * 8);
+    size_t ml_offset = 0;
+    const size_t need = decode_call_scratch_bytes(c, p.n_layers, &ml_offset);
     if (!ws || ws_bytes < need || ((uintptr_t)ws & 255)) return NGC_ERR_WORKSPACE;
     p.part_o = (float*)ws;
-    p.part_ml = (float2*)((char*)ws + align256(items * c->d * 4));
+    p.part_ml = (float2*)((char*)ws + ml_offset);
   }
 
   const bool stream_path = c->dtype == NGC_BF16 && c->d == 128 && p.g <= 16 && c->rows < 0x7fffffffLL;
@@ -630,16 +638,17 @@ int decode_impl(ngc_cache* c, const PagedView& pv, const void* q, const void* ne
       return NGC_ERR_UNSUPPORTED;
     const int64_t items = (int64_t)p.n_layers * c->B * c->Hkv * p.n_split;
     if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, [&] {
-      attr_err = cudaFuncSetAttribute(decode_stream_t_kernel<1, kStages1, kMinCtas1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      kStages1 * kStageBytes + 1024);
-      if (attr_err == cudaSuccess)
-        attr_err = cudaFuncSetAttribute(decode_stream_t_kernel<2, kStages2, kMinCtas2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kStages2 * kStageBytes + 1024);
+    // the opt-in to more than 48 KB of dynamic shared memory is stored per device
+    static PerDeviceOnce attr_once;
+    const int attr_rc = attr_once.run([] {
+      cudaError_t e = cudaFuncSetAttribute(decode_stream_t_kernel<1, kStages1, kMinCtas1>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, kStages1 * kStageBytes + 1024);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(decode_stream_t_kernel<2, kStages2, kMinCtas2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kStages2 * kStageBytes + 1024);
+      return e;
     });
-    if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+    if (attr_rc != NGC_OK) return attr_rc;
     if (p.g <= 8)
       NGC_CUDA_TRY(launch_pdl(decode_stream_t_kernel<1, kStages1, kMinCtas1>, dim3((unsigned)items), dim3(kStreamThreads),
                               kStages1 * kStageBytes + 1024, stream, maps, p));
@@ -711,17 +720,8 @@ namespace {
 
 static __device__ __align__(256) unsigned char g_static_scratch[NGC_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
-std::mutex g_static_scratch_mutex;
+PerDeviceOnce g_static_scratch_once;
 void* g_static_scratch_addr[kMaxDevices] = {nullptr};
-
-// Scratch bytes one call over `n_layers` layers uses (0 when it does not split).
-size_t decode_call_scratch_bytes(const ngc_cache* c, int n_layers) {
-  const int ns = decode_n_split(c, n_layers);
-  if (ns <= 1) return 0;
-  const size_t items = (size_t)n_layers * c->B * c->Hq * ns;
-  return align256(items * c->d * 4) + align256(items * 8);
-}
 
 }  // namespace
 }  // namespace ngc
@@ -731,21 +731,25 @@ extern "C" int ngc_decode_attn_ragged_static(ngc_cache* c, const void* q, const 
                                              void* out, int out_dtype, int32_t* dev_status, ngc_stream stream) {
   using namespace ngc;
   if (!valid_cache(c) || layer_begin < 0 || layer_end > c->L || layer_begin >= layer_end) return NGC_ERR_INVALID_ARG;
-  if (decode_call_scratch_bytes(c, layer_end - layer_begin) > (size_t)NGC_STATIC_SCRATCH_BYTES)
+  if (decode_call_scratch_bytes(c, layer_end - layer_begin, nullptr) > (size_t)NGC_STATIC_SCRATCH_BYTES)
     return NGC_ERR_STATIC_SCRATCH;
+  // Every GPU has its own copy of the array, at its own address: look it up once per device while that
+  // device is current (in host code the array's name is only a stand-in for the symbol, not an address).
   int dev = -1;
-  NGC_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= kMaxDevices) return NGC_ERR_UNSUPPORTED;
-  void* scratch = nullptr;
-  {
-    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
-    if (!g_static_scratch_addr[dev]) {
-      void* p = nullptr;
-      NGC_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));   // device address on the current device
-      g_static_scratch_addr[dev] = p;
-    }
-    scratch = g_static_scratch_addr[dev];
-  }
+  const int rc = g_static_scratch_once.run([&] {
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    void* addr = nullptr;
+    if (e == cudaSuccess) e = cudaGetSymbolAddress(&addr, g_static_scratch);
+    if (e == cudaSuccess) g_static_scratch_addr[cur] = addr;
+    return e;
+  }, &dev);
+  if (rc != NGC_OK) return rc;
+  // The scratch used is the current device's: a stream of another device would make the kernels write
+  // through an address that means something else there.
+  int stream_dev = -1;
+  NGC_CUDA_TRY(cudaStreamGetDevice((cudaStream_t)stream, &stream_dev));
+  if (stream_dev != dev) return NGC_ERR_INVALID_ARG;
   return ngc_decode_attn_ragged(c, q, new_k, new_v, layer_begin, layer_end, scale, out, out_dtype,
-                                scratch, (size_t)NGC_STATIC_SCRATCH_BYTES, dev_status, stream);
+                                g_static_scratch_addr[dev], (size_t)NGC_STATIC_SCRATCH_BYTES, dev_status, stream);
 }

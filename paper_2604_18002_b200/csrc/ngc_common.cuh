@@ -4,6 +4,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "ngc.h"
 
 namespace ngc {
@@ -49,6 +52,34 @@ __host__ __device__ inline int64_t len_index(int lens_lists, int L, int Hkv, int
 }
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// Set-up that CUDA keeps PER DEVICE (a kernel's opt-in to more than 48 KB of dynamic shared
+// memory, the address of a __device__ symbol) and that a launcher wants to do once: the first
+// call made while a given device is current runs `setup` for that device, later calls on the
+// same device return at once.  One instance per launcher (a function-local static).
+constexpr int kMaxDevices = 64;
+class PerDeviceOnce {
+ public:
+  // `setup` returns a cudaError_t.  Returns an ngc_status; *device (if given) gets the current device.
+  template <typename F> int run(F&& setup, int* device = nullptr) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return NGC_ERR_UNSUPPORTED;
+    if (device) *device = dev;
+    if (done_[dev].load(std::memory_order_acquire)) return NGC_OK;
+    std::lock_guard<std::mutex> lock(mu_);
+    if (done_[dev].load(std::memory_order_relaxed)) return NGC_OK;
+    e = setup();
+    if (e != cudaSuccess) return cuda_fail(e);
+    done_[dev].store(true, std::memory_order_release);
+    return NGC_OK;
+  }
+
+ private:
+  std::mutex mu_;
+  std::atomic<bool> done_[kMaxDevices] = {};
+};
 
 // Paged layout of a call (table == nullptr: contiguous strips addressed through seq_off).
 struct PagedView { const int32_t* table; int page, pages_cap, lists; };

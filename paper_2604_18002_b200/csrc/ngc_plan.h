@@ -14,6 +14,7 @@ constexpr int kSampleSmemMaxUnits = 16384;
 
 // Number of token-range splits a decode launch over `layers` layers uses.
 int decode_n_split(const ngc_cache* c, int layers);
+size_t decode_call_scratch_bytes(const ngc_cache* c, int n_layers, size_t* ml_offset);
 size_t decode_workspace_bytes(const ngc_cache* c, int layers);
 
 size_t sample_workspace_bytes(int B, int G, int n_max);

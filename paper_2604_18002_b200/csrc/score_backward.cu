@@ -20,7 +20,6 @@
 //      in a fixed order (no float atomics: results are reproducible).
 #include <cuda_bf16.h>
 
-#include <mutex>
 
 #include "kv_map.cuh"
 #include "ngc_common.cuh"
@@ -515,14 +514,13 @@ template <int NT>
 int launch_bwd(const CUtensorMap& map_k, const CUtensorMap& map_gk, const BwdParams& p, unsigned grid, cudaStream_t stream) {
   const int smem_a = kStagesA * kStageBytes + 1024;
   const int smem_b = kStagesB * kStageBytes + 1024 + kStageBytes + kQBytes + 2 * kDzBytes;
-  static std::once_flag attr_once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(attr_once, [&] {
-    attr_err = cudaFuncSetAttribute(score_bwd_stats_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_a);
-    if (attr_err == cudaSuccess)
-      attr_err = cudaFuncSetAttribute(score_bwd_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_b);
+  static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
+  const int attr_rc = attr_once.run([&] {
+    cudaError_t e = cudaFuncSetAttribute(score_bwd_stats_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_a);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(score_bwd_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_b);
+    return e;
   });
-  if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+  if (attr_rc != NGC_OK) return attr_rc;
   score_bwd_stats_kernel<NT><<<grid, kThreads, smem_a, stream>>>(map_k, p);
   score_bwd_kernel<NT><<<grid, kThreads, smem_b, stream>>>(map_k, map_gk, p);
   return launch_status();

@@ -40,6 +40,7 @@ struct ScoreParams {
   const int64_t* seq_off;
   const int32_t* lens;
   float* logits;
+  int32_t* n_units_out;   // [B] or null: units of the sequence's longest list
   float2* stats;     // [strips][n_chunks][rows] (max, sum exp)
   float* psi;        // [L*Hkv*R] per-token probability mass summed over the strip's rows
   int64_t rows_R;
@@ -439,12 +440,29 @@ score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, fl
 // ---------------------------------------------------------------- list reduction
 
 __global__ void __launch_bounds__(256) score_finish_kernel(ScoreParams p) {
+  __shared__ int s_seq_units;
   const int li = blockIdx.x;                    // b * G + gi
   const int b = li / p.G, gi = li - b * p.G;
   const int T_b = p.lens[p.lens_lists ? li : b];      // a length per list means lens_lists == lists
   const int n_units = (T_b + p.block - 1) / p.block;
+  // units of the sequence's longest list: with a length per list the sampler works on that many units per
+  // sequence, and the units a shorter list does not have must carry logit -inf (never drawn, no mass in Eq. (1))
+  int seq_units = n_units;
+  if (p.lens_lists) {
+    if (threadIdx.x == 0) s_seq_units = 0;
+    __syncthreads();
+    for (int g2 = threadIdx.x; g2 < p.G; g2 += blockDim.x)
+      atomicMax(&s_seq_units, (p.lens[(int64_t)b * p.G + g2] + p.block - 1) / p.block);
+    __syncthreads();
+    seq_units = s_seq_units;
+  }
+  if (p.n_units_out && gi == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.n_units_out[b] = seq_units;
   const int u = blockIdx.y * blockDim.x + threadIdx.x;
-  if (u >= n_units || u >= p.n_max) return;
+  if (u >= p.n_max) return;
+  if (u >= n_units) {
+    if (u < seq_units) p.logits[(int64_t)li * p.n_max + u] = -INFINITY;
+    return;
+  }
   int l0, l1, h0, h1;
   if (p.lists == NGC_LISTS_SHARED) { l0 = 0; l1 = p.L; h0 = 0; h1 = p.Hkv; }
   else if (p.lists == NGC_LISTS_PER_LAYER) { l0 = gi; l1 = gi + 1; h0 = 0; h1 = p.Hkv; }
@@ -492,14 +510,13 @@ template <int NT>
 int launch_score_stream(const CUtensorMap& map_k, const ScoreParams& p, float scale_log2, int32_t* dev_status,
                         unsigned grid, cudaStream_t stream) {
   const int smem = kSStages * kSStageBytes + 1024;
-  static std::once_flag attr_once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(attr_once, [&] {
-    attr_err = cudaFuncSetAttribute(score_stream_kernel<NT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (attr_err == cudaSuccess)
-      attr_err = cudaFuncSetAttribute(score_stream_kernel<NT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
+  const int attr_rc = attr_once.run([&] {
+    cudaError_t e = cudaFuncSetAttribute(score_stream_kernel<NT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(score_stream_kernel<NT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    return e;
   });
-  if (attr_err != cudaSuccess) return cuda_fail(attr_err);
+  if (attr_rc != NGC_OK) return attr_rc;
   score_stream_kernel<NT, 1><<<grid, kSThreads, smem, stream>>>(map_k, p, scale_log2, dev_status);
   score_stream_kernel<NT, 2><<<grid, kSThreads, smem, stream>>>(map_k, p, scale_log2, dev_status);
   return launch_status();
@@ -518,7 +535,7 @@ namespace ngc {
 namespace {
 
 int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, int w, int block, int lists,
-               int log_transform, float* logits, int n_max,
+               int log_transform, float* logits, int n_max, int32_t* n_units_out,
                void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {
   if (!q_recent || !logits || w <= 0 || w > 16 || block <= 0 || lists < 0 || lists > 2 || n_max <= 0)
     return NGC_ERR_INVALID_ARG;
@@ -532,6 +549,7 @@ int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, in
 
   ScoreParams p;
   p.k = c->k; p.q_recent = q_recent; p.seq_off = c->seq_off; p.lens = c->lens; p.logits = logits;
+  p.n_units_out = n_units_out;
   p.psi = (float*)ws;
   p.stats = (float2*)((char*)ws + align256((size_t)c->L * c->Hkv * c->rows * 4));
   p.rows_R = c->rows;
@@ -598,17 +616,18 @@ int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, in
 }  // namespace ngc
 
 extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, int lists,
-                               int log_transform, float* logits, int n_max,
+                               int log_transform, float* logits, int n_max, int32_t* n_units_out,
                                void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
   using namespace ngc;
   if (!valid_cache(c)) return NGC_ERR_INVALID_ARG;
   const PagedView none = {nullptr, 0, 0, NGC_LISTS_SHARED};
-  return score_impl(c, none, q_recent, w, block, lists, log_transform, logits, n_max, ws, ws_bytes, dev_status, (cudaStream_t)stream);
+  return score_impl(c, none, q_recent, w, block, lists, log_transform, logits, n_max, n_units_out, ws, ws_bytes, dev_status,
+                    (cudaStream_t)stream);
 }
 
 extern "C" int ngc_score_evict_paged(const ngc_paged_cache* pc, const void* q_recent, int w, int log_transform,
-                                     float* logits, int n_max, void* ws, size_t ws_bytes, int32_t* dev_status,
-                                     ngc_stream stream) {
+                                     float* logits, int n_max, int32_t* n_units_out, void* ws, size_t ws_bytes,
+                                     int32_t* dev_status, ngc_stream stream) {
   using namespace ngc;
   if (!pc || !pc->k || !pc->page_table || !pc->lens || pc->L <= 0 || pc->B <= 0 || pc->Hq <= 0 || pc->Hkv <= 0 ||
       pc->Hq % pc->Hkv != 0 || pc->pages_cap <= 0 || (pc->page != 32 && pc->page != 64) || pc->lists < 0 || pc->lists > 2)
@@ -621,6 +640,6 @@ extern "C" int ngc_score_evict_paged(const ngc_paged_cache* pc, const void* q_re
   c.max_len = pc->pages_cap * pc->page;
   c.lens_lists = pc->lens_per_list ? pc->lists : 0;
   const PagedView pv = {pc->page_table, pc->page, pc->pages_cap, pc->lists};
-  return score_impl(&c, pv, q_recent, w, pc->page, pc->lists, log_transform, logits, n_max, ws, ws_bytes, dev_status,
-                    (cudaStream_t)stream);
+  return score_impl(&c, pv, q_recent, w, pc->page, pc->lists, log_transform, logits, n_max, n_units_out, ws, ws_bytes,
+                    dev_status, (cudaStream_t)stream);
 }

@@ -46,6 +46,7 @@ class NgcRollout:
         self.kept_order = torch.empty((B, self.G, k_max), dtype=torch.int32, device=device)
         self.kept_sorted = torch.empty((B, self.G, k_max), dtype=torch.int32, device=device)
         self.logp = torch.empty((1, B, self.G), dtype=torch.float64, device=device)
+        self.n_units = torch.zeros((B,), dtype=torch.int32, device=device)     # written by ngc_score_evict
         self.status = ngc.new_status(device)
         self.ws_decode = ngc.alloc_workspace(ngc.workspace_bytes(ngc.OP_DECODE, self.cache), device)
         self.ws_sample = ngc.alloc_workspace(ngc.workspace_bytes(ngc.OP_SAMPLE, None, self.G, n_max, k_max, B=B), device)
@@ -58,17 +59,22 @@ class NgcRollout:
                        rnd: int, q_recent: Optional[torch.Tensor] = None, logits: Optional[torch.Tensor] = None,
                        greedy: int = 0):
         """Samples from ``logits`` if given, else from the scores of ``q_recent``.  When both are
-        given the scores are still computed (into ``score_logits``) but the draw uses ``logits``."""
+        given the scores are still computed (into ``score_logits``) but the draw uses ``logits``.
+        With a cache length per list and a draw from the scores, ``n`` is ignored: the unit counts
+        come from the scoring call."""
         if q_recent is not None:
             target = self.score_logits if logits is not None else self.logits
-            ngc.ngc_score_evict(self.cache, q_recent, self.block, self.lists, target, ws=self.ws_score, status=self.status)
+            ngc.ngc_score_evict(self.cache, q_recent, self.block, self.lists, target, ws=self.ws_score, status=self.status,
+                                n_units_out=self.n_units)
             self.launches += 3
+            if self.cache.lens_lists and logits is None:
+                n = self.n_units        # a length per list: the library reports the unit count of each rollout's longest list
         src = logits if logits is not None else self.logits
         ngc.ngc_sample_evict(src, n, n_protect, budget, seed, rnd, self.kept_order, self.kept_sorted, None,
                              greedy=greedy, list_base=self.list_base, ws=self.ws_sample, status=self.status)
         ngc.ngc_evict_logprob(src, n, n_protect, budget, self.kept_order, self.logp, status=self.status)
         ngc.ngc_compact_kv(self.cache, self.kept_sorted, budget, self.lists, self.block, status=self.status)
-        self.launches += 4
+        self.launches += 4 + (1 if self.G > 1 and not self.cache.lens_lists else 0)     # compaction's check kernel
 
     # ---- one decode step over all layers ------------------------------------------
     def decode_step(self, q: torch.Tensor, out: torch.Tensor, new_k: Optional[torch.Tensor] = None,

@@ -60,12 +60,14 @@ def normal(shape, seed: int, dtype=torch.float32, std: float = 1.0, device="cpu"
 
 
 def make_cache(L, B, Hq, Hkv, d, dtype, lens, capacity=None, seed=0, outlier_channels=0,
-               outlier_scale=8.0, device="cpu", fill_dead_rows=True) -> Cache:
+               outlier_scale=8.0, device="cpu", fill_dead_rows=True, layers=None) -> Cache:
     """K, V ~ N(0,1); optionally ``outlier_channels`` channels of K per (layer, KV head),
     fixed over tokens, scaled by ``outlier_scale`` (the channels are the first entries of a
     seeded permutation of 0..d-1).  ``capacity`` (scalar or per-sequence) is the row capacity
     of each sequence; rows at or beyond ``lens[b]`` hold random data too unless
-    ``fill_dead_rows`` is False (then zeros)."""
+    ``fill_dead_rows`` is False (then zeros).  Every (layer, KV head) plane has a seed of its own,
+    so ``layers`` (a list of layer indices) draws just those layers of the L-layer cache, with the
+    same bytes they have in the full one: ``k``/``v`` are then ``[len(layers)][Hkv][R][d]``."""
     lens = torch.as_tensor(lens, dtype=torch.int32).reshape(B)
     if capacity is None:
         cap = lens.to(torch.int64)
@@ -75,25 +77,26 @@ def make_cache(L, B, Hq, Hkv, d, dtype, lens, capacity=None, seed=0, outlier_cha
     seq_off = torch.zeros(B + 1, dtype=torch.int64)
     seq_off[1:] = torch.cumsum(cap, 0)
     R = int(seq_off[-1])
-    k = torch.empty((L, Hkv, R, d), dtype=dtype, device=device)
-    v = torch.empty((L, Hkv, R, d), dtype=dtype, device=device)
+    layer_ids = list(range(L)) if layers is None else [int(l) for l in layers]
+    k = torch.empty((len(layer_ids), Hkv, R, d), dtype=dtype, device=device)
+    v = torch.empty((len(layer_ids), Hkv, R, d), dtype=dtype, device=device)
     # plane by plane keeps the fp32 staging buffer small for the large shapes
-    for l in range(L):
+    for li, l in enumerate(layer_ids):
         for h in range(Hkv):
             kp = torch.randn((R, d), generator=_gen(seed * 1000003 + (l * Hkv + h) * 2 + 11, device),
                              dtype=torch.float32, device=device)
             if outlier_channels:
                 perm = torch.randperm(d, generator=_gen(seed * 7919 + l * Hkv + h + 5, "cpu"))[:outlier_channels]
                 kp[:, perm.to(device)] *= outlier_scale
-            k[l, h] = kp.to(dtype)
+            k[li, h] = kp.to(dtype)
             vp = torch.randn((R, d), generator=_gen(seed * 1000003 + (l * Hkv + h) * 2 + 12, device),
                              dtype=torch.float32, device=device)
-            v[l, h] = vp.to(dtype)
+            v[li, h] = vp.to(dtype)
     if not fill_dead_rows:
         for b in range(B):
             k[:, :, int(seq_off[b]) + int(lens[b]):int(seq_off[b + 1])] = 0
             v[:, :, int(seq_off[b]) + int(lens[b]):int(seq_off[b + 1])] = 0
-    return Cache(k, v, seq_off.to(device), lens.to(device), L, B, Hq, Hkv, d)
+    return Cache(k, v, seq_off.to(device), lens.to(device), len(layer_ids), B, Hq, Hkv, d)
 
 
 def make_logits(B, G, n_max, seed, std=1.0, device="cpu") -> torch.Tensor:

@@ -81,13 +81,13 @@ def test_bad_arguments_are_refused_before_launch(ngc):
     # a list longer than the shared-memory sorter needs a workspace
     assert lib.ngc_sample_evict(1, 1, None, 1, 1, 1, 20000, 4, 0, 0, 0, 0, 1, 1, None, None, 0, None, None) == -3
     assert lib.ngc_evict_logprob(1, 1, None, 1, None, 1, 1, 1, 8, 4, 1, None, 0, None, None) == -1
-    assert lib.ngc_score_evict(C.byref(good), 1, 0, 1, 0, 0, 1, 16, None, 0, None, None) == -1
-    assert lib.ngc_score_evict(C.byref(good), 1, 5, 1, 0, 0, 1, 8, None, 0, None, None) == -1     # n_max too small
-    assert lib.ngc_score_evict(C.byref(good), 1, 5, 1, 0, 0, 1, 16, None, 0, None, None) == -3    # no workspace
+    assert lib.ngc_score_evict(C.byref(good), 1, 0, 1, 0, 0, 1, 16, None, None, 0, None, None) == -1
+    assert lib.ngc_score_evict(C.byref(good), 1, 5, 1, 0, 0, 1, 8, None, None, 0, None, None) == -1     # n_max too small
+    assert lib.ngc_score_evict(C.byref(good), 1, 5, 1, 0, 0, 1, 16, None, None, 0, None, None) == -3    # no workspace
     # a length per layer cannot serve a shared or a per-head eviction list
     per_layer = ngc.CacheDesc(1, 1, 1, 1, 16, 1, 1, 2, 1, 64, ngc.F32, 16, 1)
     assert lib.ngc_compact_kv(C.byref(per_layer), 1, 1, 4, 0, 1, None, None) == -1
-    assert lib.ngc_score_evict(C.byref(per_layer), 1, 5, 1, 2, 0, 1, 16, None, 0, None, None) == -1
+    assert lib.ngc_score_evict(C.byref(per_layer), 1, 5, 1, 2, 0, 1, 16, None, None, 0, None, None) == -1
     bad_mode = ngc.CacheDesc(1, 1, 1, 1, 16, 1, 1, 2, 1, 64, ngc.F32, 16, 3)
     assert lib.ngc_compact_kv(C.byref(bad_mode), 1, 1, 4, 0, 1, None, None) == -1
 
@@ -118,7 +118,7 @@ def test_added_entry_points_refuse_bad_arguments(ngc):
     assert lib.ngc_decode_attn_paged(C.byref(pg), 16, None, None, 0, 1, 1.0, 16, 0, None, 0, None, None) == -1
     pg = ngc.PagedCacheDesc(16, 16, 16, 16, 1, 1, 4, 4, 64, ngc.F32, 32, 4, 0)
     assert lib.ngc_decode_attn_paged(C.byref(pg), 16, None, None, 0, 1, 1.0, 16, 0, None, 0, None, None) == -2
-    assert lib.ngc_score_evict_paged(C.byref(pg), 16, 5, 0, 16, 4, None, 0, None, None) == -2
+    assert lib.ngc_score_evict_paged(C.byref(pg), 16, 5, 0, 16, 4, None, None, 0, None, None) == -2
     assert lib.ngc_evict_pages(None, 1, 1, 4, None, None) == -1
     # replay
     assert lib.ngc_replay_visibility(None, 1, 1, 1, 1, 1, 1, 4, 1, 8, 0, 1, 1, None, None) == -1

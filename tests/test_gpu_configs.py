@@ -5,9 +5,10 @@ the CPU oracle: kept sets, orders and compacted rows bit-exact; log-probs
 Inputs are generated on the GPU (seeded) in the same launch configuration the
 benchmark uses; what the oracle needs (logits, the strips of a few sampled
 sequences, their queries and new rows) is copied back to the host, so both
-sides see the same bytes.  Integer outputs are checked for EVERY list; cache
-rows and attention for sampled sequences at the first, a middle and the last
-decode step.  Eq. (1) is checked literally on sampled lists and through the
+sides see the same bytes.  Integer outputs are checked for EVERY list.  The
+1.5B- and the 7B-shaped configurations check cache rows and attention for
+EVERY sequence (whole layers streamed through host memory, attention at the
+first, a middle and the last decode step); the others for sampled sequences.  Eq. (1) is checked literally on sampled lists and through the
 (cross-checked) scan for all of them.
 """
 import math
@@ -165,14 +166,107 @@ def test_config1_tiny_fp32_every_step_every_sequence():
     run_round_and_decode(1, check_steps=list(range(64)), seqs=(0, 1, 2, 3))
 
 
+def run_round_and_decode_every_sequence(cfg_id, check_steps):
+    """Configs with one shared eviction list at full size, EVERY sequence: kept sets, orders and log-probs for all
+    lists as above; then, one layer at a time streamed through host memory, the oracle takes the layer as it was
+    generated (the per-plane seeds give the same bytes again), evicts with its own kept lists, appends the new rows of
+    every decode step and recomputes attention for all sequences at ``check_steps``; at the end the whole layer
+    (compacted rows and appended rows, every live row of every sequence) must equal the device's bit for bit.
+    Nothing the oracle reads comes from the CUDA path: only seeded inputs and its own results."""
+    b = ngc()
+    from paper_2604_18002_b200.rollout import NgcRollout
+    cfg = synth.CONFIGS[cfg_id]
+    assert cfg["lists"] == 0
+    L, Hq, Hkv, d, B, steps = cfg["L"], cfg["Hq"], cfg["Hkv"], cfg["d"], cfg["B"], cfg["steps"]
+    dtype, dev = torch.bfloat16, "cuda"
+    if isinstance(cfg["T"], tuple):
+        lens = synth.ragged_lens(B, cfg["T"][0], cfg["T"][1], cfg["len_seed"])
+    else:
+        lens = torch.full((B,), cfg["T"], dtype=torch.int32)
+    budget = torch.ceil(lens.double() / 3).to(torch.int32) if cfg["budget"] == "third" else \
+        torch.full((B,), cfg["budget"], dtype=torch.int32)
+    cap = torch.maximum(lens.long(), budget.long() + steps)
+    n_max, k_max = int(lens.max()), int(budget.max())
+    gen = dict(L=L, B=B, Hq=Hq, Hkv=Hkv, d=d, dtype=dtype, lens=lens, capacity=cap, seed=cfg["data_seed"],
+               outlier_channels=cfg["outliers"], device=dev)
+    src = synth.make_cache(**gen)
+    ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=cap, n_max=n_max, k_max=k_max, lists=0, device=dev,
+                    with_score=False, kv=(src.k, src.v))
+    ro.cache.lens.copy_(src.lens)
+    so = src.seq_off.cpu().numpy()
+    del src
+    logits = synth.make_logits(B, 1, n_max, seed=cfg["data_seed"] + 7, std=cfg["logit_std"], device=dev)
+    n_t, k_t = lens.to(dev), budget.to(dev)
+    ro.eviction_round(n_t, None, k_t, cfg["noise_seed"], 0, logits=logits)
+    torch.cuda.synchronize()
+    ro.check_status()
+
+    # ---- sample and log-prob: every list
+    lg, lens_np, budget_np = logits.cpu().numpy(), lens.numpy(), budget.numpy()
+    r_ko, r_ks, _, r_st = oracle.sample_evict(lg, lens_np, None, budget_np, k_max, seed=cfg["noise_seed"], rnd=0)
+    assert not r_st.any()
+    assert np.array_equal(ro.kept_order.cpu().numpy(), r_ko), "kept_order differs"
+    assert np.array_equal(ro.kept_sorted.cpu().numpy(), r_ks), "kept_sorted differs"
+    ref_scan, rc = oracle.evict_logprob_scan(lg, lens_np, None, budget_np, r_ko)
+    assert rc == 0 and np.max(np.abs(ro.logp.cpu().numpy() - ref_scan)) <= 1e-3
+    assert np.array_equal(ro.cache.lens.cpu().numpy(), budget_np)
+
+    # ---- decode on the GPU: all steps, whole batch; keep what the oracle will need (seeded inputs) and the outputs
+    check_steps = sorted(set(check_steps))
+    nk_all = np.empty((steps, L, B, Hkv, d), np.uint16)
+    nv_all = np.empty((steps, L, B, Hkv, d), np.uint16)
+    q_chk, out_chk = {}, {}
+    out = torch.empty((L, B, Hq, d), dtype=torch.float32, device=dev)
+    for s in range(steps):
+        q = synth.make_queries(L, B, Hq, d, dtype, seed=1000 + s, device=dev)
+        nk, nv = synth.make_new_kv(L, B, Hkv, d, dtype, seed=5000 + 2 * s, device=dev)
+        ro.decode_step(q, out, nk, nv)
+        nk_all[s], nv_all[s] = synth.to_numpy(nk), synth.to_numpy(nv)
+        if s in check_steps:
+            q_chk[s], out_chk[s] = synth.to_numpy(q), out.cpu().numpy().astype(np.float64)
+    torch.cuda.synchronize()
+    ro.check_status()
+    final_lens = budget_np + steps
+    assert np.array_equal(ro.cache.lens.cpu().numpy(), final_lens)
+    live = np.zeros(int(so[-1]), bool)                       # rows that hold a live token at the end
+    for bb in range(B):
+        live[so[bb]:so[bb] + final_lens[bb]] = True
+
+    # ---- the oracle, layer by layer
+    worst = 0.0
+    for l in range(L):
+        pre = synth.make_cache(**gen, layers=[l])
+        kc, vc, nl, rc = oracle.compact_kv(synth.to_numpy(pre.k), synth.to_numpy(pre.v), so, lens_np, r_ks, budget_np, 0)
+        del pre
+        assert rc == 0 and np.array_equal(nl, budget_np)
+        o_lens = nl.copy()
+        for s in range(steps):
+            if s in check_steps:
+                ref, rc = oracle.decode_attn(kc, vc, so, o_lens, q_chk[s][l:l + 1], nk_all[s, l:l + 1], nv_all[s, l:l + 1])
+                assert rc == 0                                # appends the step's rows and advances o_lens
+                err = max_rel_err_per_vector(out_chk[s][l], ref[0])
+                worst = max(worst, err)
+                assert err <= 2e-2, (l, s, err)
+            else:
+                rows = so[:-1] + o_lens
+                kc[0][:, rows] = nk_all[s, l].transpose(1, 0, 2)
+                vc[0][:, rows] = nv_all[s, l].transpose(1, 0, 2)
+                o_lens += 1
+        assert np.array_equal(o_lens, final_lens)
+        kg, vg = synth.to_numpy(ro.cache.k[l]), synth.to_numpy(ro.cache.v[l])
+        assert np.array_equal(kg[:, live], kc[0][:, live]), f"K rows of layer {l} differ"
+        assert np.array_equal(vg[:, live], vc[0][:, live]), f"V rows of layer {l} differ"
+    print(f"config {cfg_id}: {B} sequences x {L} layers, attention at steps {check_steps}: worst rel err {worst:.2e}")
+
+
 def test_config2_gqa_b64_full_size():
     need_gpu_gb(12)
-    run_round_and_decode(2, seqs=(0, 63), check_steps=[0, 128, 255])
+    run_round_and_decode_every_sequence(2, check_steps=[0, 128, 255])
 
 
 def test_config3_ragged_b256_full_size():
     need_gpu_gb(90)
-    run_round_and_decode(3, seqs=(0, 17, 255), check_steps=[0, 64, 127])
+    run_round_and_decode_every_sequence(3, check_steps=[0, 64, 127])
 
 
 def test_config4_per_head_b128_full_size():

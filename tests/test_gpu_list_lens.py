@@ -67,15 +67,21 @@ def test_per_list_lengths_through_three_rounds(lists):
             step += 1
         torch.cuda.synchronize()
         assert np.array_equal(dc.lens.cpu().numpy(), np.stack(o_lens, 1))
-        # scores of every list at its own length; units beyond a list's length stay at -inf
+        # scores of every list at its own length; the library itself writes -inf into the units a shorter list
+        # lacks (up to the unit count of the sequence's longest list, which it also reports) and leaves the rest alone
         qr = synth.normal((L, B, Hq, w, d), 300 + rnd, dtype)
-        logits = torch.full((B, G, n_max), float("-inf"), dtype=torch.float32, device="cuda")
-        b.ngc_score_evict(dc, qr.cuda(), block, lists, logits, ws=ws_s, status=st)
+        logits = torch.full((B, G, n_max), 123.0, dtype=torch.float32, device="cuda")
+        n_out = torch.full((B,), -5, dtype=torch.int32, device="cuda")
+        b.ngc_score_evict(dc, qr.cuda(), block, lists, logits, ws=ws_s, status=st, n_units_out=n_out)
         lg = logits.cpu().numpy()
+        units_now = np.stack([(o + block - 1) // block for o in o_lens], 1)         # [B][G]
+        assert np.array_equal(n_out.cpu().numpy(), units_now.max(1))
         for g in range(G):
             ref_s = oracle.score_evict(k_ref[g], so, o_lens[g], synth.to_numpy(heads(qr, g).contiguous()), block, 0, n_max=n_max)
             live = ~np.isnan(ref_s[:, 0])
-            assert np.all(np.isneginf(lg[:, g][~live]))
+            for bb in range(B):
+                assert np.all(np.isneginf(lg[bb, g, units_now[bb, g]:units_now[bb].max()]))
+                assert np.all(lg[bb, g, units_now[bb].max():] == 123.0)
             for bb in range(B):
                 m = live[bb]
                 assert np.max(np.abs(lg[bb, g][m] - ref_s[bb, 0][m])) <= 2e-2 * ref_s[bb, 0][m].max()
@@ -127,6 +133,7 @@ def test_one_length_per_sequence_still_reports_disagreement():
     b.ngc_compact_kv(dc, ks, torch.tensor([2], dtype=torch.int32).cuda(), 1, block, status=st)
     torch.cuda.synchronize()
     assert status_value(st) == 5 and int(dc.lens.item()) == 100
+    assert torch.equal(dc.k.cpu(), c.k) and torch.equal(dc.v.cpu(), c.v)      # nothing moved
     with pytest.raises(b.NgcError):                                           # a length per layer cannot serve per-head lists
         dl = b.NgcCache(dc.k, dc.v, dc.seq_off, torch.zeros((1, 2), dtype=torch.int32, device="cuda"), Hq, 128, 1)
         b.ngc_compact_kv(dl, ks, torch.tensor([2], dtype=torch.int32).cuda(), 2, block, status=st)

@@ -199,6 +199,30 @@ def test_compact_per_list_disagreement_is_reported():
     ks[0, 1] = [0, 1]                                      # ... layer 1 keeps two full units: 6 vs 8 tokens
     dc, st = run_compact(c, ks, [2], 1, block=4)
     assert st == 5 and int(dc.lens.item()) == 10
+    # the sequence is left exactly as it was: no strip of it moved
+    assert torch.equal(dc.k.cpu(), c.k) and torch.equal(dc.v.cpu(), c.v)
+
+
+def test_compact_sequence_with_one_corrupt_list_is_left_whole():
+    """Several lists per sequence, one length per sequence: if one of a sequence's lists is corrupt, none of its strips
+    may move (a half-compacted sequence whose length still says the old value would be unusable); the other sequences
+    are compacted as usual."""
+    L, B, Hq, Hkv, d = 3, 2, 2, 1, 128
+    c = synth.make_cache(L, B, Hq, Hkv, d, torch.bfloat16, [64, 48], capacity=64, seed=12)
+    logits = synth.make_logits(B, L, 64, seed=13).numpy()
+    budget = np.array([20, 16], np.int32)
+    ko, ks, km, st = oracle.sample_evict(logits, [64, 48], None, budget, 20, seed=4, rnd=0)
+    bad = ks.copy()
+    bad[0, 1, 5] = 64                                      # layer 1 of sequence 0: a unit beyond the cache
+    dc, st = run_compact(c, bad, budget, 1)
+    assert st == 3
+    so = c.seq_off.numpy()
+    assert list(dc.lens.cpu().numpy()) == [64, 16]
+    assert torch.equal(dc.k.cpu()[:, :, :so[1]], c.k[:, :, :so[1]]) and torch.equal(dc.v.cpu()[:, :, :so[1]], c.v[:, :, :so[1]])
+    k_ref, v_ref, nl, rc = oracle.compact_kv(synth.to_numpy(c.k), synth.to_numpy(c.v), so, c.lens.numpy(), ks, budget, 1)
+    assert rc == 0
+    sl = slice(so[1], so[1] + 16)
+    assert np.array_equal(synth.to_numpy(dc.k)[:, :, sl], k_ref[:, :, sl]) and np.array_equal(synth.to_numpy(dc.v)[:, :, sl], v_ref[:, :, sl])
 
 
 # ------------------------------------------------------------------ decode attention
@@ -537,3 +561,31 @@ def test_decode_many_short_strips(Hq, Hkv):
     ref, _ = oracle.decode_attn(k_ref, v_ref, so, lens.copy(), synth.to_numpy(q))
     got = out.cpu().numpy().astype(np.float64)
     assert max_rel_err_per_vector(got, ref) <= TOL_ATTN_BF16 and np.all(got[:, 0] == 0.0)
+
+
+def test_decode_on_a_second_device_after_the_first():
+    """The kernels' opt-in to large dynamic shared memory is stored per device: a process that drives GPU 0 and then
+    GPU 1 must get the same result on both (needs two devices; one-device boxes skip)."""
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs two CUDA devices")
+    b = ngc()
+    L, B, Hq, Hkv, d, T = 2, 3, 12, 2, 128, 500
+    c = synth.make_cache(L, B, Hq, Hkv, d, torch.bfloat16, [T, 77, 300], capacity=T + 1, seed=21, outlier_channels=4)
+    q = synth.make_queries(L, B, Hq, d, torch.bfloat16, seed=22)
+    outs = []
+    for dev in (0, 1):
+        with torch.cuda.device(dev):
+            dn = f"cuda:{dev}"
+            dc = b.NgcCache(c.k.to(dn), c.v.to(dn), c.seq_off.to(dn), c.lens.to(dn), Hq, T)
+            out = torch.zeros((L, B, Hq, d), dtype=torch.float32, device=dn)
+            st = b.new_status(dn)
+            ws = b.alloc_workspace(b.workspace_bytes(b.OP_DECODE, dc), dn)
+            b.ngc_decode_attn_ragged(dc, q.to(dn), out, ws=ws, status=st)
+            qr = synth.normal((L, B, Hq, 5, d), 23, torch.bfloat16).to(dn)
+            lg = torch.zeros((B, 1, T), dtype=torch.float32, device=dn)
+            ws2 = b.alloc_workspace(b.workspace_bytes(b.OP_SCORE, dc, 1, T), dn)
+            b.ngc_score_evict(dc, qr, 1, b.LISTS_SHARED, lg, ws=ws2, status=st)
+            torch.cuda.synchronize(dev)
+            assert int(st.item()) == 0
+            outs.append((out.cpu(), lg.cpu()))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
