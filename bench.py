@@ -9,11 +9,18 @@ rollout step at B = 64: 28 layers, 12 query / 2 KV heads, d = 128, bf16 K/V,
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ngc|reference]
 
+With --gpus N > 1 and no rank environment, the script starts its own N ranks
+(one process per GPU under torch.distributed.run on 127.0.0.1); started under
+torchrun it takes the ranks it is given.  The batch of N x 64 rollouts is cut
+into contiguous shards, one per rank, with no data-path collective.
+
 Prints ONE JSON line (rank 0).  `value` is tokens/s with all inputs resident in
 HBM; `e2e` is the same step driven from pinned host buffers through the public
 host entry (copies inside the timed region); `roofline` is the decode kernel's
-achieved HBM bandwidth; `cpu_baseline` is the CPU oracle timed on a bounded
-sample of the same workload.
+achieved HBM bandwidth, `compact` the compaction kernel's, `per_call_ms` the
+time of each of the five calls; `config3` (one GPU only) repeats the per-call
+figures on the 7B-shaped ragged batch; `cpu_baseline` is the CPU oracle timed
+on a bounded sample of the same workload.
 
 Measurement aids on one GPU (not the benchmark line):
     python bench.py --config 1|3|4|5|6|7 [--paged] [--graph]   per-phase timing of the other workloads
@@ -124,6 +131,25 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def free_port():
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def spawn_ranks_if_needed(args):
+    """`python bench.py --gpus N` with N > 1 outside a launcher: start N ranks of this script, one per GPU, and
+    return their exit code (None when this process is itself a rank or N == 1)."""
+    if args.gpus <= 1 or "RANK" in os.environ:
+        return None
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    return subprocess.call(cmd, env=env)
+
+
 def dist_setup(n_gpus):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -162,21 +188,27 @@ def run_ngc(args):
     from paper_2604_18002_b200 import binding as ngc
     from paper_2604_18002_b200.rollout import HostStep, NgcRollout
 
+    from paper_2604_18002_b200.sharding import list_base, shard_batch
+
     rank, world, local = dist_setup(args.gpus)
+    if world != args.gpus and rank == 0:
+        print(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s); reporting n_gpus = {world}", file=sys.stderr)
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
     cfg = CFG
-    L, B, Hq, Hkv, d, T, K, steps = cfg["L"], cfg["B"], cfg["Hq"], cfg["Hkv"], cfg["d"], cfg["T"], cfg["budget"], cfg["steps"]
+    L, Hq, Hkv, d, T, K, steps = cfg["L"], cfg["Hq"], cfg["Hkv"], cfg["d"], cfg["T"], cfg["budget"], cfg["steps"]
     if args.decode_steps:
         steps = args.decode_steps
-    if args.batch:
-        B = args.batch
+    B_global = (args.batch or cfg["B"]) * world
     dtype = torch.bfloat16
-    # every rank owns a full batch of B rollouts (weak scaling); Philox streams use global list ids
+    # weak scaling: the job's batch is world x 64 rollouts, cut into contiguous shards balanced by cached tokens
+    # (all equal here); Philox streams use the global list index, so the draws do not depend on the sharding
+    shard = shard_batch([T] * B_global, world)[rank]
+    B = shard[1] - shard[0]
     seed = cfg["data_seed"] + 1000 * rank
     src = synth.make_cache(L, B, Hq, Hkv, d, dtype, [T] * B, capacity=T, seed=seed, outlier_channels=cfg["outliers"], device=dev)
     ro = NgcRollout(L, B, Hq, Hkv, d, dtype, capacity=T, n_max=T, k_max=K, lists=cfg["lists"], device=dev,
-                    list_base=rank * B, w=W_RECENT, kv=(src.k, src.v))
+                    list_base=list_base(shard, 1), w=W_RECENT, kv=(src.k, src.v))
     del src
     lens0 = torch.full((B,), T, dtype=torch.int32, device=dev)
     logits = synth.make_logits(B, 1, T, seed=seed + 7, std=cfg["logit_std"], device=dev)
@@ -188,20 +220,35 @@ def run_ngc(args):
     out = torch.empty((steps, L, B, Hq, d), dtype=torch.float32, device=dev)
     noise_seed = cfg["noise_seed"]
 
-    ev_pairs = []
+    ev_marks = []
 
-    def one_step(step_idx, time_decode=False):
+    def one_step(step_idx, timed=False):
+        """The whole hot path once.  Timed steps drop an event between the calls (score | sample | log-prob | compact |
+        all decode calls of the step, none between those)."""
+        marks = []
+
+        def mark():
+            if timed:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record()
+                marks.append(e)
         ro.cache.lens.copy_(lens0, non_blocking=True)
-        ro.eviction_round(n_t, None, k_t, noise_seed, step_idx, q_recent=q_recent, logits=logits)
-        if time_decode:       # one event pair around the step's decode calls (none between them)
-            e0 = torch.cuda.Event(enable_timing=True)
-            e1 = torch.cuda.Event(enable_timing=True)
-            e0.record()
+        mark()
+        ngc.ngc_score_evict(ro.cache, q_recent, 1, cfg["lists"], ro.score_logits, ws=ro.ws_score, status=ro.status)
+        mark()
+        ngc.ngc_sample_evict(logits, n_t, None, k_t, noise_seed, step_idx, ro.kept_order, ro.kept_sorted, None,
+                             list_base=ro.list_base, ws=ro.ws_sample, status=ro.status)
+        mark()
+        ngc.ngc_evict_logprob(logits, n_t, None, k_t, ro.kept_order, ro.logp, status=ro.status)
+        mark()
+        ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, cfg["lists"], 1, status=ro.status)
+        mark()
+        ro.launches += 7          # score 3, sample 1, log-prob 1, compaction 2
         for s in range(steps):
             ro.decode_step(q[s], out[s], nk[s], nv[s])
-        if time_decode:
-            e1.record()
-            ev_pairs.append((e0, e1))
+        mark()
+        if timed:
+            ev_marks.append(marks)
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -219,7 +266,7 @@ def run_ngc(args):
     wall0 = time.perf_counter()
     t0.record()
     for k in range(args.steps):
-        one_step(args.warmup + k, time_decode=True)
+        one_step(args.warmup + k, timed=True)
     t1.record()
     torch.cuda.synchronize()
     wall1 = time.perf_counter()
@@ -232,8 +279,11 @@ def run_ngc(args):
     tokens = B * steps * world
     value = tokens / (ms_per_step * 1e-3)
 
-    # roofline of the dominant kernel (decode): algorithmic K/V bytes per launch / mean launch time
-    dec_ms = [a.elapsed_time(b) for a, b in ev_pairs]          # per step: all decode calls of the step
+    # per-call times (median over the timed steps); roofline of the dominant kernel (decode): algorithmic K/V bytes
+    # per launch / mean launch time; the same for compaction (every kept row read once and written once)
+    call_names = ["score", "sample", "logprob", "compact", "decode"]
+    per_call = {n: float(np.median([m[i].elapsed_time(m[i + 1]) for m in ev_marks])) for i, n in enumerate(call_names)}
+    dec_ms = [m[4].elapsed_time(m[5]) for m in ev_marks]       # per step: all decode calls of the step
     mean_dec_ms = float(np.sum(dec_ms)) / (len(dec_ms) * steps)   # average duration of one decode call
     visible_total = sum(B * (K + s + 1) for s in range(steps)) / steps      # per launch, averaged over the step
     bytes_per_launch = algorithmic_decode_bytes(cfg, visible_total)
@@ -244,15 +294,25 @@ def run_ngc(args):
                 "frac": round(achieved / peak, 4),
                 "traffic": int(args.traffic if args.traffic else NCU_TRAFFIC_RATIO * bytes_per_launch),
                 "traffic_source": "ncu capture of a B=16 launch scaled by tokens processed (profiles/decode_stream_t_kernel_config2.md)", "bytes_per_launch": int(bytes_per_launch),
-                "ms_per_launch": round(mean_dec_ms, 4), "decode_share_of_step": round(sum(dec_ms) / ms_total, 4)}
+                "ms_per_launch": round(mean_dec_ms, 4), "decode_share_of_step": round(sum(dec_ms) / ms_total, 4),
+                "frac_of_nominal_8TBs": round(achieved / 8000.0, 4)}
+    row_bytes = L * Hkv * 2 * d * 2
+    compact_bytes = 2.0 * B * K * row_bytes
+    cmp_gbs = compact_bytes / (per_call["compact"] * 1e-3) / 1e9
+    compact = {"kernel": "compact_kernel<16> (+ the length kernel behind it: time per ngc_compact_kv call)", "bytes": int(compact_bytes),
+               "ms": round(per_call["compact"], 4), "GB/s": round(cmp_gbs, 1), "frac": round(cmp_gbs / peak, 4), "peak_kind": f"of {peak_kind}",
+               "frac_of_nominal_8TBs": round(cmp_gbs / 8000.0, 4),
+               "note": "algorithmic bytes = every kept row of K and V read once and written once (2 x B x kept x 28672 B)"}
 
     result = {"metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
               "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
               "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-              "config": {"workload": WORKLOAD, "decode_steps": steps, "batch_per_gpu": B, "parallelism": f"batch-shard x{world}, no collective",
+              "config": {"workload": WORKLOAD, "decode_steps": steps, "batch_per_gpu": B, "batch_global": B_global,
+                         "parallelism": f"batch-shard x{world} (contiguous shards of {B}, global Philox list ids), no collective",
                          "l2": "inputs larger than L2 (7.5 GB cache streamed per decode step)", "score_in_step": True,
                          "logits": "synthetic N(0, var 2), shared list"},
-              "gpu_launches": int(launches), "roofline": roofline}
+              "gpu_launches": int(launches), "roofline": roofline, "compact": compact,
+              "per_call_ms": {n: round(v, 4) for n, v in per_call.items()}}
     if clocks is not None:
         result["clocks"] = clocks
 
@@ -295,7 +355,23 @@ def run_ngc(args):
         result["e2e"] = {"value": round(tokens / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
                          "d2h_bytes_per_step": int(d2h), "ms_per_step": round(e2e_ms, 3), "steps": e2e_steps,
                          "api": "paper_2604_18002_b200.rollout.HostStep.run (pinned host buffers; every step uploads the next step's cache into a second device buffer while it computes, decode inputs and outputs stream on copy streams)"}
-        del h_k, h_v, h_q, h_out
+        del h_k, h_v, h_q, h_nk, h_nv, h_out, hs
+
+    # ---- the 7B-shaped ragged batch, per call (one GPU only): same kernels, second target shape ----
+    if world == 1 and not args.no_config3:
+        del ro, q, nk, nv, out, logits, q_recent
+        torch.cuda.empty_cache()
+        sub = argparse.Namespace(**vars(args))
+        sub.config, sub.steps, sub.warmup, sub.batch, sub.decode_steps, sub.graph, sub.paged = 3, args.config3_steps, 3, 0, 0, False, False
+        free, _ = torch.cuda.mem_get_info()
+        if free < 90 * 2 ** 30:
+            result["config3"] = {"skipped": f"needs 90 GB of free device memory, {free / 2 ** 30:.0f} GB available"}
+        else:
+            r3 = measure_other(sub)
+            result["config3"] = {k: r3[k] for k in ("value", "unit", "ms_per_step", "steps", "warmup", "per_call_ms", "roofline", "compact",
+                                                   "gpu_launches", "clocks")}
+            result["config3"]["workload"] = r3["config"]["workload"]
+            torch.cuda.empty_cache()
 
     # ---- CPU oracle on a bounded sample (rank 0, N = 1 only) ----
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -310,7 +386,11 @@ def run_ngc(args):
 # ------------------------------------------------------------------------------------ other workloads (measurement aid)
 
 def run_other(args):
-    """Configs 3, 4 and 5 on one GPU: the same hot path, timed per phase.  Decode inputs come from a ring of
+    print(json.dumps(measure_other(args)), flush=True)
+
+
+def measure_other(args):
+    """Configs 1 and 3..8 on one GPU: the same hot path, timed per phase.  Decode inputs come from a ring of
     `ring` distinct steps (the full set would not fit beside the 60+ GB caches); outputs of a step overwrite the ring slot."""
     from paper_2604_18002_b200 import binding as ngc
     from paper_2604_18002_b200.rollout import NgcRollout
@@ -396,7 +476,7 @@ def run_other(args):
         else:
             ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, lists, block, status=ro.status)
         e[4].record()
-        ro.launches += 7          # score 3, sample 1, log-prob 1, compaction 2
+        ro.launches += 7 + (1 if G > 1 and not per_list and paged is None else 0)   # score 3, sample 1, log-prob 1, compaction 2 (+ check)
         t.append(e)
 
     graph = None
@@ -503,13 +583,15 @@ def run_other(args):
               "per_call_ms": med,
               "roofline": {"bound": "hbm", "kernel": "decode_stream_t_kernel (all decode calls of a step, launch gaps included)",
                            "achieved": round(dec_gbs, 1), "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                           "frac": round(dec_gbs / peak, 4), "decode_ms_per_step": round(dec_ms, 3), "decode_calls": steps, "traffic": None},
-              "compact": {"bytes": int(compact_bytes), "GB/s": round(cmp_gbs, 1), "frac_of_peak": round(cmp_gbs / peak, 4),
+                           "frac": round(dec_gbs / peak, 4), "frac_of_nominal_8TBs": round(dec_gbs / 8000.0, 4),
+                           "decode_ms_per_step": round(dec_ms, 3), "decode_calls": steps, "traffic": None},
+              "compact": {"bytes": int(compact_bytes), "ms": med["compact"], "GB/s": round(cmp_gbs, 1), "frac": round(cmp_gbs / peak, 4),
+                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": round(cmp_gbs / 8000.0, 4),
                           "note": "algorithmic bytes = every kept row read once and written once (rows already in place are skipped by the kernel)"},
               "score": {"bytes": int(score_bytes), "GB/s": round(score_bytes / (med["score"] * 1e-3) / 1e9, 1),
                         "note": "algorithmic bytes = K read once; the kernel streams K twice"},
               "gpu_launches": int(ro.launches - launches0), "clocks": clocks}
-    print(json.dumps(result), flush=True)
+    return result
 
 
 # ------------------------------------------------------------------------------------ training-side kernels (measurement aid)
@@ -656,17 +738,39 @@ def run_reference(args):
         "gpu_launches": 0}), flush=True)
 
 
+def run_launch_check(args):
+    """Plumbing check of the multi-rank launch (no GPU work): every rank joins the process group (gloo without CUDA),
+    takes its shard of the job's batch, meets the barrier and the max-over-ranks reduction the timed region uses;
+    rank 0 prints what it saw."""
+    from paper_2604_18002_b200.sharding import shard_batch
+    rank, world, local = dist_setup(args.gpus)
+    lens = synth.ragged_lens(64 * world, 1024, 8192, 2).tolist()
+    shards = shard_batch(lens, world)
+    barrier(world)
+    dev = f"cuda:{local}" if torch.cuda.is_available() else "cpu"
+    top = max_over_ranks(float(rank + 1), world, dev)
+    if rank == 0:
+        print(json.dumps({"impl": "launch-check", "n_gpus": world, "requested": args.gpus, "max_over_ranks": top,
+                          "shards": shards, "shard_tokens": [sum(lens[a:b]) for a, b in shards]}), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ngc", choices=["ngc", "reference"])
+    ap.add_argument("--impl", default="ngc", choices=["ngc", "reference", "launch-check"],
+                    help="ngc = the CUDA library; reference = the CPU oracle on a bounded sample; launch-check = rank plumbing only")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's 256 decode steps (profiling only)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's B = 64 (profiling only)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-config3", action="store_true", help="skip the per-call pass over the 7B-shaped ragged batch")
+    ap.add_argument("--config3-steps", type=int, default=2)
     ap.add_argument("--cpu-seqs", type=int, default=4)
     ap.add_argument("--cpu-decode-steps", type=int, default=48)
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8],
@@ -681,8 +785,13 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ngc" and not (args.decode_steps or args.batch):
         args.warmup = 3
+    rc = spawn_ranks_if_needed(args)
+    if rc is not None:
+        raise SystemExit(rc)
     if args.impl == "reference":
         run_reference(args)
+    elif args.impl == "launch-check":
+        run_launch_check(args)
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the CPU oracle")

@@ -80,7 +80,8 @@ typedef enum {
   NGC_DEV_BAD_KEPT = 3,       /* kept list out of range, repeated or not ascending */
   NGC_DEV_STRIP_FULL = 4,     /* append would exceed the sequence's row capacity */
   NGC_DEV_LISTS_DISAGREE = 5, /* lists of one sequence keep different token counts */
-  NGC_DEV_TIMEOUT = 6         /* a bounded wait inside a kernel ran out */
+  NGC_DEV_TIMEOUT = 6,        /* a bounded wait inside a kernel ran out */
+  NGC_DEV_DEBUG_BOUNDS = 7    /* bounds-checking build only: a kernel computed an index outside its array */
 } ngc_dev_status;
 
 typedef enum { NGC_F32 = 0, NGC_BF16 = 1 } ngc_dtype;
@@ -415,6 +416,20 @@ int ngc_decode_attn_paged(ngc_paged_cache* c, const void* q, const void* new_k, 
 int ngc_decode_attn_ragged_static(ngc_cache* c, const void* q, const void* new_k, const void* new_v,
                                   int layer_begin, int layer_end, float scale,
                                   void* out, int out_dtype, int32_t* dev_status, ngc_stream stream);
+
+/*
+ * Self-test of the bounded wait.  (The paper has no counterpart: this is a
+ * diagnostic of the library's own safety contract.)  The streaming kernels wait
+ * for their TMA data on mbarriers with a time limit; when a wait runs out the
+ * kernel records NGC_DEV_TIMEOUT in *dev_status and runs on to its end.  This
+ * call launches one warp that waits, for at most limit_us microseconds
+ * (1 .. 100000), on a barrier that nothing ever completes, so that the path
+ * can be exercised on a healthy device: afterwards *dev_status is
+ * NGC_DEV_TIMEOUT (if it was 0 before), *waited_ns (device uint64, may be
+ * NULL) holds the time spent waiting, and the stream and context are usable as
+ * before.  dev_status must not be NULL.
+ */
+int ngc_selftest_bounded_wait(uint32_t limit_us, int32_t* dev_status, uint64_t* waited_ns, ngc_stream stream);
 
 #ifdef __cplusplus
 }

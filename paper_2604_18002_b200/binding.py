@@ -7,6 +7,7 @@ and so does every call made without a CUDA device.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes as C
 import os
 from dataclasses import dataclass
@@ -22,11 +23,11 @@ LISTS_SHARED, LISTS_PER_LAYER, LISTS_PER_LAYER_KVHEAD = 0, 1, 2
 OP_SCORE, OP_SAMPLE, OP_LOGPROB, OP_COMPACT, OP_DECODE, OP_SCORE_BACKWARD = range(6)
 
 DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "strip full",
-              5: "lists disagree", 6: "timeout"}
+              5: "lists disagree", 6: "timeout", 7: "index out of bounds (bounds-checking build)"}
 
 EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
            "ngc_sample_evict", "ngc_evict_logprob", "ngc_evict_logprob_backward", "ngc_compact_kv", "ngc_decode_attn_ragged",
-           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged", "ngc_replay_visibility", "ngc_score_evict_backward", "ngc_replay_attn"]
+           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged", "ngc_replay_visibility", "ngc_score_evict_backward", "ngc_replay_attn", "ngc_selftest_bounded_wait"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -49,12 +50,12 @@ class PagedCacheDesc(C.Structure):
                 ("lens_per_list", C.c_int32)]
 
 
-def _load():
-    if not os.path.exists(LIB_PATH):
+def _load(path: str = LIB_PATH):
+    if not os.path.exists(path):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2604_18002_b200.build` "
+            f"{path} is missing: build it with `python -m paper_2604_18002_b200.build` "
             "(there is no CPU fallback)")
-    lib = C.CDLL(LIB_PATH)
+    lib = C.CDLL(path)
     vp, i32, u32, u64, sz = C.c_void_p, C.c_int, C.c_uint32, C.c_uint64, C.c_size_t
     lib.ngc_version.restype = i32
     lib.ngc_strerror.restype = C.c_char_p
@@ -86,6 +87,8 @@ def _load():
     lib.ngc_replay_attn.argtypes = [C.POINTER(CacheDesc), vp, i32, vp, vp, vp, i32, i32, i32, C.c_float, vp, i32, vp, vp]
     lib.ngc_replay_visibility.restype = i32
     lib.ngc_replay_visibility.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.ngc_selftest_bounded_wait.restype = i32
+    lib.ngc_selftest_bounded_wait.argtypes = [u32, vp, vp, vp]
     lib.ngc_evict_pages.restype = i32
     lib.ngc_evict_pages.argtypes = [C.POINTER(PagedCacheDesc), vp, vp, i32, vp, vp]
     lib.ngc_decode_attn_paged.restype = i32
@@ -94,6 +97,18 @@ def _load():
 
 
 lib = _load()
+
+
+@contextlib.contextmanager
+def use_library(path: str):
+    """Route every call of this module to another build of the library (the bounds-checking or the
+    NVTX build) for the duration of the block."""
+    global lib
+    saved, lib = lib, _load(path)
+    try:
+        yield lib
+    finally:
+        lib = saved
 
 
 def _check(rc: int, what: str):
@@ -381,3 +396,10 @@ def ngc_replay_attn(cache: NgcCache, q: torch.Tensor, out: torch.Tensor, alive_p
     rc = lib.ngc_replay_attn(C.byref(d), _ptr(q), t_max, _ptr(alive_pos), _ptr(alive_count), _ptr(total_before), n_rounds, kt_max,
                              lists, scale, _ptr(out), _dtype_code(out), _ptr(status), _stream())
     _check(rc, "ngc_replay_attn")
+
+
+def ngc_selftest_bounded_wait(limit_us: int, status: torch.Tensor, waited_ns: Optional[torch.Tensor] = None):
+    """One warp waits at most ``limit_us`` microseconds on a barrier that never completes; ``status`` becomes the
+    timeout code and the call returns normally (diagnostic of the kernels' bounded waits)."""
+    rc = lib.ngc_selftest_bounded_wait(limit_us, _ptr(status), _ptr(waited_ns), _stream())
+    _check(rc, "ngc_selftest_bounded_wait")

@@ -110,6 +110,9 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
   const int my_row = threadIdx.x / RV, my_col = threadIdx.x % RV;
   uint4* strip = (kv ? p.v : p.k) + (int64_t)(l * p.Hkv + h) * p.plane_vecs + p.seq_off[b] * RV + my_col;
   const int block = p.block;
+#ifdef NGC_DEBUG
+  const int64_t cap = p.seq_off[b + 1] - p.seq_off[b];        // rows this sequence owns in the plane
+#endif
   uint4 cur[kVecPerThread], nxt[kVecPerThread];
 
   auto load_tile = [&](int t0, uint4 (&r)[kVecPerThread]) {
@@ -124,7 +127,8 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
           const int unit = jt / block;
           src = (int64_t)kept[unit] * block + (jt - unit * block);
         }
-        r[u] = __ldcs(strip + src * RV);
+        // a kept row never lies in front of its destination, and always inside the live part of the strip
+        if (NGC_IN_BOUNDS(p.dev_status, src >= jt && src < len && src < cap)) r[u] = __ldcs(strip + src * RV);
       }
     }
   };
@@ -132,7 +136,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
       const int jt = t0 + u * kRowsPerPass + my_row;
-      if (jt < tokens) strip[(int64_t)jt * RV] = r[u];
+      if (jt < tokens && NGC_IN_BOUNDS(p.dev_status, jt < len && jt < cap)) strip[(int64_t)jt * RV] = r[u];
     }
   };
 
@@ -283,7 +287,8 @@ __global__ void evict_pages_kernel(PageEvictParams p) {
     for (int j = lane; j < p.pages_cap; j += 32) old_row[j] = row[j];
     __syncwarp();
     // kept pages to the front
-    for (int j = lane; j < K; j += 32) row[j] = old_row[kept[j]];
+    for (int j = lane; j < K; j += 32)
+      if (NGC_IN_BOUNDS(p.dev_status, kept[j] >= 0 && kept[j] < p.pages_cap && j < p.pages_cap)) row[j] = old_row[kept[j]];
     // the others behind them: walk the old row 32 entries at a time; an entry is kept iff it
     // appears in the (ascending) kept list, found by binary search
     int out = K;
@@ -296,7 +301,8 @@ __global__ void evict_pages_kernel(PageEvictParams p) {
         is_free = !(lo < K && kept[lo] == j);
       }
       const uint32_t m = __ballot_sync(0xffffffffu, is_free);
-      if (is_free) row[out + __popc(m & ((1u << lane) - 1u))] = old_row[j];
+      if (is_free && NGC_IN_BOUNDS(p.dev_status, out + __popc(m & ((1u << lane) - 1u)) < p.pages_cap))
+        row[out + __popc(m & ((1u << lane) - 1u))] = old_row[j];
       out += __popc(m);
     }
     __syncwarp();
@@ -313,6 +319,7 @@ __global__ void evict_pages_kernel(PageEvictParams p) {
 
 extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const int32_t* budget, int k_max,
                               int lists, int block, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_compact_kv");
   using namespace ngc;
   if (!valid_cache(c) || !kept_sorted || !budget || k_max <= 0 || block <= 0 || lists < 0 || lists > 2)
     return NGC_ERR_INVALID_ARG;
@@ -353,6 +360,7 @@ extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const in
 
 extern "C" int ngc_evict_pages(ngc_paged_cache* c, const int32_t* kept_sorted, const int32_t* budget, int k_max,
                                int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_evict_pages");
   using namespace ngc;
   if (!c || !c->page_table || !c->lens || !kept_sorted || !budget || k_max <= 0 || c->B <= 0 || c->L <= 0 || c->Hkv <= 0 ||
       c->pages_cap <= 0 || c->page <= 0 || c->lists < 0 || c->lists > 2)

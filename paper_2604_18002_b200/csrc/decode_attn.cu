@@ -181,8 +181,10 @@ __global__ void __launch_bounds__(kGenWarps * 32) decode_generic_kernel(DecodePa
   if (t_new >= t_begin && t_new < t_end && hq == h * p.g && warp < 2) {
     const T* src = warp ? vnew : knew;
     T* dst = (warp ? vbase : kbase) + (int64_t)t_new * D;
+    if (NGC_IN_BOUNDS(p.dev_status, t_new < p.seq_off[b + 1] - p.seq_off[b])) {
 #pragma unroll
-    for (int i = 0; i < VPL; ++i) dst[lane * VPL + i] = src[lane * VPL + i];
+      for (int i = 0; i < VPL; ++i) dst[lane * VPL + i] = src[lane * VPL + i];
+    }
   }
   if (lane == 0) { sm_m[warp] = m; sm_l[warp] = lsum; }
 #pragma unroll
@@ -262,6 +264,17 @@ __device__ __forceinline__ void issue_tile(const DecodeParams& p, const KvMaps& 
     for (int sb = 0; sb < n_sub; ++sb) {
       const int y = table ? (b * p.pages_cap + table[tile * n_sub + sb]) * p.page : row0 + t0;
       uint8_t* dst = st + sb * sub_bytes;
+      // a full tile lies inside the plane (an out-of-range TMA box would read zeros, not fault: a wrong answer)
+      if (!NGC_IN_BOUNDS(p.dev_status, y >= 0 && (int64_t)y + kTileT / n_sub <= p.rows &&
+                                           (!table || (tile * n_sub + sb < p.pages_cap && table[tile * n_sub + sb] >= 0 &&
+                                                       table[tile * n_sub + sb] < p.pages_cap)))) {
+        // keep the byte count of the stage right so that the consumers are released: fetch row 0 instead
+        ptx::tma_load_3d(dst, &m.k, 0, 0, plane, bar);
+        ptx::tma_load_3d(dst + kBoxBytes, &m.k, 64, 0, plane, bar);
+        ptx::tma_load_3d(dst + kTileBytes, &m.v, 0, 0, plane, bar);
+        ptx::tma_load_3d(dst + kTileBytes + kBoxBytes, &m.v, 64, 0, plane, bar);
+        continue;
+      }
       ptx::tma_load_3d(dst, &m.k, 0, y, plane, bar);
       ptx::tma_load_3d(dst + kBoxBytes, &m.k, 64, y, plane, bar);
       ptx::tma_load_3d(dst + kTileBytes, &m.v, 0, y, plane, bar);
@@ -272,8 +285,10 @@ __device__ __forceinline__ void issue_tile(const DecodeParams& p, const KvMaps& 
     ptx::mbar_expect_tx(bar, (uint32_t)n16 * 4 * 16 * 128);
     for (int r = 0; r < n16; ++r) {
       const int t = t0 + 16 * r;
-      const int y = table ? (b * p.pages_cap + table[t / p.page]) * p.page + t % p.page : row0 + t;
+      int y = table ? (b * p.pages_cap + table[t / p.page]) * p.page + t % p.page : row0 + t;
       uint8_t* dst = st + r * 16 * 128;
+      // the first row of every 16-row box holds a live token, hence lies inside the plane
+      if (!NGC_IN_BOUNDS(p.dev_status, y >= 0 && y < p.rows && (!table || t / p.page < p.pages_cap))) y = 0;
       ptx::tma_load_3d(dst, &m.k16, 0, y, plane, bar);
       ptx::tma_load_3d(dst + kBoxBytes, &m.k16, 64, y, plane, bar);
       ptx::tma_load_3d(dst + kTileBytes, &m.v16, 0, y, plane, bar);
@@ -394,7 +409,8 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
         *reinterpret_cast<uint4*>(dst) = piece;
         const int64_t row = table ? ((int64_t)b * p.pages_cap + table[t_new / p.page]) * p.page + t_new % p.page
                                   : p.seq_off[b] + t_new;
-        ((uint4*)(isv ? p.v : p.k))[((int64_t)(l * p.Hkv + h) * p.rows + row) * 16 + c] = piece;
+        if (NGC_IN_BOUNDS(p.dev_status, row >= 0 && row < p.rows && t_new < seq_capacity(p, b)))
+          ((uint4*)(isv ? p.v : p.k))[((int64_t)(l * p.Hkv + h) * p.rows + row) * 16 + c] = piece;
         ptx::fence_proxy_async();
         __syncwarp();
       }
@@ -542,8 +558,10 @@ decode_stream_t_kernel(const __grid_constant__ KvMaps maps, DecodeParams p) {
         store_out(p, (((int64_t)l * p.B + b) * p.Hq + hq) * 128 + c, ls > 0.f ? o / ls : 0.f);
       } else {
         const int64_t pit = (((int64_t)lr * p.B + b) * p.Hq + hq) * p.n_split + split;
-        p.part_o[pit * 128 + c] = o;
-        if (c == 0) p.part_ml[pit] = make_float2(mg, ls);
+        if (NGC_IN_BOUNDS(p.dev_status, pit >= 0 && pit < (int64_t)p.n_layers * p.B * p.Hq * p.n_split)) {
+          p.part_o[pit * 128 + c] = o;
+          if (c == 0) p.part_ml[pit] = make_float2(mg, ls);
+        }
       }
     }
   }
@@ -679,6 +697,7 @@ extern "C" int ngc_decode_attn_ragged(ngc_cache* c, const void* q, const void* n
                                       int layer_begin, int layer_end, float scale,
                                       void* out, int out_dtype,
                                       void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_decode_attn_ragged");
   using namespace ngc;
   if (!valid_cache(c)) return NGC_ERR_INVALID_ARG;
   const PagedView none = {nullptr, 0, 0, NGC_LISTS_SHARED};
@@ -690,6 +709,7 @@ extern "C" int ngc_decode_attn_paged(ngc_paged_cache* pc, const void* q, const v
                                      int layer_begin, int layer_end, float scale,
                                      void* out, int out_dtype,
                                      void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_decode_attn_paged");
   using namespace ngc;
   if (!pc || !pc->k || !pc->v || !pc->page_table || !pc->lens || pc->L <= 0 || pc->B <= 0 || pc->Hq <= 0 || pc->Hkv <= 0 ||
       pc->Hq % pc->Hkv != 0 || pc->pages_cap <= 0 || (pc->page != 32 && pc->page != 64) || pc->lists < 0 || pc->lists > 2)
@@ -729,6 +749,7 @@ void* g_static_scratch_addr[kMaxDevices] = {nullptr};
 extern "C" int ngc_decode_attn_ragged_static(ngc_cache* c, const void* q, const void* new_k, const void* new_v,
                                              int layer_begin, int layer_end, float scale,
                                              void* out, int out_dtype, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_decode_attn_ragged_static");
   using namespace ngc;
   if (!valid_cache(c) || layer_begin < 0 || layer_end > c->L || layer_begin >= layer_end) return NGC_ERR_INVALID_ARG;
   if (decode_call_scratch_bytes(c, layer_end - layer_begin, nullptr) > (size_t)NGC_STATIC_SCRATCH_BYTES)

@@ -407,6 +407,7 @@ extern "C" int ngc_evict_logprob(const float* logits, const int32_t* n, const in
                                  const int32_t* budget, const int32_t* kept_order,
                                  int n_batches, int B, int G, int n_max, int k_max, double* logp,
                                  void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_evict_logprob");
   using namespace ngc;
   (void)ws; (void)ws_bytes;
   if (!logits || !n || !budget || !kept_order || !logp || n_batches <= 0 || B <= 0 || G <= 0 || n_max <= 0 || k_max <= 0)
@@ -431,6 +432,7 @@ extern "C" int ngc_evict_logprob_backward(const float* logits, const int32_t* n,
                                           const int32_t* budget, const int32_t* kept_order, const double* grad_logp,
                                           int n_batches, int B, int G, int n_max, int k_max, float* grad_logits,
                                           void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_evict_logprob_backward");
   using namespace ngc;
   (void)ws; (void)ws_bytes;
   if (!logits || !n || !budget || !kept_order || !grad_logits || n_batches <= 0 || B <= 0 || G <= 0 || n_max <= 0 || k_max <= 0)

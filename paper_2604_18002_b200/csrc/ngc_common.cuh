@@ -7,6 +7,10 @@
 #include <atomic>
 #include <mutex>
 
+#ifdef NGC_NVTX
+#include <nvtx3/nvtx3.hpp>
+#endif
+
 #include "ngc.h"
 
 namespace ngc {
@@ -24,6 +28,27 @@ inline int cuda_fail(cudaError_t e) {
     cudaError_t _e = (expr);                            \
     if (_e != cudaSuccess) return ::ngc::cuda_fail(_e); \
   } while (0)
+
+// Optional NVTX range around every C-ABI call (build with -DNGC_NVTX): profiler timelines and launch lists then
+// name the call each kernel belongs to.  Compiles to nothing otherwise.
+#ifdef NGC_NVTX
+#define NGC_API_RANGE(name) ::nvtx3::scoped_range ngc_api_range_ { name }
+#else
+#define NGC_API_RANGE(name) do { } while (0)
+#endif
+
+// Bounds-checking build (-DNGC_DEBUG, a second library beside the normal one).  The normal build already
+// validates everything that comes from the caller (kept lists, counts, lengths); this build also checks the
+// indices the kernels COMPUTE from them (source and destination rows, TMA row coordinates, page-table slots,
+// positions in partial and output arrays) right before use.  The first violation is recorded in the status
+// word as NGC_DEV_DEBUG_BOUNDS and that access is skipped, so a wrong index shows up as a status code instead
+// of as a stray read or write.  It stands in for a memory checker: the tests rerun the small parity cases on
+// this build and require status 0.  Expands to `true` in the normal build.
+#ifdef NGC_DEBUG
+#define NGC_IN_BOUNDS(status_ptr, cond) ((cond) ? true : (::ngc::set_dev_status((status_ptr), NGC_DEV_DEBUG_BOUNDS), false))
+#else
+#define NGC_IN_BOUNDS(status_ptr, cond) (true)
+#endif
 
 // Check the launch that was just enqueued.
 inline int launch_status() {

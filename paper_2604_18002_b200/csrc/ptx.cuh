@@ -41,15 +41,16 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Waits for the phase with the given parity, for at most about one second.
-// Returns false if the wait ran out (the caller records NGC_DEV_TIMEOUT and
-// carries on so that the kernel always terminates).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+// Waits for the phase with the given parity, for at most `limit_ns` (about one second unless the caller says
+// otherwise).  Returns false if the wait ran out (the caller records NGC_DEV_TIMEOUT and carries on so that the
+// kernel always terminates).
+constexpr uint64_t kWaitLimitNs = 1000000000ull;
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   for (uint32_t spins = 0;; ++spins) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spins & 63u) == 63u && globaltimer_ns() - t0 > 1000000000ull) return false;
+    if ((spins & 63u) == 63u && globaltimer_ns() - t0 > limit_ns) return false;
   }
 }
 

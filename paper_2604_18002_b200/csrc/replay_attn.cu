@@ -295,6 +295,7 @@ extern "C" int ngc_replay_attn(const ngc_cache* c, const void* q, int t_max,
                                const int32_t* alive_pos, const int32_t* alive_count, const int32_t* total_before,
                                int n_rounds, int kt_max, int lists, float scale, void* out, int out_dtype,
                                int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_replay_attn");
   using namespace ngc;
   if (!valid_cache(c) || !q || !out || t_max <= 0 || n_rounds < 0 || lists < 0 || lists > 2 ||
       (n_rounds > 0 && (!alive_pos || !alive_count || !total_before || kt_max <= 0)))

@@ -52,7 +52,8 @@ __global__ void __launch_bounds__(kThreads) replay_visibility_kernel(ReplayParam
         fail = NGC_DEV_BAD_COUNTS;
       } else {
         if (tid == 0) s_bad = 0;
-        for (int i = tid; i < grow; i += kThreads) cur[n_prev + i] = total - grow + i;
+        for (int i = tid; i < grow; i += kThreads)
+          if (NGC_IN_BOUNDS(p.dev_status, n_prev + i < p.alive_max)) cur[n_prev + i] = total - grow + i;
         __syncthreads();
         int bad = K > n_units ? 1 : 0;
         for (int j = tid; j < K && !bad; j += kThreads) {
@@ -72,8 +73,11 @@ __global__ void __launch_bounds__(kThreads) replay_visibility_kernel(ReplayParam
             int v = -1;
             if (i < count) {
               const int j = i / p.block;
-              v = cur[kept[j] * p.block + (i - j * p.block)];
-              nxt[i] = v;
+              const int src = kept[j] * p.block + (i - j * p.block);
+              if (NGC_IN_BOUNDS(p.dev_status, src >= 0 && src < n_alive && i < p.alive_max)) {
+                v = cur[src];
+                nxt[i] = v;
+              }
             }
             out[i] = v;
           }
@@ -98,6 +102,7 @@ __global__ void __launch_bounds__(kThreads) replay_visibility_kernel(ReplayParam
 extern "C" int ngc_replay_visibility(const int32_t* kept_sorted, const int32_t* budget, const int32_t* alive_before,
                                      const int32_t* total_before, int R, int B, int G, int k_max, int block, int alive_max,
                                      int per_list, int32_t* alive_pos, int32_t* alive_count, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_replay_visibility");
   using namespace ngc;
   if (!kept_sorted || !budget || !alive_before || !total_before || !alive_pos || !alive_count || R <= 0 || B <= 0 || G <= 0 ||
       k_max <= 0 || block <= 0 || alive_max <= 0)

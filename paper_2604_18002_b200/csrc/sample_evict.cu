@@ -271,7 +271,8 @@ __global__ void sample_kernel(SampleParams p) {
     if (j < Kp) {
       idx = kRadix ? P + (int)idx_a[(j & (order_per - 1)) * nthr + (j >> order_per_log)]
                    : (int)(0xFFFFFFFFu - (uint32_t)(keys[j] & 0xFFFFFFFFull));
-      atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
+      if (NGC_IN_BOUNDS(p.dev_status, idx >= P && idx < n)) atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
+      else idx = -1;
     }
     ko[j] = idx;
   }
@@ -299,7 +300,8 @@ __global__ void sample_kernel(SampleParams p) {
     while (mm) {
       const int bit = __ffs(mm) - 1;
       mm &= mm - 1;
-      ks[pos++] = (wd << 5) + bit;
+      if (NGC_IN_BOUNDS(p.dev_status, pos >= 0 && pos < p.k_max)) ks[pos] = (wd << 5) + bit;
+      ++pos;
     }
     __syncthreads();
     if (tid == 0) {
@@ -367,10 +369,10 @@ __global__ void __launch_bounds__(kTinyWarps * 32) sample_tiny_kernel(SamplePara
   for (int j = 0; j < 32; ++j) rank += __shfl_sync(0xffffffffu, key, j) > key ? 1 : 0;
   const bool drawn = cand && rank < Kp;
   const bool kept = drawn || (lane < P);
-  if (drawn) ko[rank] = lane;
+  if (drawn && NGC_IN_BOUNDS(p.dev_status, rank < p.k_max)) ko[rank] = lane;
   for (int j = Kp + lane; j < p.k_max; j += 32) ko[j] = -1;
   const uint32_t mask = __ballot_sync(0xffffffffu, kept);
-  if (kept) ks[__popc(mask & ((1u << lane) - 1u))] = lane;
+  if (kept && NGC_IN_BOUNDS(p.dev_status, __popc(mask & ((1u << lane) - 1u)) < p.k_max)) ks[__popc(mask & ((1u << lane) - 1u))] = lane;
   for (int j = K + lane; j < p.k_max; j += 32) ks[j] = -1;
   if (km && lane < p.n_max) km[lane] = kept ? 1 : 0;
 }
@@ -395,6 +397,7 @@ extern "C" int ngc_sample_evict(const float* logits, const int32_t* n, const int
                                 uint64_t seed, uint64_t round, uint32_t list_base, int greedy,
                                 int32_t* kept_order, int32_t* kept_sorted, uint8_t* keep_mask,
                                 void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_sample_evict");
   using namespace ngc;
   if (!logits || !n || !budget || !kept_order || !kept_sorted || B <= 0 || G <= 0 || n_max <= 0 || k_max <= 0)
     return NGC_ERR_INVALID_ARG;

@@ -539,6 +539,7 @@ extern "C" int ngc_score_evict_backward(const ngc_cache* c, const void* q_recent
                                         const float* logits, const float* grad_logits, int n_max,
                                         float* grad_q_recent, void* grad_k,
                                         void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream_) {
+  NGC_API_RANGE("ngc_score_evict_backward");
   using namespace ngc;
   cudaStream_t stream = (cudaStream_t)stream_;
   if (!valid_cache(c) || !q_recent || !grad_logits || !grad_q_recent || !grad_k || w <= 0 || w > 16 || block <= 0 || lists < 0 ||

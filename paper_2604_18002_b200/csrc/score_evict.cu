@@ -287,6 +287,8 @@ score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, fl
           } else {
             y = row0 + (tile_lo + it) * kSTileT;
           }
+          // the first row of a tile holds a live token (a box that overhangs the plane reads zeros)
+          if (!NGC_IN_BOUNDS(dev_status, y >= 0 && y < p.rows_R)) y = 0;
           ptx::tma_load_3d(sp + sb * sub_bytes, &map_k, 0, y, plane, &bar_full[s]);
           ptx::tma_load_3d(sp + sb * sub_bytes + kSBoxBytes, &map_k, 64, y, plane, &bar_full[s]);
         }
@@ -398,7 +400,7 @@ score_stream_kernel(const __grid_constant__ CUtensorMap map_k, ScoreParams p, fl
           p0 += __shfl_xor_sync(0xffffffffu, p0, 2);
           p1 += __shfl_xor_sync(0xffffffffu, p1, 1);
           p1 += __shfl_xor_sync(0xffffffffu, p1, 2);
-          if (tig == 0) {
+          if (tig == 0 && NGC_IN_BOUNDS(dev_status, psi_row0(p, b) + t1 < p.rows_R || t1 >= T_b)) {
             if (t0 < T_b) psi_strip[t0] = p0;
             if (t1 < T_b) psi_strip[t1] = p1;
           }
@@ -618,6 +620,7 @@ int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, in
 extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, int lists,
                                int log_transform, float* logits, int n_max, int32_t* n_units_out,
                                void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_score_evict");
   using namespace ngc;
   if (!valid_cache(c)) return NGC_ERR_INVALID_ARG;
   const PagedView none = {nullptr, 0, 0, NGC_LISTS_SHARED};
@@ -628,6 +631,7 @@ extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, 
 extern "C" int ngc_score_evict_paged(const ngc_paged_cache* pc, const void* q_recent, int w, int log_transform,
                                      float* logits, int n_max, int32_t* n_units_out, void* ws, size_t ws_bytes,
                                      int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_score_evict_paged");
   using namespace ngc;
   if (!pc || !pc->k || !pc->page_table || !pc->lens || pc->L <= 0 || pc->B <= 0 || pc->Hq <= 0 || pc->Hkv <= 0 ||
       pc->Hq % pc->Hkv != 0 || pc->pages_cap <= 0 || (pc->page != 32 && pc->page != 64) || pc->lists < 0 || pc->lists > 2)

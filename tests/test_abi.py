@@ -128,3 +128,17 @@ def test_added_entry_points_refuse_bad_arguments(ngc):
     assert lib.ngc_replay_attn(C.byref(bf), 16, 8, None, None, None, 2, 4, 0, 1.0, 16, 0, None, None) == -1   # rounds without lists
     assert lib.ngc_replay_attn(C.byref(bf), None, 8, None, None, None, 0, 0, 0, 1.0, 16, 0, None, None) == -1
     assert ngc.lib.ngc_workspace_bytes(ngc.OP_SCORE_BACKWARD, C.byref(bf), 1, 0, 0) > 0
+
+
+def test_bounds_checking_and_nvtx_builds_load_and_export_everything(ngc):
+    """The two optional builds (kernels that check their indices; an NVTX range around every call) are separate
+    libraries with the same C ABI."""
+    from paper_2604_18002_b200 import build
+    for kw in (dict(debug=True), dict(nvtx=True)):
+        path = build.build(**kw)
+        assert path != ngc.LIB_PATH and os.path.exists(path)
+        lib = C.CDLL(path)
+        for s in declared_symbols():
+            assert hasattr(lib, s), f"{s} missing from {os.path.basename(path)}"
+        lib.ngc_version.restype = C.c_int
+        assert lib.ngc_version() == ngc.version()

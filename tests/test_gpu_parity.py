@@ -589,3 +589,23 @@ def test_decode_on_a_second_device_after_the_first():
             assert int(st.item()) == 0
             outs.append((out.cpu(), lg.cpu()))
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """The kernels wait for their TMA data with a time limit.  A wait that nothing ever completes (an mbarrier no one
+    arrives on, limit 2 ms) must end in NGC_DEV_TIMEOUT with a normal return, and the context must stay usable."""
+    b = ngc()
+    st = b.new_status()
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    b.ngc_selftest_bounded_wait(2000, st, waited)
+    torch.cuda.synchronize()
+    assert status_value(st) == 6                      # NGC_DEV_TIMEOUT
+    assert 2_000_000 <= int(waited.item()) < 200_000_000
+    # the device still works: an ordinary call behind it
+    c = synth.make_cache(1, 1, 4, 4, 64, torch.float32, [9], capacity=9, seed=1)
+    q = synth.make_queries(1, 1, 4, 64, torch.float32, seed=2)
+    dc, got, st2 = run_decode(c, q)
+    _, _, _, ref, rc = oracle_decode(c, q)
+    assert st2 == 0 and rc == 0 and np.max(np.abs(got - ref)) <= TOL_ATTN_F32
+    with pytest.raises(b.NgcError):
+        b.ngc_selftest_bounded_wait(10_000_000, st)   # limits beyond 100 ms are refused
