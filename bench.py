@@ -654,7 +654,8 @@ def run_kernel(args):
         dc = ngc.NgcCache(c.k, c.v, c.seq_off, c.lens, Hq, T)
         q = synth.normal((L, B, Hq, T, d), 1, torch.bfloat16, device=dev)
         out = torch.empty((L, B, Hq, T, d), dtype=torch.bfloat16, device=dev)
-        ms = best_of(lambda: ngc.ngc_replay_attn(dc, q, out, pos, cnt, total_before, lists=ngc.LISTS_PER_LAYER, status=st), args.steps)
+        ms = best_of(lambda: ngc.ngc_replay_attn(dc, q, out, pos, cnt, total_before, lists=ngc.LISTS_PER_LAYER, status=st,
+                                                 variant=args.variant), args.steps)
         vis = sum(t + 1 for t in range(alive)) + sum(sum(K + s + 1 for s in range(min(delta, T - (alive + (r - 1) * delta)))) for r in range(1, R + 1))
         flops = 4.0 * d * vis * Hq * L * B
         tf_peak = 1590.0
@@ -662,7 +663,8 @@ def run_kernel(args):
         if os.path.exists(pk):
             with open(pk) as f:
                 tf_peak = float(json.load(f)["bf16_tflops"])
-        res = {"kernel": "ngc_replay_attn", "workload": f"config-5 history: {L} layers, B={B}, T={T}, {R} rounds, {K} kept per round and layer",
+        res = {"kernel": "ngc_replay_attn", "path": {None: "default (tcgen05)", 0: "default (tcgen05)", 1: "mma.sync", 2: "tcgen05"}[args.variant],
+               "workload": f"config-5 history: {L} layers, B={B}, T={T}, {R} rounds, {K} kept per round and layer",
                "ms": round(ms, 3),
                "roofline": {"bound": "tensor", "achieved": round(flops / ms / 1e9, 1), "peak": tf_peak, "unit": "TFLOP/s",
                             "frac": round(flops / ms / 1e9 / tf_peak, 4), "flops": "4*d per visible key per query per head (masked keys not counted)"}}
@@ -778,6 +780,8 @@ def main():
     ap.add_argument("--kernel", default=None, choices=["score_backward", "replay_attn"],
                     help="time one training-side call instead of the benchmark step (one GPU)")
     ap.add_argument("--layers", type=int, default=4, help="--kernel replay_attn: layers of the history to run")
+    ap.add_argument("--variant", type=int, default=None, choices=[0, 1, 2],
+                    help="--kernel replay_attn: device path (1 = the warp-level MMA kernel, 2 = tcgen05; default: what the library picks)")
     ap.add_argument("--graph", action="store_true", help="--config 1|3..7: replay the decode calls of a round as one CUDA graph")
     ap.add_argument("--paged", action="store_true", help="--config 6|7 only: paged cache, one eviction unit = one page")
     ap.add_argument("--ring", type=int, default=8, help="distinct decode-input steps kept on the device for --config 3|4|5")

@@ -273,12 +273,23 @@ int ngc_replay_visibility(const int32_t* kept_sorted, const int32_t* budget, con
  *   lists        how G maps to (layer, KV head), as everywhere
  *   out          [L][B][Hq][t_max][d] fp32 or bf16; rows >= lens[b] are not written
  * fp32 scores, softmax and accumulation; probabilities rounded to bf16 for P*V.
- * Needs no workspace.
+ * Needs no workspace.  Runs on the tcgen05 tensor cores with accumulators in
+ * tensor memory; every wait inside is bounded (NGC_DEV_TIMEOUT).
  */
 int ngc_replay_attn(const ngc_cache* c, const void* q, int t_max,
                     const int32_t* alive_pos, const int32_t* alive_count, const int32_t* total_before,
                     int n_rounds, int kt_max, int lists, float scale, void* out, int out_dtype,
                     int32_t* dev_status, ngc_stream stream);
+
+/* ngc_replay_attn with the device path chosen by the caller (same arguments, same contract; for
+ * measuring one path against the other).  AUTO is what ngc_replay_attn runs: the tcgen05 kernel
+ * (S and O accumulators in tensor memory, one CTA per 128 query tokens of two heads).  MMA_SYNC is
+ * the earlier warp-level kernel (64 query tokens of one head per CTA). */
+typedef enum { NGC_REPLAY_ATTN_AUTO = 0, NGC_REPLAY_ATTN_MMA_SYNC = 1, NGC_REPLAY_ATTN_TCGEN05 = 2 } ngc_replay_attn_path;
+int ngc_replay_attn_variant(const ngc_cache* c, const void* q, int t_max,
+                            const int32_t* alive_pos, const int32_t* alive_count, const int32_t* total_before,
+                            int n_rounds, int kt_max, int lists, float scale, void* out, int out_dtype, int variant,
+                            int32_t* dev_status, ngc_stream stream);
 
 /*
  * Physical eviction -- Section 4.1 (entries that are not kept are gone for good).  In place:

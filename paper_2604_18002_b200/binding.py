@@ -27,7 +27,7 @@ DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "
 
 EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
            "ngc_sample_evict", "ngc_evict_logprob", "ngc_evict_logprob_backward", "ngc_compact_kv", "ngc_decode_attn_ragged",
-           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged", "ngc_replay_visibility", "ngc_score_evict_backward", "ngc_replay_attn", "ngc_selftest_bounded_wait"]
+           "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged", "ngc_replay_visibility", "ngc_score_evict_backward", "ngc_replay_attn", "ngc_replay_attn_variant", "ngc_selftest_bounded_wait"]
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -85,6 +85,8 @@ def _load(path: str = LIB_PATH):
     lib.ngc_score_evict_backward.argtypes = [C.POINTER(CacheDesc), vp, i32, i32, i32, i32, vp, vp, i32, vp, vp, vp, sz, vp, vp]
     lib.ngc_replay_attn.restype = i32
     lib.ngc_replay_attn.argtypes = [C.POINTER(CacheDesc), vp, i32, vp, vp, vp, i32, i32, i32, C.c_float, vp, i32, vp, vp]
+    lib.ngc_replay_attn_variant.restype = i32
+    lib.ngc_replay_attn_variant.argtypes = [C.POINTER(CacheDesc), vp, i32, vp, vp, vp, i32, i32, i32, C.c_float, vp, i32, i32, vp, vp]
     lib.ngc_replay_visibility.restype = i32
     lib.ngc_replay_visibility.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.ngc_selftest_bounded_wait.restype = i32
@@ -383,18 +385,27 @@ def ngc_score_evict_backward(cache: NgcCache, q_recent: torch.Tensor, block: int
     _check(rc, "ngc_score_evict_backward")
 
 
+REPLAY_ATTN_AUTO, REPLAY_ATTN_MMA_SYNC, REPLAY_ATTN_TCGEN05 = 0, 1, 2
+
+
 def ngc_replay_attn(cache: NgcCache, q: torch.Tensor, out: torch.Tensor, alive_pos: Optional[torch.Tensor] = None,
                     alive_count: Optional[torch.Tensor] = None, total_before: Optional[torch.Tensor] = None,
-                    lists: int = LISTS_SHARED, scale: Optional[float] = None, status: Optional[torch.Tensor] = None):
-    """q, out [L][B][Hq][t_max][d]; cache holds the full sequences (lens = total tokens)."""
+                    lists: int = LISTS_SHARED, scale: Optional[float] = None, status: Optional[torch.Tensor] = None,
+                    variant: Optional[int] = None):
+    """q, out [L][B][Hq][t_max][d]; cache holds the full sequences (lens = total tokens).  ``variant`` picks the device
+    path (REPLAY_ATTN_*) through ngc_replay_attn_variant; None calls ngc_replay_attn itself."""
     t_max = q.shape[3]
     if scale is None:
         scale = 1.0 / (cache.d ** 0.5)
     n_rounds = 0 if alive_pos is None else alive_pos.shape[0]
     kt_max = 0 if alive_pos is None else alive_pos.shape[3]
     d = cache.desc()
-    rc = lib.ngc_replay_attn(C.byref(d), _ptr(q), t_max, _ptr(alive_pos), _ptr(alive_count), _ptr(total_before), n_rounds, kt_max,
-                             lists, scale, _ptr(out), _dtype_code(out), _ptr(status), _stream())
+    if variant is None:
+        rc = lib.ngc_replay_attn(C.byref(d), _ptr(q), t_max, _ptr(alive_pos), _ptr(alive_count), _ptr(total_before), n_rounds, kt_max,
+                                 lists, scale, _ptr(out), _dtype_code(out), _ptr(status), _stream())
+    else:
+        rc = lib.ngc_replay_attn_variant(C.byref(d), _ptr(q), t_max, _ptr(alive_pos), _ptr(alive_count), _ptr(total_before), n_rounds,
+                                         kt_max, lists, scale, _ptr(out), _dtype_code(out), variant, _ptr(status), _stream())
     _check(rc, "ngc_replay_attn")
 
 

@@ -1,5 +1,6 @@
-// ngc_replay_attn: attention of EVERY token of a rollout under its replay mask (paper Section 4.5
-// and Appendix A.3): one pass over the full, uncompacted sequence in which the query at position t
+// ngc_replay_attn, warp-level MMA path (kept as the comparison arm of the tcgen05 kernel in
+// replay_attn_umma.cu, which is what ngc_replay_attn runs): attention of EVERY token of a rollout
+// under its replay mask (paper Section 4.5 and Appendix A.3): one pass over the full, uncompacted sequence in which the query at position t
 // sees what it saw at generation time -- the entries the last eviction round before t left alive
 // (kept_r, a list of original positions from ngc_replay_visibility) plus, causally, the tokens
 // generated since that round.  The paper feeds dense B x T x T masks to a stock attention; here the
@@ -16,6 +17,7 @@
 
 #include "ngc_common.cuh"
 #include "ptx.cuh"
+#include "replay_attn.cuh"
 
 namespace ngc {
 namespace {
@@ -28,22 +30,6 @@ constexpr int kBoxBytes = kKTile * 128;       // 64 rows x 64 channels of bf16
 constexpr int kTileBytes = 2 * kBoxBytes;     // K (or V) tile
 constexpr int kStageBytes = 2 * kTileBytes;   // K + V
 constexpr int kMaxSeg = 66;                   // rounds one query tile can straddle (+ the contiguous part)
-
-struct ReplayAttnParams {
-  const __nv_bfloat16* k;        // [L][Hkv][R][128]: every token of every sequence, original order
-  const __nv_bfloat16* v;
-  const int64_t* seq_off;
-  const int32_t* lens;           // T_b
-  const __nv_bfloat16* q;        // [L][B][Hq][t_max][128]
-  const int32_t* alive_pos;      // [n_rounds][B][G][kt_max]
-  const int32_t* alive_count;    // [n_rounds][B][G]
-  const int32_t* total_before;   // [n_rounds][B]
-  void* out;                     // [L][B][Hq][t_max][128]
-  int32_t* dev_status;
-  int64_t rows_R;
-  int L, B, Hq, Hkv, g, t_max, n_rounds, G, kt_max, lists, out_bf16, q_tiles;
-  float scale_log2;
-};
 
 // swizzled byte offset of 16-byte piece c (0..15) of row r inside a K or V tile
 __device__ __forceinline__ uint32_t tile_off(int r, int c) {
@@ -291,13 +277,14 @@ __global__ void __launch_bounds__(kThreads, 3) replay_attn_kernel(ReplayAttnPara
 }  // namespace
 }  // namespace ngc
 
-extern "C" int ngc_replay_attn(const ngc_cache* c, const void* q, int t_max,
-                               const int32_t* alive_pos, const int32_t* alive_count, const int32_t* total_before,
-                               int n_rounds, int kt_max, int lists, float scale, void* out, int out_dtype,
-                               int32_t* dev_status, ngc_stream stream) {
-  NGC_API_RANGE("ngc_replay_attn");
-  using namespace ngc;
-  if (!valid_cache(c) || !q || !out || t_max <= 0 || n_rounds < 0 || lists < 0 || lists > 2 ||
+namespace ngc {
+namespace {
+
+int replay_attn_impl(const ngc_cache* c, const void* q, int t_max,
+                     const int32_t* alive_pos, const int32_t* alive_count, const int32_t* total_before,
+                     int n_rounds, int kt_max, int lists, float scale, void* out, int out_dtype, int variant,
+                     int32_t* dev_status, cudaStream_t stream) {
+  if (!valid_cache(c) || !q || !out || t_max <= 0 || n_rounds < 0 || lists < 0 || lists > 2 || variant < 0 || variant > 2 ||
       (n_rounds > 0 && (!alive_pos || !alive_count || !total_before || kt_max <= 0)))
     return NGC_ERR_INVALID_ARG;
   if (out_dtype != NGC_F32 && out_dtype != NGC_BF16) return NGC_ERR_INVALID_ARG;
@@ -313,10 +300,32 @@ extern "C" int ngc_replay_attn(const ngc_cache* c, const void* q, int t_max,
   p.G = lists_G(lists, c->L, c->Hkv); p.kt_max = kt_max; p.lists = lists; p.out_bf16 = out_dtype == NGC_BF16;
   p.q_tiles = (t_max + kQTile - 1) / kQTile;
   p.scale_log2 = scale * 1.4426950408889634f;
+  if (variant != NGC_REPLAY_ATTN_MMA_SYNC) return launch_replay_attn_umma(p, stream);
   const int64_t ctas = (int64_t)c->L * c->B * c->Hq * p.q_tiles;
   if (ctas > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
   const int smem = 2 * kStageBytes + 1024;
   NGC_CUDA_TRY(cudaFuncSetAttribute(replay_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  replay_attn_kernel<<<(unsigned)ctas, kThreads, smem, (cudaStream_t)stream>>>(p);
+  replay_attn_kernel<<<(unsigned)ctas, kThreads, smem, stream>>>(p);
   return launch_status();
+}
+
+}  // namespace
+}  // namespace ngc
+
+extern "C" int ngc_replay_attn(const ngc_cache* c, const void* q, int t_max,
+                               const int32_t* alive_pos, const int32_t* alive_count, const int32_t* total_before,
+                               int n_rounds, int kt_max, int lists, float scale, void* out, int out_dtype,
+                               int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_replay_attn");
+  return ngc::replay_attn_impl(c, q, t_max, alive_pos, alive_count, total_before, n_rounds, kt_max, lists, scale, out, out_dtype,
+                               NGC_REPLAY_ATTN_AUTO, dev_status, (cudaStream_t)stream);
+}
+
+extern "C" int ngc_replay_attn_variant(const ngc_cache* c, const void* q, int t_max,
+                                       const int32_t* alive_pos, const int32_t* alive_count, const int32_t* total_before,
+                                       int n_rounds, int kt_max, int lists, float scale, void* out, int out_dtype, int variant,
+                                       int32_t* dev_status, ngc_stream stream) {
+  NGC_API_RANGE("ngc_replay_attn_variant");
+  return ngc::replay_attn_impl(c, q, t_max, alive_pos, alive_count, total_before, n_rounds, kt_max, lists, scale, out, out_dtype,
+                               variant, dev_status, (cudaStream_t)stream);
 }

@@ -1,0 +1,447 @@
+// ngc_replay_attn on the 5th-generation tensor cores (paper Section 4.5 replay pass, Appendix A.3 masks).
+//
+// The replay pass is the one compute-bound contraction of this library: every token of a rollout
+// attends to the kept list of the last eviction round before it plus, causally, its own block.
+// One CTA takes 128 query tokens of TWO query heads that share a KV head; the 128 rows of a head are
+// the 128 lanes of tensor memory.
+//
+//   producer warps (2)   gather 64-key K/V tiles by position (kept lists, then the contiguous block)
+//                        with 16-byte cp.async into a 4-stage ring, 128-byte swizzled, and publish a
+//                        stage with a proxy fence + mbarrier arrival once its copies have landed.  Tile
+//                        i - 1 is published right after tile i has been issued, BEFORE the producer may
+//                        block on a free stage: the MMA warp needs tile i + 1 to finish tile i, so a
+//                        producer that sat on landed tiles while waiting for a stage would deadlock;
+//   MMA warp (1 thread)  S_h = Q_h K^T (tcgen05.mma, M = 128, N = 64, both operands K-major) into a
+//                        double-buffered S in tensor memory, and O_h += P_h V (M = 128, N = 128, V as
+//                        MN-major B operand); completion is committed to mbarriers;
+//   softmax warps (2x4)  one warpgroup per head, one thread per query row: S row from tensor memory
+//                        (tcgen05.ld), replay mask, online softmax in the log2 domain, P row as bf16
+//                        into 128-byte-swizzled shared memory for the second product.  The running
+//                        maximum used for the exponentials only moves when the true maximum has grown
+//                        by more than 8 (a factor 256, exact in bf16 / fp32), so the O accumulator in
+//                        tensor memory is rescaled rarely; when it is, the row's owner does it in place
+//                        (tcgen05.ld / st) after the previous P V product has completed.
+//
+// The S product of tile i+1 is issued before the P V product of tile i, so the tensor pipe works on
+// one head while the other head's rows are in the softmax.  Every wait is bounded: a wait that runs
+// out raises a CTA-wide abort flag, every role leaves its loop, in-flight copies and MMAs are
+// drained (bounded again), tensor memory is freed and NGC_DEV_TIMEOUT is reported.
+#include <cuda_bf16.h>
+
+#include "ngc_common.cuh"
+#include "ptx.cuh"
+#include "replay_attn.cuh"
+#include "umma.cuh"
+
+namespace ngc {
+namespace {
+
+constexpr int kQRows = 128;                   // query tokens per CTA = tensor-memory lanes
+constexpr int kKeys = 64;                     // keys per pipeline stage
+constexpr int kStages = 4;
+constexpr int kSoftmaxWarps = 8;              // two groups of four, one query head each
+constexpr int kMmaWarp = 8;
+constexpr int kProducerWarp0 = 9;
+constexpr int kProducerLanes = 64;
+constexpr int kThreads = kProducerWarp0 * 32 + kProducerLanes;     // 352
+constexpr int kQHalf = kQRows * 128;          // one 64-channel half of a Q tile (128 rows x 128 B)
+constexpr int kQBytes = 2 * kQHalf;           // 32 KB per head
+constexpr int kKBox = kKeys * 128;            // 64 keys x 64 channels
+constexpr int kKTile = 2 * kKBox;             // K (or V) tile, 16 KB
+constexpr int kStageBytes = 2 * kKTile;       // K + V
+constexpr int kPBytes = kQRows * 128;         // P tile of a head: 128 rows x 64 keys of bf16
+constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 2 * kPBytes + 1024;
+constexpr uint32_t kTmemCols = 512;           // S[h][buf] at (2h + buf) * 64, O[h] at 256 + 128 h
+constexpr int kMaxSeg = 66;                   // rounds one query tile can straddle (+ the contiguous part)
+constexpr float kLazyRescale = 8.f;           // log2 units the row maximum may grow before O is rescaled
+
+struct Shared {
+  uint64_t kv_full[kStages], kv_empty[kStages], s_full[2][2], p_full[2], o_done[2], drain;
+  uint32_t tmem;
+  int abort;
+  int seg_rho[kMaxSeg], seg_n[kMaxSeg], seg_first[kMaxSeg + 1];
+  int nseg, c_lo, uniform;
+};
+
+// Bounded wait that also gives up as soon as another thread of the CTA has given up.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Shared* sh, int32_t* dev_status) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = ptx::globaltimer_ns();
+  for (uint32_t spins = 0;; ++spins) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((spins & 63u) == 63u) {
+      if (*(volatile int*)&sh->abort) return false;
+      if (ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs) {
+        *(volatile int*)&sh->abort = 1;
+        set_dev_status(dev_status, NGC_DEV_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+// swizzled byte offset of 16-byte piece c (0..15) of row r inside a tile of `half_bytes`-sized 64-channel halves
+__device__ __forceinline__ uint32_t tile_off(int half_bytes, int r, int c) {
+  return (uint32_t)((c >> 3) * half_bytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAttnParams p) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ Shared sh;
+
+  uint8_t* base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = base;                                   // [2 heads][32 KB]
+  uint8_t* stage = sQ + 2 * kQBytes;                    // [kStages][K 16 KB | V 16 KB]
+  uint8_t* sP = stage + kStages * kStageBytes;          // [2 heads][16 KB]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  const int pairs = (p.g + 1) >> 1;
+  int item = blockIdx.x;
+  const int m = item % p.q_tiles; item /= p.q_tiles;
+  const int pair = item % pairs; item /= pairs;
+  const int h = item % p.Hkv; item /= p.Hkv;
+  const int b = item % p.B;
+  const int l = item / p.B;
+  const int T_b = min(p.lens[b], p.t_max);
+  const int q0 = m * kQRows;
+  if (q0 >= T_b) return;                                // nothing allocated yet
+  const int hq0 = h * p.g + 2 * pair;
+  const bool has1 = 2 * pair + 1 < p.g;                 // an odd group leaves the last pair half empty
+  const int gi = list_of(p.lists, l, h, p.Hkv);
+  const int q_last = min(q0 + kQRows - 1, T_b - 1);
+
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&sh.kv_full[s], kProducerLanes); ptx::mbar_init(&sh.kv_empty[s], 1); }
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      ptx::mbar_init(&sh.s_full[hh][0], 1); ptx::mbar_init(&sh.s_full[hh][1], 1);
+      ptx::mbar_init(&sh.p_full[hh], 128); ptx::mbar_init(&sh.o_done[hh], 1);
+    }
+    ptx::mbar_init(&sh.drain, 1);
+    ptx::fence_barrier_init();
+    sh.abort = 0;
+    // key sources of this query tile: the kept lists of the rounds it straddles, then the contiguous run
+    int r_lo = 0, r_hi = 0;                             // rounds fired before the first / last query of the tile
+    for (int r = 0; r < p.n_rounds; ++r) {
+      const int tb = p.total_before[r * p.B + b];
+      r_lo += tb <= q0;
+      r_hi += tb <= q_last;
+    }
+    int nseg = 0, first = 0;
+    for (int rho = max(r_lo, 1); rho <= r_hi; ++rho) {
+      if (nseg >= kMaxSeg - 1) { set_dev_status(p.dev_status, NGC_DEV_BAD_COUNTS); break; }
+      int n = p.alive_count[((int64_t)(rho - 1) * p.B + b) * p.G + gi];
+      if (n < 0 || n > p.kt_max) { set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); n = 0; }
+      if (n > 0) {
+        sh.seg_rho[nseg] = rho; sh.seg_n[nseg] = n; sh.seg_first[nseg] = first;
+        first += (n + kKeys - 1) / kKeys;
+        ++nseg;
+      }
+    }
+    const int c_lo = r_lo >= 1 ? p.total_before[(r_lo - 1) * p.B + b] : 0;
+    sh.c_lo = c_lo;
+    sh.seg_rho[nseg] = -1; sh.seg_n[nseg] = q_last - c_lo + 1; sh.seg_first[nseg] = first;
+    first += (q_last - c_lo + kKeys) / kKeys;
+    ++nseg;
+    sh.seg_first[nseg] = first;
+    sh.nseg = nseg;
+    sh.uniform = r_lo == r_hi;                          // every query of the tile lies in the same block
+  }
+  if (warp == kMmaWarp) umma::tmem_alloc(&sh.tmem, kTmemCols);
+
+  // Q tiles of the two heads -> shared memory (rows beyond the sequence: zeros)
+  {
+    const int n_heads = has1 ? 2 : 1;
+    for (int i = tid; i < n_heads * kQRows * 16; i += kThreads) {
+      const int hh = i / (kQRows * 16), rest = i - hh * kQRows * 16;
+      const int r = rest >> 4, c = rest & 15;
+      uint8_t* dst = sQ + hh * kQBytes + tile_off(kQHalf, r, c);
+      const int t = q0 + r;
+      if (t < T_b) {
+        const __nv_bfloat16* src = p.q + ((((int64_t)l * p.B + b) * p.Hq + hq0 + hh) * (int64_t)p.t_max + t) * 128 + 8 * c;
+        ptx::cp_async_cg_16(ptx::smem_u32(dst), src);
+      } else {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    ptx::cp_async_commit();
+    ptx::cp_async_wait_group<0>();
+    ptx::fence_proxy_async();
+  }
+  umma::fence_before_sync();
+  __syncthreads();
+  umma::fence_after_sync();
+  const uint32_t tmem = sh.tmem;
+  const int nseg = sh.nseg, c_lo = sh.c_lo, n_tiles = sh.seg_first[nseg];
+  const bool uniform = sh.uniform != 0;
+
+  if (warp >= kProducerWarp0) {
+    // ------------------------------------------------------------------ producers
+    const int ptid = tid - kProducerWarp0 * 32;
+    const __nv_bfloat16* k_strip = p.k + ((int64_t)(l * p.Hkv + h) * p.rows_R + p.seq_off[b]) * 128;
+    const __nv_bfloat16* v_strip = p.v + ((int64_t)(l * p.Hkv + h) * p.rows_R + p.seq_off[b]) * 128;
+    int issued = 0, published = 0, sgi = 0;
+    auto publish = [&](int t) {                         // this lane's copies of tile t have landed
+      ptx::fence_proxy_async();
+      ptx::mbar_arrive(&sh.kv_full[t % kStages]);
+    };
+    for (int i = 0; i < n_tiles; ++i) {
+      const int s = i % kStages;
+      if (i >= kStages) {
+        const bool ok = wait_or_abort(&sh.kv_empty[s], ((i / kStages) - 1) & 1, &sh, p.dev_status);
+        if (!__all_sync(0xffffffffu, ok)) break;
+      }
+      while (sgi + 1 < nseg && i >= sh.seg_first[sgi + 1]) ++sgi;
+      const int rho = sh.seg_rho[sgi], n = sh.seg_n[sgi], kt = i - sh.seg_first[sgi];
+      const int32_t* list = rho >= 1 ? p.alive_pos + (((int64_t)(rho - 1) * p.B + b) * p.G + gi) * p.kt_max : nullptr;
+      uint8_t* st = stage + s * kStageBytes;
+#pragma unroll 4
+      for (int u = 0; u < 16; ++u) {
+        const int slot = u * kProducerLanes + ptid;
+        const int row = slot >> 4, c = slot & 15;
+        const int kidx = kt * kKeys + row;
+        int pos = -1;
+        if (kidx < n) pos = list ? list[kidx] : c_lo + kidx;
+        const uint32_t off = tile_off(kKBox, row, c);
+        if (pos >= 0 && pos < T_b) {
+          ptx::cp_async_cg_16(ptx::smem_u32(st + off), k_strip + (int64_t)pos * 128 + 8 * c);
+          ptx::cp_async_cg_16(ptx::smem_u32(st + kKTile + off), v_strip + (int64_t)pos * 128 + 8 * c);
+        } else {      // past the end of the source: zeros (a stale NaN times P = 0 would poison the sum)
+          if (kidx < n && c == 0) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
+          *reinterpret_cast<uint4*>(st + off) = make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(st + kKTile + off) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      ptx::cp_async_commit();
+      ++issued;
+      if (issued - published > 1) {                     // everything but the tile just issued has landed
+        ptx::cp_async_wait_group<1>();
+        publish(published++);
+      }
+    }
+    ptx::cp_async_wait_group<0>();
+    if (issued - published == 1) publish(published++);
+  } else if (warp == kMmaWarp) {
+    // ------------------------------------------------------------------ MMA issue (one thread)
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = umma::instr_desc(kQRows, kKeys, false);
+      constexpr uint32_t idesc_o = umma::instr_desc(kQRows, 128, true);
+      const uint32_t q_addr = ptx::smem_u32(sQ), p_addr = ptx::smem_u32(sP), st_addr = ptx::smem_u32(stage);
+      const int n_heads = has1 ? 2 : 1;
+      auto issue_s = [&](int i) {                       // S_h(i) = Q_h K(i)^T into buffer i & 1
+        const uint32_t k_addr = st_addr + (i % kStages) * kStageBytes;
+        for (int hh = 0; hh < n_heads; ++hh) {
+          const uint32_t d = tmem + (uint32_t)((2 * hh + (i & 1)) * kKeys);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t a = umma::smem_desc_sw128(q_addr + hh * kQBytes + (ks >> 2) * kQHalf + (ks & 3) * 32, 16, 1024);
+            const uint64_t bd = umma::smem_desc_sw128(k_addr + (ks >> 2) * kKBox + (ks & 3) * 32, 16, 1024);
+            umma::mma_bf16(d, a, bd, idesc_s, ks > 0);
+          }
+          umma::commit(&sh.s_full[hh][i & 1]);
+        }
+      };
+      bool ok = wait_or_abort(&sh.kv_full[0], 0, &sh, p.dev_status);
+      if (ok) {
+        umma::fence_after_sync();
+        issue_s(0);
+      }
+      for (int i = 0; ok && i < n_tiles; ++i) {
+        if (i + 1 < n_tiles) {
+          ok = wait_or_abort(&sh.kv_full[(i + 1) % kStages], ((i + 1) / kStages) & 1, &sh, p.dev_status);
+          if (!ok) break;
+          umma::fence_after_sync();
+          issue_s(i + 1);                               // its S buffer was read out before P(i - 1) was published
+        }
+        const uint32_t v_addr = st_addr + (i % kStages) * kStageBytes + kKTile;
+        for (int hh = 0; hh < n_heads; ++hh) {
+          ok = wait_or_abort(&sh.p_full[hh], i & 1, &sh, p.dev_status);
+          if (!ok) break;
+          umma::fence_after_sync();
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {              // 16 keys per step
+            const uint64_t a = umma::smem_desc_sw128(p_addr + hh * kPBytes + kk * 32, 16, 1024);
+            const uint64_t bd = umma::smem_desc_sw128(v_addr + kk * 2048, kKBox, 1024);   // next 64 channels: one box on
+            umma::mma_bf16(tmem + 256u + 128u * hh, a, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma::commit(&sh.o_done[hh]);
+        }
+        if (!ok) break;
+        umma::commit(&sh.kv_empty[i % kStages]);        // K and V of this stage have been consumed
+      }
+      // everything issued has completed before tensor memory is released
+      umma::commit(&sh.drain);
+      wait_or_abort(&sh.drain, 0, &sh, p.dev_status);
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ softmax: one thread per query row
+    const int hh = warp >> 2;
+    if (hh == 0 || has1) {
+      const int row = 32 * (warp & 3) + lane;
+      const int t_q = q0 + row;
+      int blk = 0, lo_row = 0;                          // round index of the row's block, its first position
+      for (int r = 0; r < p.n_rounds; ++r) {
+        const int tb = p.total_before[r * p.B + b];
+        if (tb <= t_q) { blk += 1; lo_row = tb; }
+      }
+      const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
+      const uint32_t o_addr = tmem + lane_base + 256u + 128u * hh;
+      uint8_t* p_row = sP + hh * kPBytes + row * 128;
+      float m_use = -INFINITY, l_run = 0.f;
+      int o_seen = -1;                                  // last tile whose P V product is known to be complete
+      int sgi = 0;
+      bool ok = true;
+      for (int i = 0; i < n_tiles; ++i) {
+        ok = wait_or_abort(&sh.s_full[hh][i & 1], (i >> 1) & 1, &sh, p.dev_status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        umma::fence_after_sync();
+        uint32_t zr[2][32];
+        const uint32_t s_addr = tmem + lane_base + (uint32_t)((2 * hh + (i & 1)) * kKeys);
+        umma::tmem_ld32(s_addr, zr[0]);
+        umma::tmem_ld32(s_addr + 32, zr[1]);
+        umma::tmem_ld_wait();
+        while (sgi + 1 < nseg && i >= sh.seg_first[sgi + 1]) ++sgi;
+        const int rho = sh.seg_rho[sgi], kt = i - sh.seg_first[sgi];
+        const int n_here = min(kKeys, sh.seg_n[sgi] - kt * kKeys);
+        // a tile needs no mask when every query of the CTA lies in one block and the tile is a full tile of that
+        // block's kept list, or lies entirely before the first query
+        const bool need_mask = !uniform || (rho >= 1 ? n_here < kKeys : c_lo + kt * kKeys + kKeys - 1 > q0);
+        float mx = -INFINITY;
+        if (need_mask) {
+          const int j0 = c_lo + kt * kKeys;
+#pragma unroll
+          for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int jj = 32 * half + j;
+              bool vis;
+              if (rho >= 1) vis = jj < n_here && blk == rho;                   // a kept entry of the round before this row's block
+              else vis = j0 + jj >= lo_row && j0 + jj <= t_q;                  // a token of the row's own block, causal
+              const float z = vis ? __uint_as_float(zr[half][j]) * p.scale_log2 : -INFINITY;
+              zr[half][j] = __float_as_uint(z);
+              mx = fmaxf(mx, z);
+            }
+        } else {
+#pragma unroll
+          for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float z = __uint_as_float(zr[half][j]) * p.scale_log2;
+              zr[half][j] = __float_as_uint(z);
+              mx = fmaxf(mx, z);
+            }
+        }
+        // the maximum used for the exponentials follows the true one lazily
+        const bool grow = mx > m_use + kLazyRescale;                          // also the first visible key (m_use = -inf)
+        const bool rescale = grow && m_use != -INFINITY && i > 0;             // O already holds something for this row
+        if (__any_sync(0xffffffffu, rescale)) {
+          if (o_seen < i - 1) {
+            ok = wait_or_abort(&sh.o_done[hh], (i - 1) & 1, &sh, p.dev_status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            o_seen = i - 1;
+            umma::fence_after_sync();
+          }
+          const float alpha = rescale ? ptx::ex2_approx(m_use - mx) : 1.f;
+          l_run *= alpha;
+#pragma unroll 1
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t o[32];
+            umma::tmem_ld32(o_addr + c0, o);
+            umma::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+            umma::tmem_st32(o_addr + c0, o);
+          }
+          umma::tmem_st_wait();
+        }
+        if (grow) m_use = mx;
+        const float m_eff = m_use == -INFINITY ? 0.f : m_use;                 // nothing visible yet: every exponential is 0
+        uint32_t pk[32];
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = ptx::ex2_approx(__uint_as_float(zr[half][j]) - m_eff);
+            const float p1 = ptx::ex2_approx(__uint_as_float(zr[half][j + 1]) - m_eff);
+            l_run += p0 + p1;
+            pk[16 * half + (j >> 1)] = ptx::pack_bf16x2(p0, p1);
+          }
+        if (i > 0 && o_seen < i - 1) {                                        // the P tile is free once P V (i - 1) has completed
+          ok = wait_or_abort(&sh.o_done[hh], (i - 1) & 1, &sh, p.dev_status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          o_seen = i - 1;
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          *reinterpret_cast<uint4*>(p_row + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        ptx::fence_proxy_async();
+        umma::fence_before_sync();
+        ptx::mbar_arrive(&sh.p_full[hh]);
+      }
+      if (ok) {
+        ok = wait_or_abort(&sh.o_done[hh], (n_tiles - 1) & 1, &sh, p.dev_status);
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      if (ok) {
+        umma::fence_after_sync();
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+        const int64_t o_base = ((((int64_t)l * p.B + b) * p.Hq + hq0 + hh) * (int64_t)p.t_max + t_q) * 128;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t o[32];
+          umma::tmem_ld32(o_addr + c0, o);
+          umma::tmem_ld_wait();
+          if (t_q < T_b) {
+            if (p.out_bf16) {
+              uint4* dst = reinterpret_cast<uint4*>((__nv_bfloat16*)p.out + o_base + c0);
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                dst[j] = make_uint4(ptx::pack_bf16x2(__uint_as_float(o[8 * j]) * inv, __uint_as_float(o[8 * j + 1]) * inv),
+                                    ptx::pack_bf16x2(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv),
+                                    ptx::pack_bf16x2(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv),
+                                    ptx::pack_bf16x2(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv));
+            } else {
+              float4* dst = reinterpret_cast<float4*>((float*)p.out + o_base + c0);
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                dst[j] = make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
+                                     __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
+            }
+          }
+        }
+      }
+    }
+  }
+  // ---- teardown: every role has left its loop; nothing of this CTA is in flight any more
+  umma::fence_before_sync();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    umma::fence_after_sync();
+    umma::tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+}  // namespace
+
+int launch_replay_attn_umma(const ReplayAttnParams& p, cudaStream_t stream) {
+  const int pairs = (p.g + 1) / 2;
+  ReplayAttnParams q = p;
+  q.q_tiles = (p.t_max + kQRows - 1) / kQRows;
+  const int64_t ctas = (int64_t)p.L * p.B * p.Hkv * pairs * q.q_tiles;
+  if (ctas > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+  static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
+  const int rc = attr_once.run([] {
+    return cudaFuncSetAttribute(replay_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  });
+  if (rc != NGC_OK) return rc;
+  // One CTA per SM by construction (197 KB of shared memory each): a CTA owns all 512 columns of its SM's tensor memory.
+  replay_attn_umma_kernel<<<(unsigned)ctas, kThreads, kSmemBytes, stream>>>(q);
+  return launch_status();
+}
+
+}  // namespace ngc

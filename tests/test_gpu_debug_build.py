@@ -63,7 +63,8 @@ CASES = [
     (t_lens.test_per_list_lengths_through_three_rounds, (1,)),
     (t_replay.test_replay_visibility_matches_oracle, (5, 2, 3, 4, 5, 70)),
     (t_replay.test_replay_visibility_figure_and_failures, ()),
-    (t_rattn.test_replay_attn_matches_oracle, (2, 4, 3, 30, 200)),
+    (t_rattn.test_replay_attn_matches_oracle, (2, 4, 3, 30, 200, None)),
+    (t_rattn.test_replay_attn_matches_oracle, (1, 32, 2, 100, 300, 1)),
     (t_sbwd.test_score_backward_matches_oracle, (12, 2, 5, 1, 32, 0)),
 ]
 
@@ -188,7 +189,7 @@ def test_canaries_survive_score_sample_and_logprob():
     L, B, Hq, Hkv, d, T, w = 2, 3, 12, 2, 128, 600, 5
     lens = [T, 77, 300]
     host, dc, bufs, so = guarded_cache(L, B, Hq, Hkv, d, lens, [T + 2] * B, seed=33)
-    G, n_max, k_max = L, T, T // 2
+    G, n_max, k_max = L, T + 2, T // 2                      # n_max covers the row capacity
     logits, lg_whole, lg_fill = guarded((B, G, n_max), torch.float32)
     qr = synth.normal((L, B, Hq, w, d), 34, bf16).cuda()
     st = b.new_status()
@@ -226,7 +227,7 @@ def test_canaries_survive_paged_eviction():
     table, table_whole, t_fill = guarded((B, G, pages_cap), torch.int32)
     table.copy_(pc.page_table)
     pc.page_table = table
-    k0, v0 = pc.k.clone(), pc.v.clone()
+    k0, v0 = pc.k.view(torch.int16).clone(), pc.v.view(torch.int16).clone()    # bit patterns: the free pages hold junk, NaNs included
     units = [(l + page - 1) // page for l in lens]
     budget = np.array([max(1, u // 2) for u in units], np.int32)
     logits = synth.make_logits(B, G, pages_cap, seed=37).numpy()
@@ -236,7 +237,7 @@ def test_canaries_survive_paged_eviction():
     b.ngc_evict_pages(pc, torch.as_tensor(ks).cuda(), torch.as_tensor(budget).cuda(), status=st)
     torch.cuda.synchronize()
     assert status_value(st) == 0
-    assert torch.equal(pc.k, k0) and torch.equal(pc.v, v0)                  # eviction on a paged cache moves no K/V row
+    assert torch.equal(pc.k.view(torch.int16), k0) and torch.equal(pc.v.view(torch.int16), v0)   # eviction on a paged cache moves no K/V row
     assert bool((table_whole[table.numel():] == t_fill).all())
     rows = table.cpu().numpy()
     assert np.all(np.sort(rows, -1) == np.arange(pages_cap))               # every row is still a permutation of the pool
