@@ -56,11 +56,12 @@ constexpr int kMaxSeg = 66;                   // rounds one query tile can strad
 constexpr float kLazyRescale = 8.f;           // log2 units the row maximum may grow before O is rescaled
 
 struct Shared {
-  uint64_t kv_full[kStages], kv_empty[kStages], s_full[2][2], p_full[2], o_done[2], drain;
+  uint64_t kv_full[kStages], kv_empty[kStages], s_full[2][2], p_full[2], o_done[2], q_full, drain;
   uint32_t tmem;
   int abort;
   int seg_rho[kMaxSeg], seg_n[kMaxSeg], seg_first[kMaxSeg + 1];
-  int nseg, c_lo, uniform;
+  int tb[kMaxSeg];              // sequence length at the rounds r_lo .. r_hi - 1 (those that fire inside the query tile)
+  int nseg, c_lo, uniform, r_lo, r_hi;
 };
 
 // Bounded wait that also gives up as soon as another thread of the CTA has given up.
@@ -110,6 +111,7 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
   const int gi = list_of(p.lists, l, h, p.Hkv);
   const int q_last = min(q0 + kQRows - 1, T_b - 1);
 
+  constexpr int kQLoaders = kProducerWarp0 * 32;        // the softmax warps and the MMA warp bring Q in
   if (tid == 0) {
 #pragma unroll
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&sh.kv_full[s], kProducerLanes); ptx::mbar_init(&sh.kv_empty[s], 1); }
@@ -118,42 +120,74 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
       ptx::mbar_init(&sh.s_full[hh][0], 1); ptx::mbar_init(&sh.s_full[hh][1], 1);
       ptx::mbar_init(&sh.p_full[hh], 128); ptx::mbar_init(&sh.o_done[hh], 1);
     }
+    ptx::mbar_init(&sh.q_full, kQLoaders);
     ptx::mbar_init(&sh.drain, 1);
     ptx::fence_barrier_init();
     sh.abort = 0;
-    // key sources of this query tile: the kept lists of the rounds it straddles, then the contiguous run
-    int r_lo = 0, r_hi = 0;                             // rounds fired before the first / last query of the tile
-    for (int r = 0; r < p.n_rounds; ++r) {
-      const int tb = p.total_before[r * p.B + b];
-      r_lo += tb <= q0;
-      r_hi += tb <= q_last;
-    }
-    int nseg = 0, first = 0;
-    for (int rho = max(r_lo, 1); rho <= r_hi; ++rho) {
-      if (nseg >= kMaxSeg - 1) { set_dev_status(p.dev_status, NGC_DEV_BAD_COUNTS); break; }
-      int n = p.alive_count[((int64_t)(rho - 1) * p.B + b) * p.G + gi];
-      if (n < 0 || n > p.kt_max) { set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); n = 0; }
-      if (n > 0) {
-        sh.seg_rho[nseg] = rho; sh.seg_n[nseg] = n; sh.seg_first[nseg] = first;
-        first += (n + kKeys - 1) / kKeys;
-        ++nseg;
-      }
-    }
-    const int c_lo = r_lo >= 1 ? p.total_before[(r_lo - 1) * p.B + b] : 0;
-    sh.c_lo = c_lo;
-    sh.seg_rho[nseg] = -1; sh.seg_n[nseg] = q_last - c_lo + 1; sh.seg_first[nseg] = first;
-    first += (q_last - c_lo + kKeys) / kKeys;
-    ++nseg;
-    sh.seg_first[nseg] = first;
-    sh.nseg = nseg;
-    sh.uniform = r_lo == r_hi;                          // every query of the tile lies in the same block
   }
   if (warp == kMmaWarp) umma::tmem_alloc(&sh.tmem, kTmemCols);
+  if (warp == 0) {
+    // key sources of this query tile: the kept lists of the rounds it straddles, then the contiguous run.
+    // Rounds fired before the first / last query of the tile: counted by the whole warp (independent loads).
+    int n_lo = 0, n_hi = 0;
+    for (int r = lane; r < p.n_rounds; r += 32) {
+      const int tb = p.total_before[r * p.B + b];
+      n_lo += tb <= q0;
+      n_hi += tb <= q_last;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      n_lo += __shfl_xor_sync(0xffffffffu, n_lo, o);
+      n_hi += __shfl_xor_sync(0xffffffffu, n_hi, o);
+    }
+    const int r_lo = n_lo;
+    int r_hi = n_hi;
+    // per round that can be visible from this tile: its kept count and the sequence length when it fired
+    const int rho0 = max(r_lo, 1);
+    if (r_hi - rho0 + 1 > kMaxSeg - 1) {                // more rounds inside one query tile than the tables hold
+      if (lane == 0) set_dev_status(p.dev_status, NGC_DEV_BAD_COUNTS);
+      r_hi = rho0 + kMaxSeg - 2;
+    }
+    for (int rho = rho0 + lane; rho <= r_hi; rho += 32) {       // (at most three passes)
+      int n = p.alive_count[((int64_t)(rho - 1) * p.B + b) * p.G + gi];
+      if (n < 0 || n > p.kt_max) { set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); n = 0; }
+      sh.seg_n[rho - rho0] = n;                         // provisional: compacted below by lane 0
+    }
+    for (int r = r_lo + lane; r < r_hi; r += 32) sh.tb[r - r_lo] = p.total_before[r * p.B + b];
+    const int c_lo = r_lo >= 1 ? p.total_before[(r_lo - 1) * p.B + b] : 0;
+    __syncwarp();
+    if (lane == 0) {
+      int nseg = 0, first = 0;
+      for (int rho = rho0; rho <= r_hi; ++rho) {
+        const int n = sh.seg_n[rho - rho0];             // read before the slot can be overwritten (nseg <= rho - rho0)
+        if (n > 0) {
+          sh.seg_rho[nseg] = rho; sh.seg_n[nseg] = n; sh.seg_first[nseg] = first;
+          first += (n + kKeys - 1) / kKeys;
+          ++nseg;
+        }
+      }
+      sh.c_lo = c_lo;
+      sh.seg_rho[nseg] = -1; sh.seg_n[nseg] = q_last - c_lo + 1; sh.seg_first[nseg] = first;
+      first += (q_last - c_lo + kKeys) / kKeys;
+      ++nseg;
+      sh.seg_first[nseg] = first;
+      sh.nseg = nseg;
+      sh.uniform = r_lo == r_hi;                        // every query of the tile lies in the same block
+      sh.r_lo = r_lo; sh.r_hi = r_hi;
+    }
+  }
+  umma::fence_before_sync();
+  __syncthreads();
+  umma::fence_after_sync();
+  const uint32_t tmem = sh.tmem;
+  const int nseg = sh.nseg, c_lo = sh.c_lo, n_tiles = sh.seg_first[nseg];
+  const bool uniform = sh.uniform != 0;
 
-  // Q tiles of the two heads -> shared memory (rows beyond the sequence: zeros)
-  {
+  if (warp < kProducerWarp0) {
+    // Q tiles of the two heads -> shared memory (rows beyond the sequence: zeros); the producers are already
+    // gathering K and V meanwhile
     const int n_heads = has1 ? 2 : 1;
-    for (int i = tid; i < n_heads * kQRows * 16; i += kThreads) {
+    for (int i = tid; i < n_heads * kQRows * 16; i += kQLoaders) {
       const int hh = i / (kQRows * 16), rest = i - hh * kQRows * 16;
       const int r = rest >> 4, c = rest & 15;
       uint8_t* dst = sQ + hh * kQBytes + tile_off(kQHalf, r, c);
@@ -168,13 +202,8 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
     ptx::cp_async_commit();
     ptx::cp_async_wait_group<0>();
     ptx::fence_proxy_async();
+    ptx::mbar_arrive(&sh.q_full);
   }
-  umma::fence_before_sync();
-  __syncthreads();
-  umma::fence_after_sync();
-  const uint32_t tmem = sh.tmem;
-  const int nseg = sh.nseg, c_lo = sh.c_lo, n_tiles = sh.seg_first[nseg];
-  const bool uniform = sh.uniform != 0;
 
   if (warp >= kProducerWarp0) {
     // ------------------------------------------------------------------ producers
@@ -186,29 +215,41 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
       ptx::fence_proxy_async();
       ptx::mbar_arrive(&sh.kv_full[t % kStages]);
     };
+    const int pw = ptid >> 5;                           // producer warp w gathers rows 32 w .. 32 w + 31 of a tile
+    // position of key row 32 pw + lane of tile i (-1: no such key, -2: a kept position outside the sequence);
+    // one coalesced load per lane and tile, fetched one tile ahead
+    int sgi_pf = 0;
+    auto tile_pos = [&](int i) {
+      while (sgi_pf + 1 < nseg && i >= sh.seg_first[sgi_pf + 1]) ++sgi_pf;
+      const int rho = sh.seg_rho[sgi_pf], n = sh.seg_n[sgi_pf];
+      const int kidx = (i - sh.seg_first[sgi_pf]) * kKeys + 32 * pw + lane;
+      if (kidx >= n) return -1;
+      const int pos = rho >= 1 ? p.alive_pos[(((int64_t)(rho - 1) * p.B + b) * p.G + gi) * p.kt_max + kidx] : c_lo + kidx;
+      return (pos >= 0 && pos < T_b) ? pos : -2;
+    };
+    int pos_next = n_tiles > 0 ? tile_pos(0) : -1;
     for (int i = 0; i < n_tiles; ++i) {
       const int s = i % kStages;
+      const int pos_mine = pos_next;
+      if (i + 1 < n_tiles) pos_next = tile_pos(i + 1);
+      if (pos_mine == -2) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
       if (i >= kStages) {
         const bool ok = wait_or_abort(&sh.kv_empty[s], ((i / kStages) - 1) & 1, &sh, p.dev_status);
         if (!__all_sync(0xffffffffu, ok)) break;
       }
-      while (sgi + 1 < nseg && i >= sh.seg_first[sgi + 1]) ++sgi;
-      const int rho = sh.seg_rho[sgi], n = sh.seg_n[sgi], kt = i - sh.seg_first[sgi];
-      const int32_t* list = rho >= 1 ? p.alive_pos + (((int64_t)(rho - 1) * p.B + b) * p.G + gi) * p.kt_max : nullptr;
+      (void)sgi;
       uint8_t* st = stage + s * kStageBytes;
+      const int c = lane & 15;
 #pragma unroll 4
-      for (int u = 0; u < 16; ++u) {
-        const int slot = u * kProducerLanes + ptid;
-        const int row = slot >> 4, c = slot & 15;
-        const int kidx = kt * kKeys + row;
-        int pos = -1;
-        if (kidx < n) pos = list ? list[kidx] : c_lo + kidx;
+      for (int u = 0; u < 16; ++u) {                    // two rows per step, 16 lanes (16-byte pieces) per row
+        const int rl = 2 * u + (lane >> 4);
+        const int pos = __shfl_sync(0xffffffffu, pos_mine, rl);
+        const int row = 32 * pw + rl;
         const uint32_t off = tile_off(kKBox, row, c);
-        if (pos >= 0 && pos < T_b) {
+        if (pos >= 0) {
           ptx::cp_async_cg_16(ptx::smem_u32(st + off), k_strip + (int64_t)pos * 128 + 8 * c);
           ptx::cp_async_cg_16(ptx::smem_u32(st + kKTile + off), v_strip + (int64_t)pos * 128 + 8 * c);
         } else {      // past the end of the source: zeros (a stale NaN times P = 0 would poison the sum)
-          if (kidx < n && c == 0) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
           *reinterpret_cast<uint4*>(st + off) = make_uint4(0, 0, 0, 0);
           *reinterpret_cast<uint4*>(st + kKTile + off) = make_uint4(0, 0, 0, 0);
         }
@@ -242,7 +283,8 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
           umma::commit(&sh.s_full[hh][i & 1]);
         }
       };
-      bool ok = wait_or_abort(&sh.kv_full[0], 0, &sh, p.dev_status);
+      bool ok = wait_or_abort(&sh.q_full, 0, &sh, p.dev_status);
+      ok = ok && wait_or_abort(&sh.kv_full[0], 0, &sh, p.dev_status);
       if (ok) {
         umma::fence_after_sync();
         issue_s(0);
@@ -281,9 +323,9 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
     if (hh == 0 || has1) {
       const int row = 32 * (warp & 3) + lane;
       const int t_q = q0 + row;
-      int blk = 0, lo_row = 0;                          // round index of the row's block, its first position
-      for (int r = 0; r < p.n_rounds; ++r) {
-        const int tb = p.total_before[r * p.B + b];
+      int blk = sh.r_lo, lo_row = c_lo;                 // round index of the row's block, its first position
+      for (int r = sh.r_lo; r < sh.r_hi; ++r) {         // the rounds that fire inside this query tile
+        const int tb = sh.tb[r - sh.r_lo];
         if (tb <= t_q) { blk += 1; lo_row = tb; }
       }
       const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
