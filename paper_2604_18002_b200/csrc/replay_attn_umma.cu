@@ -2,14 +2,19 @@
 //
 // The replay pass is the one compute-bound contraction of this library: every token of a rollout
 // attends to the kept list of the last eviction round before it plus, causally, its own block.
-// One CTA takes 128 query tokens of TWO query heads that share a KV head; the 128 rows of a head are
-// the 128 lanes of tensor memory.
+// A work item is 128 query tokens of TWO query heads that share a KV head; the 128 rows of a head
+// are the 128 lanes of tensor memory.  The kernel is persistent: one CTA per SM walks a strided
+// list of items, and its warps are specialised roles that only meet at mbarriers, so the gathers,
+// the Q load and the tile bookkeeping of the next item run under the arithmetic of the current one.
 //
+//   planner warp (1)     per item: which kept lists and which contiguous run the 128 queries see
+//                        (a small table in a two-slot ring), then the Q tiles of both heads into
+//                        shared memory as soon as the previous item's last S product has read them;
 //   producer warps (2)   gather 64-key K/V tiles by position (kept lists, then the contiguous block)
 //                        with 16-byte cp.async into a 4-stage ring, 128-byte swizzled, and publish a
 //                        stage with a proxy fence + mbarrier arrival once its copies have landed.  Tile
-//                        i - 1 is published right after tile i has been issued, BEFORE the producer may
-//                        block on a free stage: the MMA warp needs tile i + 1 to finish tile i, so a
+//                        t - 1 is published right after tile t has been issued, BEFORE the producer may
+//                        block on a free stage: the MMA warp needs tile t + 1 to finish tile t, so a
 //                        producer that sat on landed tiles while waiting for a stage would deadlock;
 //   MMA warp (1 thread)  S_h = Q_h K^T (tcgen05.mma, M = 128, N = 64, both operands K-major) into a
 //                        double-buffered S in tensor memory, and O_h += P_h V (M = 128, N = 128, V as
@@ -20,11 +25,12 @@
 //                        maximum used for the exponentials only moves when the true maximum has grown
 //                        by more than 8 (a factor 256, exact in bf16 / fp32), so the O accumulator in
 //                        tensor memory is rescaled rarely; when it is, the row's owner does it in place
-//                        (tcgen05.ld / st) after the previous P V product has completed.
+//                        (tcgen05.ld / st) after the previous P V product has completed.  At the end of
+//                        an item the same thread normalises its O row and writes it out.
 //
-// The S product of tile i+1 is issued before the P V product of tile i, so the tensor pipe works on
+// The S product of tile t+1 is issued before the P V product of tile t, so the tensor pipe works on
 // one head while the other head's rows are in the softmax.  Every wait is bounded: a wait that runs
-// out raises a CTA-wide abort flag, every role leaves its loop, in-flight copies and MMAs are
+// out raises a CTA-wide abort flag, every role leaves its loops, in-flight copies and MMAs are
 // drained (bounded again), tensor memory is freed and NGC_DEV_TIMEOUT is reported.
 #include <cuda_bf16.h>
 
@@ -36,14 +42,14 @@
 namespace ngc {
 namespace {
 
-constexpr int kQRows = 128;                   // query tokens per CTA = tensor-memory lanes
+constexpr int kQRows = 128;                   // query tokens per item = tensor-memory lanes
 constexpr int kKeys = 64;                     // keys per pipeline stage
 constexpr int kStages = 4;
-constexpr int kSoftmaxWarps = 8;              // two groups of four, one query head each
-constexpr int kMmaWarp = 8;
-constexpr int kProducerWarp0 = 9;
+constexpr int kMmaWarp = 8;                   // warps 0-7: softmax (two groups of four, one query head each)
+constexpr int kProducerWarp0 = 9;             // warps 9, 10
 constexpr int kProducerLanes = 64;
-constexpr int kThreads = kProducerWarp0 * 32 + kProducerLanes;     // 352
+constexpr int kPlannerWarp = 11;
+constexpr int kThreads = 12 * 32;
 constexpr int kQHalf = kQRows * 128;          // one 64-channel half of a Q tile (128 rows x 128 B)
 constexpr int kQBytes = 2 * kQHalf;           // 32 KB per head
 constexpr int kKBox = kKeys * 128;            // 64 keys x 64 channels
@@ -52,16 +58,26 @@ constexpr int kStageBytes = 2 * kKTile;       // K + V
 constexpr int kPBytes = kQRows * 128;         // P tile of a head: 128 rows x 64 keys of bf16
 constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 2 * kPBytes + 1024;
 constexpr uint32_t kTmemCols = 512;           // S[h][buf] at (2h + buf) * 64, O[h] at 256 + 128 h
-constexpr int kMaxSeg = 66;                   // rounds one query tile can straddle (+ the contiguous part)
+constexpr int kMaxSeg = 34;                   // rounds one query tile can straddle (+ the contiguous part)
 constexpr float kLazyRescale = 8.f;           // log2 units the row maximum may grow before O is rescaled
+constexpr int kPlanSlots = 2;
+constexpr int kPlanReaders = 8 + 1 + 2;       // one arrival per softmax warp, the MMA thread, per producer warp
+
+// What the roles need to know about one item.
+struct Plan {
+  int l, b, h, hq0, has1, gi, q0, T_b;
+  int n_tiles;                                // 0: nothing to do (query tile beyond the sequence)
+  int nseg, c_lo, uniform, r_lo, r_hi;
+  int seg_rho[kMaxSeg], seg_n[kMaxSeg], seg_first[kMaxSeg + 1];
+  int tb[kMaxSeg];                            // sequence length at the rounds r_lo .. r_hi - 1 (those that fire inside the query tile)
+};
 
 struct Shared {
-  uint64_t kv_full[kStages], kv_empty[kStages], s_full[2][2], p_full[2], o_done[2], q_full, drain;
+  uint64_t kv_full[kStages], kv_empty[kStages], s_full[2][2], p_full[2], o_done[2];
+  uint64_t q_full, q_empty, plan_full[kPlanSlots], plan_empty[kPlanSlots], drain;
   uint32_t tmem;
   int abort;
-  int seg_rho[kMaxSeg], seg_n[kMaxSeg], seg_first[kMaxSeg + 1];
-  int tb[kMaxSeg];              // sequence length at the rounds r_lo .. r_hi - 1 (those that fire inside the query tile)
-  int nseg, c_lo, uniform, r_lo, r_hi;
+  Plan plan[kPlanSlots];
 };
 
 // Bounded wait that also gives up as soon as another thread of the CTA has given up.
@@ -80,13 +96,17 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Sh
     }
   }
 }
+// The same for a whole warp: every lane gets the same answer.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, Shared* sh, int32_t* dev_status) {
+  return __all_sync(0xffffffffu, wait_or_abort(bar, parity, sh, dev_status));
+}
 
 // swizzled byte offset of 16-byte piece c (0..15) of row r inside a tile of `half_bytes`-sized 64-channel halves
 __device__ __forceinline__ uint32_t tile_off(int half_bytes, int r, int c) {
   return (uint32_t)((c >> 3) * half_bytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAttnParams p) {
+__global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAttnParams p, int n_items) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ Shared sh;
 
@@ -95,23 +115,8 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
   uint8_t* stage = sQ + 2 * kQBytes;                    // [kStages][K 16 KB | V 16 KB]
   uint8_t* sP = stage + kStages * kStageBytes;          // [2 heads][16 KB]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
   const int pairs = (p.g + 1) >> 1;
-  int item = blockIdx.x;
-  const int m = item % p.q_tiles; item /= p.q_tiles;
-  const int pair = item % pairs; item /= pairs;
-  const int h = item % p.Hkv; item /= p.Hkv;
-  const int b = item % p.B;
-  const int l = item / p.B;
-  const int T_b = min(p.lens[b], p.t_max);
-  const int q0 = m * kQRows;
-  if (q0 >= T_b) return;                                // nothing allocated yet
-  const int hq0 = h * p.g + 2 * pair;
-  const bool has1 = 2 * pair + 1 < p.g;                 // an odd group leaves the last pair half empty
-  const int gi = list_of(p.lists, l, h, p.Hkv);
-  const int q_last = min(q0 + kQRows - 1, T_b - 1);
 
-  constexpr int kQLoaders = kProducerWarp0 * 32;        // the softmax warps and the MMA warp bring Q in
   if (tid == 0) {
 #pragma unroll
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&sh.kv_full[s], kProducerLanes); ptx::mbar_init(&sh.kv_empty[s], 1); }
@@ -120,146 +125,189 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
       ptx::mbar_init(&sh.s_full[hh][0], 1); ptx::mbar_init(&sh.s_full[hh][1], 1);
       ptx::mbar_init(&sh.p_full[hh], 128); ptx::mbar_init(&sh.o_done[hh], 1);
     }
-    ptx::mbar_init(&sh.q_full, kQLoaders);
+#pragma unroll
+    for (int s = 0; s < kPlanSlots; ++s) { ptx::mbar_init(&sh.plan_full[s], 1); ptx::mbar_init(&sh.plan_empty[s], kPlanReaders); }
+    ptx::mbar_init(&sh.q_full, 32);
+    ptx::mbar_init(&sh.q_empty, 1);
     ptx::mbar_init(&sh.drain, 1);
     ptx::fence_barrier_init();
     sh.abort = 0;
   }
   if (warp == kMmaWarp) umma::tmem_alloc(&sh.tmem, kTmemCols);
-  if (warp == 0) {
-    // key sources of this query tile: the kept lists of the rounds it straddles, then the contiguous run.
-    // Rounds fired before the first / last query of the tile: counted by the whole warp (independent loads).
-    int n_lo = 0, n_hi = 0;
-    for (int r = lane; r < p.n_rounds; r += 32) {
-      const int tb = p.total_before[r * p.B + b];
-      n_lo += tb <= q0;
-      n_hi += tb <= q_last;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      n_lo += __shfl_xor_sync(0xffffffffu, n_lo, o);
-      n_hi += __shfl_xor_sync(0xffffffffu, n_hi, o);
-    }
-    const int r_lo = n_lo;
-    int r_hi = n_hi;
-    // per round that can be visible from this tile: its kept count and the sequence length when it fired
-    const int rho0 = max(r_lo, 1);
-    if (r_hi - rho0 + 1 > kMaxSeg - 1) {                // more rounds inside one query tile than the tables hold
-      if (lane == 0) set_dev_status(p.dev_status, NGC_DEV_BAD_COUNTS);
-      r_hi = rho0 + kMaxSeg - 2;
-    }
-    for (int rho = rho0 + lane; rho <= r_hi; rho += 32) {       // (at most three passes)
-      int n = p.alive_count[((int64_t)(rho - 1) * p.B + b) * p.G + gi];
-      if (n < 0 || n > p.kt_max) { set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); n = 0; }
-      sh.seg_n[rho - rho0] = n;                         // provisional: compacted below by lane 0
-    }
-    for (int r = r_lo + lane; r < r_hi; r += 32) sh.tb[r - r_lo] = p.total_before[r * p.B + b];
-    const int c_lo = r_lo >= 1 ? p.total_before[(r_lo - 1) * p.B + b] : 0;
-    __syncwarp();
-    if (lane == 0) {
-      int nseg = 0, first = 0;
-      for (int rho = rho0; rho <= r_hi; ++rho) {
-        const int n = sh.seg_n[rho - rho0];             // read before the slot can be overwritten (nseg <= rho - rho0)
-        if (n > 0) {
-          sh.seg_rho[nseg] = rho; sh.seg_n[nseg] = n; sh.seg_first[nseg] = first;
-          first += (n + kKeys - 1) / kKeys;
-          ++nseg;
-        }
-      }
-      sh.c_lo = c_lo;
-      sh.seg_rho[nseg] = -1; sh.seg_n[nseg] = q_last - c_lo + 1; sh.seg_first[nseg] = first;
-      first += (q_last - c_lo + kKeys) / kKeys;
-      ++nseg;
-      sh.seg_first[nseg] = first;
-      sh.nseg = nseg;
-      sh.uniform = r_lo == r_hi;                        // every query of the tile lies in the same block
-      sh.r_lo = r_lo; sh.r_hi = r_hi;
-    }
-  }
   umma::fence_before_sync();
   __syncthreads();
   umma::fence_after_sync();
   const uint32_t tmem = sh.tmem;
-  const int nseg = sh.nseg, c_lo = sh.c_lo, n_tiles = sh.seg_first[nseg];
-  const bool uniform = sh.uniform != 0;
 
-  if (warp < kProducerWarp0) {
-    // Q tiles of the two heads -> shared memory (rows beyond the sequence: zeros); the producers are already
-    // gathering K and V meanwhile
-    const int n_heads = has1 ? 2 : 1;
-    for (int i = tid; i < n_heads * kQRows * 16; i += kQLoaders) {
-      const int hh = i / (kQRows * 16), rest = i - hh * kQRows * 16;
-      const int r = rest >> 4, c = rest & 15;
-      uint8_t* dst = sQ + hh * kQBytes + tile_off(kQHalf, r, c);
-      const int t = q0 + r;
-      if (t < T_b) {
-        const __nv_bfloat16* src = p.q + ((((int64_t)l * p.B + b) * p.Hq + hq0 + hh) * (int64_t)p.t_max + t) * 128 + 8 * c;
-        ptx::cp_async_cg_16(ptx::smem_u32(dst), src);
-      } else {
-        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+  // Every role walks the same items in the same order: item k of this CTA is blockIdx.x + k * gridDim.x and uses plan
+  // slot k & 1.  Ring positions and barrier phases follow from running counters that every role keeps for itself:
+  // tiles of all items so far -> K/V stage, S buffer and P / O phases of head 0; tiles of the items that have a second
+  // head -> those of head 1.
+
+  if (warp == kPlannerWarp) {
+    // ------------------------------------------------------------------ planner: item tables, then Q
+    int n_q = 0;                                        // items that had tiles (Q loads) so far
+    int k = 0;
+    for (int it = blockIdx.x; it < n_items; it += gridDim.x, ++k) {
+      const int slot = k & 1;
+      if (k >= kPlanSlots && !warp_wait(&sh.plan_empty[slot], ((k >> 1) - 1) & 1, &sh, p.dev_status)) break;
+      Plan& pl = sh.plan[slot];
+      int item = it;
+      const int m = item % p.q_tiles; item /= p.q_tiles;
+      const int pair = item % pairs; item /= pairs;
+      const int h = item % p.Hkv; item /= p.Hkv;
+      const int b = item % p.B;
+      const int l = item / p.B;
+      const int T_b = min(p.lens[b], p.t_max);
+      const int q0 = m * kQRows;
+      const int hq0 = h * p.g + 2 * pair;
+      const int has1 = 2 * pair + 1 < p.g;              // an odd group leaves the last pair half empty
+      const int gi = list_of(p.lists, l, h, p.Hkv);
+      int n_tiles = 0;
+      if (q0 < T_b) {
+        const int q_last = min(q0 + kQRows - 1, T_b - 1);
+        // rounds fired before the first / last query of the tile: counted by the whole warp (independent loads)
+        int n_lo = 0, n_hi = 0;
+        for (int r = lane; r < p.n_rounds; r += 32) {
+          const int tb = p.total_before[r * p.B + b];
+          n_lo += tb <= q0;
+          n_hi += tb <= q_last;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          n_lo += __shfl_xor_sync(0xffffffffu, n_lo, o);
+          n_hi += __shfl_xor_sync(0xffffffffu, n_hi, o);
+        }
+        const int r_lo = n_lo;
+        int r_hi = n_hi;
+        // key sources of the tile: the kept lists of the rounds it straddles (rho = r_lo .. r_hi, from 1), then the contiguous run
+        const int rho0 = max(r_lo, 1);
+        if (r_hi - rho0 + 1 > kMaxSeg - 1) {            // more rounds inside one query tile than the table holds
+          if (lane == 0) set_dev_status(p.dev_status, NGC_DEV_BAD_COUNTS);
+          r_hi = rho0 + kMaxSeg - 2;
+        }
+        for (int rho = rho0 + lane; rho <= r_hi; rho += 32) {
+          int n = p.alive_count[((int64_t)(rho - 1) * p.B + b) * p.G + gi];
+          if (n < 0 || n > p.kt_max) { set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT); n = 0; }
+          pl.seg_n[rho - rho0] = n;                     // provisional: compacted below by lane 0
+        }
+        for (int r = r_lo + lane; r < r_hi; r += 32) pl.tb[r - r_lo] = p.total_before[r * p.B + b];
+        const int c_lo = r_lo >= 1 ? p.total_before[(r_lo - 1) * p.B + b] : 0;
+        __syncwarp();
+        if (lane == 0) {
+          int nseg = 0, first = 0;
+          for (int rho = rho0; rho <= r_hi; ++rho) {
+            const int n = pl.seg_n[rho - rho0];         // read before the slot can be overwritten (nseg <= rho - rho0)
+            if (n > 0) {
+              pl.seg_rho[nseg] = rho; pl.seg_n[nseg] = n; pl.seg_first[nseg] = first;
+              first += (n + kKeys - 1) / kKeys;
+              ++nseg;
+            }
+          }
+          pl.c_lo = c_lo;
+          pl.seg_rho[nseg] = -1; pl.seg_n[nseg] = q_last - c_lo + 1; pl.seg_first[nseg] = first;
+          first += (q_last - c_lo + kKeys) / kKeys;
+          ++nseg;
+          pl.seg_first[nseg] = first;
+          pl.nseg = nseg;
+          pl.uniform = r_lo == r_hi;                    // every query of the tile lies in the same block
+          pl.r_lo = r_lo; pl.r_hi = r_hi;
+          pl.n_tiles = first;
+        }
+        __syncwarp();
+        n_tiles = pl.n_tiles;
       }
+      if (lane == 0) {
+        pl.l = l; pl.b = b; pl.h = h; pl.hq0 = hq0; pl.has1 = has1; pl.gi = gi; pl.q0 = q0; pl.T_b = T_b;
+        if (n_tiles == 0) pl.n_tiles = 0;
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&sh.plan_full[slot]);
+      if (n_tiles == 0) continue;
+      // Q tiles of the two heads -> shared memory (rows beyond the sequence: zeros), once the previous item's
+      // last S product has read the buffer
+      if (n_q >= 1 && !warp_wait(&sh.q_empty, (n_q - 1) & 1, &sh, p.dev_status)) break;
+      const int n_heads = has1 ? 2 : 1;
+      for (int i = lane; i < n_heads * kQRows * 16; i += 32) {
+        const int hh = i / (kQRows * 16), rest = i - hh * kQRows * 16;
+        const int r = rest >> 4, c = rest & 15;
+        uint8_t* dst = sQ + hh * kQBytes + tile_off(kQHalf, r, c);
+        const int t = q0 + r;
+        if (t < T_b) {
+          const __nv_bfloat16* src = p.q + ((((int64_t)l * p.B + b) * p.Hq + hq0 + hh) * (int64_t)p.t_max + t) * 128 + 8 * c;
+          ptx::cp_async_cg_16(ptx::smem_u32(dst), src);
+        } else {
+          *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      ptx::cp_async_commit();
+      ptx::cp_async_wait_group<0>();
+      ptx::fence_proxy_async();
+      ptx::mbar_arrive(&sh.q_full);
+      ++n_q;
     }
-    ptx::cp_async_commit();
     ptx::cp_async_wait_group<0>();
-    ptx::fence_proxy_async();
-    ptx::mbar_arrive(&sh.q_full);
-  }
-
-  if (warp >= kProducerWarp0) {
+  } else if (warp >= kProducerWarp0) {
     // ------------------------------------------------------------------ producers
     const int ptid = tid - kProducerWarp0 * 32;
-    const __nv_bfloat16* k_strip = p.k + ((int64_t)(l * p.Hkv + h) * p.rows_R + p.seq_off[b]) * 128;
-    const __nv_bfloat16* v_strip = p.v + ((int64_t)(l * p.Hkv + h) * p.rows_R + p.seq_off[b]) * 128;
-    int issued = 0, published = 0, sgi = 0;
+    const int pw = ptid >> 5;                           // producer warp w gathers rows 32 w .. 32 w + 31 of a tile
+    int issued = 0, published = 0;                      // tiles, over all items
     auto publish = [&](int t) {                         // this lane's copies of tile t have landed
       ptx::fence_proxy_async();
       ptx::mbar_arrive(&sh.kv_full[t % kStages]);
     };
-    const int pw = ptid >> 5;                           // producer warp w gathers rows 32 w .. 32 w + 31 of a tile
-    // position of key row 32 pw + lane of tile i (-1: no such key, -2: a kept position outside the sequence);
-    // one coalesced load per lane and tile, fetched one tile ahead
-    int sgi_pf = 0;
-    auto tile_pos = [&](int i) {
-      while (sgi_pf + 1 < nseg && i >= sh.seg_first[sgi_pf + 1]) ++sgi_pf;
-      const int rho = sh.seg_rho[sgi_pf], n = sh.seg_n[sgi_pf];
-      const int kidx = (i - sh.seg_first[sgi_pf]) * kKeys + 32 * pw + lane;
-      if (kidx >= n) return -1;
-      const int pos = rho >= 1 ? p.alive_pos[(((int64_t)(rho - 1) * p.B + b) * p.G + gi) * p.kt_max + kidx] : c_lo + kidx;
-      return (pos >= 0 && pos < T_b) ? pos : -2;
-    };
-    int pos_next = n_tiles > 0 ? tile_pos(0) : -1;
-    for (int i = 0; i < n_tiles; ++i) {
-      const int s = i % kStages;
-      const int pos_mine = pos_next;
-      if (i + 1 < n_tiles) pos_next = tile_pos(i + 1);
-      if (pos_mine == -2) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
-      if (i >= kStages) {
-        const bool ok = wait_or_abort(&sh.kv_empty[s], ((i / kStages) - 1) & 1, &sh, p.dev_status);
-        if (!__all_sync(0xffffffffu, ok)) break;
-      }
-      (void)sgi;
-      uint8_t* st = stage + s * kStageBytes;
-      const int c = lane & 15;
+    bool ok = true;
+    int k = 0;
+    for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x, ++k) {
+      const int slot = k & 1;
+      if (!warp_wait(&sh.plan_full[slot], (k >> 1) & 1, &sh, p.dev_status)) break;
+      const Plan& pl = sh.plan[slot];
+      const int n_tiles = pl.n_tiles, nseg = pl.nseg, c_lo = pl.c_lo, T_b = pl.T_b, b = pl.b, gi = pl.gi;
+      const __nv_bfloat16* k_strip = p.k + ((int64_t)(pl.l * p.Hkv + pl.h) * p.rows_R + p.seq_off[b]) * 128;
+      const __nv_bfloat16* v_strip = p.v + ((int64_t)(pl.l * p.Hkv + pl.h) * p.rows_R + p.seq_off[b]) * 128;
+      // position of key row 32 pw + lane of tile i (-1: no such key, -2: a kept position outside the sequence);
+      // one coalesced load per lane and tile, fetched one tile ahead
+      int sgi = 0;
+      auto tile_pos = [&](int i) {
+        while (sgi + 1 < nseg && i >= pl.seg_first[sgi + 1]) ++sgi;
+        const int rho = pl.seg_rho[sgi], n = pl.seg_n[sgi];
+        const int kidx = (i - pl.seg_first[sgi]) * kKeys + 32 * pw + lane;
+        if (kidx >= n) return -1;
+        const int pos = rho >= 1 ? p.alive_pos[(((int64_t)(rho - 1) * p.B + b) * p.G + gi) * p.kt_max + kidx] : c_lo + kidx;
+        return (pos >= 0 && pos < T_b) ? pos : -2;
+      };
+      int pos_next = n_tiles > 0 ? tile_pos(0) : -1;
+      for (int i = 0; i < n_tiles; ++i) {
+        const int s = issued % kStages;
+        const int pos_mine = pos_next;
+        if (i + 1 < n_tiles) pos_next = tile_pos(i + 1);
+        if (pos_mine == -2) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
+        if (issued >= kStages && !warp_wait(&sh.kv_empty[s], ((issued / kStages) - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+        uint8_t* st = stage + s * kStageBytes;
+        const int c = lane & 15;
 #pragma unroll 4
-      for (int u = 0; u < 16; ++u) {                    // two rows per step, 16 lanes (16-byte pieces) per row
-        const int rl = 2 * u + (lane >> 4);
-        const int pos = __shfl_sync(0xffffffffu, pos_mine, rl);
-        const int row = 32 * pw + rl;
-        const uint32_t off = tile_off(kKBox, row, c);
-        if (pos >= 0) {
-          ptx::cp_async_cg_16(ptx::smem_u32(st + off), k_strip + (int64_t)pos * 128 + 8 * c);
-          ptx::cp_async_cg_16(ptx::smem_u32(st + kKTile + off), v_strip + (int64_t)pos * 128 + 8 * c);
-        } else {      // past the end of the source: zeros (a stale NaN times P = 0 would poison the sum)
-          *reinterpret_cast<uint4*>(st + off) = make_uint4(0, 0, 0, 0);
-          *reinterpret_cast<uint4*>(st + kKTile + off) = make_uint4(0, 0, 0, 0);
+        for (int u = 0; u < 16; ++u) {                  // two rows per step, 16 lanes (16-byte pieces) per row
+          const int rl = 2 * u + (lane >> 4);
+          const int pos = __shfl_sync(0xffffffffu, pos_mine, rl);
+          const int row = 32 * pw + rl;
+          const uint32_t off = tile_off(kKBox, row, c);
+          if (pos >= 0) {
+            ptx::cp_async_cg_16(ptx::smem_u32(st + off), k_strip + (int64_t)pos * 128 + 8 * c);
+            ptx::cp_async_cg_16(ptx::smem_u32(st + kKTile + off), v_strip + (int64_t)pos * 128 + 8 * c);
+          } else {    // past the end of the source: zeros (a stale NaN times P = 0 would poison the sum)
+            *reinterpret_cast<uint4*>(st + off) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(st + kKTile + off) = make_uint4(0, 0, 0, 0);
+          }
+        }
+        ptx::cp_async_commit();
+        ++issued;
+        if (issued - published > 1) {                   // everything but the tile just issued has landed
+          ptx::cp_async_wait_group<1>();
+          publish(published++);
         }
       }
-      ptx::cp_async_commit();
-      ++issued;
-      if (issued - published > 1) {                     // everything but the tile just issued has landed
-        ptx::cp_async_wait_group<1>();
-        publish(published++);
-      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&sh.plan_empty[slot]);
     }
     ptx::cp_async_wait_group<0>();
     if (issued - published == 1) publish(published++);
@@ -269,48 +317,63 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
       constexpr uint32_t idesc_s = umma::instr_desc(kQRows, kKeys, false);
       constexpr uint32_t idesc_o = umma::instr_desc(kQRows, 128, true);
       const uint32_t q_addr = ptx::smem_u32(sQ), p_addr = ptx::smem_u32(sP), st_addr = ptx::smem_u32(stage);
-      const int n_heads = has1 ? 2 : 1;
-      auto issue_s = [&](int i) {                       // S_h(i) = Q_h K(i)^T into buffer i & 1
-        const uint32_t k_addr = st_addr + (i % kStages) * kStageBytes;
-        for (int hh = 0; hh < n_heads; ++hh) {
-          const uint32_t d = tmem + (uint32_t)((2 * hh + (i & 1)) * kKeys);
+      int t0 = 0, t1 = 0, n_q = 0;                      // tiles so far (head 0 = all, head 1), items with tiles so far
+      bool ok = true;
+      int k = 0;
+      for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x, ++k) {
+        const int slot = k & 1;
+        if (!wait_or_abort(&sh.plan_full[slot], (k >> 1) & 1, &sh, p.dev_status)) break;
+        const int n_tiles = sh.plan[slot].n_tiles;
+        const int n_heads = sh.plan[slot].has1 ? 2 : 1;
+        ptx::mbar_arrive(&sh.plan_empty[slot]);         // nothing else of the table is needed here
+        if (n_tiles == 0) continue;
+        auto issue_s = [&](int i) {                     // S_h = Q_h K^T for tile i of this item, into the head's next S buffer
+          const uint32_t k_addr = st_addr + ((t0 + i) % kStages) * kStageBytes;
+          for (int hh = 0; hh < n_heads; ++hh) {
+            const int buf = ((hh ? t1 : t0) + i) & 1;
+            const uint32_t d = tmem + (uint32_t)((2 * hh + buf) * kKeys);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t a = umma::smem_desc_sw128(q_addr + hh * kQBytes + (ks >> 2) * kQHalf + (ks & 3) * 32, 16, 1024);
-            const uint64_t bd = umma::smem_desc_sw128(k_addr + (ks >> 2) * kKBox + (ks & 3) * 32, 16, 1024);
-            umma::mma_bf16(d, a, bd, idesc_s, ks > 0);
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint64_t a = umma::smem_desc_sw128(q_addr + hh * kQBytes + (ks >> 2) * kQHalf + (ks & 3) * 32, 16, 1024);
+              const uint64_t bd = umma::smem_desc_sw128(k_addr + (ks >> 2) * kKBox + (ks & 3) * 32, 16, 1024);
+              umma::mma_bf16(d, a, bd, idesc_s, ks > 0);
+            }
+            umma::commit(&sh.s_full[hh][buf]);
           }
-          umma::commit(&sh.s_full[hh][i & 1]);
-        }
-      };
-      bool ok = wait_or_abort(&sh.q_full, 0, &sh, p.dev_status);
-      ok = ok && wait_or_abort(&sh.kv_full[0], 0, &sh, p.dev_status);
-      if (ok) {
+          if (i == n_tiles - 1) umma::commit(&sh.q_empty);     // the item's last product that reads Q
+        };
+        ok = wait_or_abort(&sh.q_full, n_q & 1, &sh, p.dev_status) &&
+             wait_or_abort(&sh.kv_full[t0 % kStages], (t0 / kStages) & 1, &sh, p.dev_status);
+        if (!ok) break;
         umma::fence_after_sync();
         issue_s(0);
-      }
-      for (int i = 0; ok && i < n_tiles; ++i) {
-        if (i + 1 < n_tiles) {
-          ok = wait_or_abort(&sh.kv_full[(i + 1) % kStages], ((i + 1) / kStages) & 1, &sh, p.dev_status);
-          if (!ok) break;
-          umma::fence_after_sync();
-          issue_s(i + 1);                               // its S buffer was read out before P(i - 1) was published
-        }
-        const uint32_t v_addr = st_addr + (i % kStages) * kStageBytes + kKTile;
-        for (int hh = 0; hh < n_heads; ++hh) {
-          ok = wait_or_abort(&sh.p_full[hh], i & 1, &sh, p.dev_status);
-          if (!ok) break;
-          umma::fence_after_sync();
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {              // 16 keys per step
-            const uint64_t a = umma::smem_desc_sw128(p_addr + hh * kPBytes + kk * 32, 16, 1024);
-            const uint64_t bd = umma::smem_desc_sw128(v_addr + kk * 2048, kKBox, 1024);   // next 64 channels: one box on
-            umma::mma_bf16(tmem + 256u + 128u * hh, a, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+        for (int i = 0; i < n_tiles; ++i) {
+          const int t = t0 + i;
+          if (i + 1 < n_tiles) {
+            ok = wait_or_abort(&sh.kv_full[(t + 1) % kStages], ((t + 1) / kStages) & 1, &sh, p.dev_status);
+            if (!ok) break;
+            umma::fence_after_sync();
+            issue_s(i + 1);                             // its S buffer was read out before P of two tiles ago was published
           }
-          umma::commit(&sh.o_done[hh]);
+          const uint32_t v_addr = st_addr + (t % kStages) * kStageBytes + kKTile;
+          for (int hh = 0; hh < n_heads; ++hh) {
+            ok = wait_or_abort(&sh.p_full[hh], ((hh ? t1 : t0) + i) & 1, &sh, p.dev_status);
+            if (!ok) break;
+            umma::fence_after_sync();
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {            // 16 keys per step
+              const uint64_t a = umma::smem_desc_sw128(p_addr + hh * kPBytes + kk * 32, 16, 1024);
+              const uint64_t bd = umma::smem_desc_sw128(v_addr + kk * 2048, kKBox, 1024);   // next 64 channels: one box on
+              umma::mma_bf16(tmem + 256u + 128u * hh, a, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+            }
+            umma::commit(&sh.o_done[hh]);
+          }
+          if (!ok) break;
+          umma::commit(&sh.kv_empty[t % kStages]);      // K and V of this stage have been consumed
         }
-        if (!ok) break;
-        umma::commit(&sh.kv_empty[i % kStages]);        // K and V of this stage have been consumed
+        t0 += n_tiles;
+        if (n_heads == 2) t1 += n_tiles;
+        ++n_q;
       }
       // everything issued has completed before tensor memory is released
       umma::commit(&sh.drain);
@@ -320,119 +383,121 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
   } else {
     // ------------------------------------------------------------------ softmax: one thread per query row
     const int hh = warp >> 2;
-    if (hh == 0 || has1) {
-      const int row = 32 * (warp & 3) + lane;
-      const int t_q = q0 + row;
-      int blk = sh.r_lo, lo_row = c_lo;                 // round index of the row's block, its first position
-      for (int r = sh.r_lo; r < sh.r_hi; ++r) {         // the rounds that fire inside this query tile
-        const int tb = sh.tb[r - sh.r_lo];
-        if (tb <= t_q) { blk += 1; lo_row = tb; }
-      }
-      const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
-      const uint32_t o_addr = tmem + lane_base + 256u + 128u * hh;
-      uint8_t* p_row = sP + hh * kPBytes + row * 128;
-      float m_use = -INFINITY, l_run = 0.f;
-      int o_seen = -1;                                  // last tile whose P V product is known to be complete
-      int sgi = 0;
-      bool ok = true;
-      for (int i = 0; i < n_tiles; ++i) {
-        ok = wait_or_abort(&sh.s_full[hh][i & 1], (i >> 1) & 1, &sh, p.dev_status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        umma::fence_after_sync();
-        uint32_t zr[2][32];
-        const uint32_t s_addr = tmem + lane_base + (uint32_t)((2 * hh + (i & 1)) * kKeys);
-        umma::tmem_ld32(s_addr, zr[0]);
-        umma::tmem_ld32(s_addr + 32, zr[1]);
-        umma::tmem_ld_wait();
-        while (sgi + 1 < nseg && i >= sh.seg_first[sgi + 1]) ++sgi;
-        const int rho = sh.seg_rho[sgi], kt = i - sh.seg_first[sgi];
-        const int n_here = min(kKeys, sh.seg_n[sgi] - kt * kKeys);
-        // a tile needs no mask when every query of the CTA lies in one block and the tile is a full tile of that
-        // block's kept list, or lies entirely before the first query
-        const bool need_mask = !uniform || (rho >= 1 ? n_here < kKeys : c_lo + kt * kKeys + kKeys - 1 > q0);
-        float mx = -INFINITY;
-        if (need_mask) {
-          const int j0 = c_lo + kt * kKeys;
-#pragma unroll
-          for (int half = 0; half < 2; ++half)
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int jj = 32 * half + j;
-              bool vis;
-              if (rho >= 1) vis = jj < n_here && blk == rho;                   // a kept entry of the round before this row's block
-              else vis = j0 + jj >= lo_row && j0 + jj <= t_q;                  // a token of the row's own block, causal
-              const float z = vis ? __uint_as_float(zr[half][j]) * p.scale_log2 : -INFINITY;
-              zr[half][j] = __float_as_uint(z);
-              mx = fmaxf(mx, z);
-            }
-        } else {
-#pragma unroll
-          for (int half = 0; half < 2; ++half)
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float z = __uint_as_float(zr[half][j]) * p.scale_log2;
-              zr[half][j] = __float_as_uint(z);
-              mx = fmaxf(mx, z);
-            }
+    const int row = 32 * (warp & 3) + lane;
+    const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
+    const uint32_t o_addr = tmem + lane_base + 256u + 128u * hh;
+    uint8_t* p_row = sP + hh * kPBytes + row * 128;
+    int tc = 0;                                         // tiles this head has been through, over all items
+    bool ok = true;
+    int k = 0;
+    for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x, ++k) {
+      const int slot = k & 1;
+      if (!warp_wait(&sh.plan_full[slot], (k >> 1) & 1, &sh, p.dev_status)) break;
+      const Plan& pl = sh.plan[slot];
+      const int n_tiles = (hh == 0 || pl.has1) ? pl.n_tiles : 0;
+      if (n_tiles > 0) {
+        const int q0 = pl.q0, T_b = pl.T_b, c_lo = pl.c_lo, nseg = pl.nseg;
+        const bool uniform = pl.uniform != 0;
+        const int t_q = q0 + row;
+        int blk = pl.r_lo, lo_row = c_lo;               // round index of the row's block, its first position
+        for (int r = pl.r_lo; r < pl.r_hi; ++r) {       // the rounds that fire inside this query tile
+          const int tb = pl.tb[r - pl.r_lo];
+          if (tb <= t_q) { blk += 1; lo_row = tb; }
         }
-        // the maximum used for the exponentials follows the true one lazily
-        const bool grow = mx > m_use + kLazyRescale;                          // also the first visible key (m_use = -inf)
-        const bool rescale = grow && m_use != -INFINITY && i > 0;             // O already holds something for this row
-        if (__any_sync(0xffffffffu, rescale)) {
-          if (o_seen < i - 1) {
-            ok = wait_or_abort(&sh.o_done[hh], (i - 1) & 1, &sh, p.dev_status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            o_seen = i - 1;
-            umma::fence_after_sync();
+        float m_use = -INFINITY, l_run = 0.f;
+        int o_seen = tc - 1;                            // last tile whose P V product is known to be complete
+        int sgi = 0;
+        for (int i = 0; i < n_tiles; ++i) {
+          const int t = tc + i;
+          if (!warp_wait(&sh.s_full[hh][t & 1], (t >> 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+          umma::fence_after_sync();
+          uint32_t zr[2][32];
+          const uint32_t s_addr = tmem + lane_base + (uint32_t)((2 * hh + (t & 1)) * kKeys);
+          umma::tmem_ld32(s_addr, zr[0]);
+          umma::tmem_ld32(s_addr + 32, zr[1]);
+          umma::tmem_ld_wait();
+          while (sgi + 1 < nseg && i >= pl.seg_first[sgi + 1]) ++sgi;
+          const int rho = pl.seg_rho[sgi], kt = i - pl.seg_first[sgi];
+          const int n_here = min(kKeys, pl.seg_n[sgi] - kt * kKeys);
+          // a tile needs no mask when every query of the item lies in one block and the tile is a full tile of that
+          // block's kept list, or lies entirely before the first query
+          const bool need_mask = !uniform || (rho >= 1 ? n_here < kKeys : c_lo + kt * kKeys + kKeys - 1 > q0);
+          float mx = -INFINITY;
+          if (need_mask) {
+            const int j0 = c_lo + kt * kKeys;
+#pragma unroll
+            for (int half = 0; half < 2; ++half)
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const int jj = 32 * half + j;
+                bool vis;
+                if (rho >= 1) vis = jj < n_here && blk == rho;                 // a kept entry of the round before this row's block
+                else vis = j0 + jj >= lo_row && j0 + jj <= t_q;                // a token of the row's own block, causal
+                const float z = vis ? __uint_as_float(zr[half][j]) * p.scale_log2 : -INFINITY;
+                zr[half][j] = __float_as_uint(z);
+                mx = fmaxf(mx, z);
+              }
+          } else {
+#pragma unroll
+            for (int half = 0; half < 2; ++half)
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float z = __uint_as_float(zr[half][j]) * p.scale_log2;
+                zr[half][j] = __float_as_uint(z);
+                mx = fmaxf(mx, z);
+              }
           }
-          const float alpha = rescale ? ptx::ex2_approx(m_use - mx) : 1.f;
-          l_run *= alpha;
+          // the maximum used for the exponentials follows the true one lazily
+          const bool grow = mx > m_use + kLazyRescale;                        // also the first visible key (m_use = -inf)
+          const bool rescale = grow && m_use != -INFINITY && i > 0;           // O already holds something for this row
+          if (__any_sync(0xffffffffu, rescale)) {
+            if (o_seen < t - 1) {
+              if (!warp_wait(&sh.o_done[hh], (t - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+              o_seen = t - 1;
+              umma::fence_after_sync();
+            }
+            const float alpha = rescale ? ptx::ex2_approx(m_use - mx) : 1.f;
+            l_run *= alpha;
 #pragma unroll 1
-          for (int c0 = 0; c0 < 128; c0 += 32) {
-            uint32_t o[32];
-            umma::tmem_ld32(o_addr + c0, o);
-            umma::tmem_ld_wait();
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+              uint32_t o[32];
+              umma::tmem_ld32(o_addr + c0, o);
+              umma::tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-            umma::tmem_st32(o_addr + c0, o);
+              for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+              umma::tmem_st32(o_addr + c0, o);
+            }
+            umma::tmem_st_wait();
           }
-          umma::tmem_st_wait();
-        }
-        if (grow) m_use = mx;
-        const float m_eff = m_use == -INFINITY ? 0.f : m_use;                 // nothing visible yet: every exponential is 0
-        uint32_t pk[32];
+          if (grow) m_use = mx;
+          const float m_eff = m_use == -INFINITY ? 0.f : m_use;               // nothing visible yet: every exponential is 0
+          uint32_t pk[32];
 #pragma unroll
-        for (int half = 0; half < 2; ++half)
+          for (int half = 0; half < 2; ++half)
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float p0 = ptx::ex2_approx(__uint_as_float(zr[half][j]) - m_eff);
-            const float p1 = ptx::ex2_approx(__uint_as_float(zr[half][j + 1]) - m_eff);
-            l_run += p0 + p1;
-            pk[16 * half + (j >> 1)] = ptx::pack_bf16x2(p0, p1);
+            for (int j = 0; j < 32; j += 2) {
+              const float p0 = ptx::ex2_approx(__uint_as_float(zr[half][j]) - m_eff);
+              const float p1 = ptx::ex2_approx(__uint_as_float(zr[half][j + 1]) - m_eff);
+              l_run += p0 + p1;
+              pk[16 * half + (j >> 1)] = ptx::pack_bf16x2(p0, p1);
+            }
+          if (t > 0 && o_seen < t - 1) {                                      // the P tile is free once the previous P V has completed
+            if (!warp_wait(&sh.o_done[hh], (t - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+            o_seen = t - 1;
           }
-        if (i > 0 && o_seen < i - 1) {                                        // the P tile is free once P V (i - 1) has completed
-          ok = wait_or_abort(&sh.o_done[hh], (i - 1) & 1, &sh, p.dev_status);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          o_seen = i - 1;
-        }
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-          *reinterpret_cast<uint4*>(p_row + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-        ptx::fence_proxy_async();
-        umma::fence_before_sync();
-        ptx::mbar_arrive(&sh.p_full[hh]);
-      }
-      if (ok) {
-        ok = wait_or_abort(&sh.o_done[hh], (n_tiles - 1) & 1, &sh, p.dev_status);
-        ok = __all_sync(0xffffffffu, ok);
-      }
-      if (ok) {
+          for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<uint4*>(p_row + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+          ptx::fence_proxy_async();
+          umma::fence_before_sync();
+          ptx::mbar_arrive(&sh.p_full[hh]);
+        }
+        if (!ok) break;
+        tc += n_tiles;
+        if (!warp_wait(&sh.o_done[hh], (tc - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
         umma::fence_after_sync();
         const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-        const int64_t o_base = ((((int64_t)l * p.B + b) * p.Hq + hq0 + hh) * (int64_t)p.t_max + t_q) * 128;
+        const int64_t o_base = ((((int64_t)pl.l * p.B + pl.b) * p.Hq + pl.hq0 + hh) * (int64_t)p.t_max + t_q) * 128;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 32) {
           uint32_t o[32];
@@ -456,10 +521,14 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
             }
           }
         }
+        // (the next item's first P V overwrites O only after this thread has published its next P row, which comes
+        // after these reads)
       }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&sh.plan_empty[slot]);
     }
   }
-  // ---- teardown: every role has left its loop; nothing of this CTA is in flight any more
+  // ---- teardown: every role has left its loops; nothing of this CTA is in flight any more
   umma::fence_before_sync();
   __syncthreads();
   if (warp == kMmaWarp) {
@@ -474,15 +543,24 @@ int launch_replay_attn_umma(const ReplayAttnParams& p, cudaStream_t stream) {
   const int pairs = (p.g + 1) / 2;
   ReplayAttnParams q = p;
   q.q_tiles = (p.t_max + kQRows - 1) / kQRows;
-  const int64_t ctas = (int64_t)p.L * p.B * p.Hkv * pairs * q.q_tiles;
-  if (ctas > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+  const int64_t items = (int64_t)p.L * p.B * p.Hkv * pairs * q.q_tiles;
+  if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
   static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
-  const int rc = attr_once.run([] {
-    return cudaFuncSetAttribute(replay_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-  });
+  static int sm_count[kMaxDevices] = {0};
+  int dev = -1;
+  const int rc = attr_once.run([&] {
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count[cur], cudaDevAttrMultiProcessorCount, cur);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(replay_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    return e;
+  }, &dev);
   if (rc != NGC_OK) return rc;
-  // One CTA per SM by construction (197 KB of shared memory each): a CTA owns all 512 columns of its SM's tensor memory.
-  replay_attn_umma_kernel<<<(unsigned)ctas, kThreads, kSmemBytes, stream>>>(q);
+  // One CTA per SM by construction (226 KB of shared memory each): a CTA owns all 512 columns of its SM's tensor
+  // memory, and walks the items blockIdx.x, blockIdx.x + gridDim.x, ...
+  const int grid = (int)(items < sm_count[dev] ? items : sm_count[dev]);
+  replay_attn_umma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(q, (int)items);
   return launch_status();
 }
 

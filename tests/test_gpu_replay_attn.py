@@ -101,4 +101,26 @@ def test_replay_attn_running_maximum_moves_many_times():
 
 def test_replay_attn_many_rounds_inside_one_query_tile():
     """Rounds every few tokens: a 128-token query tile straddles dozens of eviction rounds, each with its own kept list."""
-    run_case(1, 2, 2, 1, 0, 1, 30, 2, 6, tail=[9, 3], seed=13)
+    run_case(1, 2, 2, 1, 0, 1, 30, 5, 9, tail=[9, 3], seed=13)
+
+
+def test_replay_attn_more_rounds_in_a_tile_than_the_table_holds_is_reported():
+    """A round every other token puts more than 33 eviction rounds inside one 128-token query tile; the tcgen05 kernel
+    keeps a fixed table per tile, so it reports the sequence (bad counts) instead of computing a wrong answer silently,
+    and returns normally."""
+    b = ngc()
+    rng = np.random.default_rng(5)
+    R, B, G, L, Hq, Hkv, d = 50, 1, 1, 1, 2, 1, 128
+    ks, budget, alive_before, total_before = random_history(rng, R, B, G, 1, 2, 2)
+    pos, cnt, st0 = gpu_replay(ks, budget, alive_before, total_before, 1, int(alive_before.max()))
+    assert st0 == 0
+    T = int(total_before[-1, 0]) + 5
+    c = synth.make_cache(L, B, Hq, Hkv, d, torch.bfloat16, [T], capacity=T, seed=1)
+    dc = b.NgcCache(c.k.cuda(), c.v.cuda(), c.seq_off.cuda(), c.lens.cuda(), Hq, T)
+    q = synth.normal((L, B, Hq, T, d), 2, torch.bfloat16).cuda()
+    out = torch.zeros((L, B, Hq, T, d), dtype=torch.float32, device="cuda")
+    st = b.new_status()
+    b.ngc_replay_attn(dc, q, out, torch.as_tensor(pos).cuda(), torch.as_tensor(cnt).cuda(), torch.as_tensor(total_before).cuda(), status=st)
+    torch.cuda.synchronize()
+    assert status_value(st) == 1
+    assert bool(torch.isfinite(out).all())
