@@ -9,19 +9,25 @@
 //
 //   planner warp (1)     per item: which kept lists and which contiguous run the 128 queries see
 //                        (a small table in a two-slot ring), then the Q tiles of both heads into
-//                        shared memory as soon as the previous item's last S product has read them;
-//   producer warps (2)   gather 64-key K/V tiles by position (kept lists, then the contiguous block)
-//                        with 16-byte cp.async into a 4-stage ring, 128-byte swizzled, and publish a
-//                        stage with a proxy fence + mbarrier arrival once its copies have landed.  Tile
-//                        t - 1 is published right after tile t has been issued, BEFORE the producer may
-//                        block on a free stage: the MMA warp needs tile t + 1 to finish tile t, so a
-//                        producer that sat on landed tiles while waiting for a stage would deadlock;
-//   MMA warp (1 thread)  S_h = Q_h K^T (tcgen05.mma, M = 128, N = 64, both operands K-major) into a
-//                        double-buffered S in tensor memory, and O_h += P_h V (M = 128, N = 128, V as
-//                        MN-major B operand); completion is committed to mbarriers;
+//                        shared memory by tiled TMA as soon as the previous item's last S product has
+//                        read them;
+//   producer warps (4)   gather 64-key K/V tiles by position (kept lists, then the contiguous block)
+//                        with 16-byte cp.async into a 5-stage ring, 128-byte swizzled.  Every lane hands
+//                        its copies of a tile to the stage's mbarrier with cp.async.mbarrier.arrive.noinc:
+//                        the arrival fires when the copies have landed, nobody waits for it, so the
+//                        producers run a full ring ahead and a tile becomes visible to the MMA warp the
+//                        moment it is complete.  (Publishing from the producer after a cp.async wait
+//                        ties a tile's visibility to the issue of a later tile: the ring then runs in
+//                        lockstep with the consumer.  TMA row gathers, tile::gather4, were measured too:
+//                        about 80 cycles per four-row instruction, one 32 KB tile per 5000 cycles.)
+//   MMA warp (1 thread)  S_h = Q_h K^T (tcgen05.mma, M = 128, N = 64, both operands K-major in shared
+//                        memory) into a double-buffered S in tensor memory, and O_h += P_h V (M = 128,
+//                        N = 128, P read from TENSOR MEMORY as the A operand, V as MN-major B operand);
+//                        completion is committed to mbarriers;
 //   softmax warps (2x4)  one warpgroup per head, one thread per query row: S row from tensor memory
-//                        (tcgen05.ld), replay mask, online softmax in the log2 domain, P row as bf16
-//                        into 128-byte-swizzled shared memory for the second product.  The running
+//                        (tcgen05.ld), replay mask, online softmax in the log2 domain, P row as packed
+//                        bf16 back into the first 32 columns of the S buffer it came from (tcgen05.st),
+//                        so P never touches shared memory and is double-buffered with S.  The running
 //                        maximum used for the exponentials only moves when the true maximum has grown
 //                        by more than 8 (a factor 256, exact in bf16 / fp32), so the O accumulator in
 //                        tensor memory is rescaled rarely; when it is, the row's owner does it in place
@@ -32,8 +38,10 @@
 // one head while the other head's rows are in the softmax.  Every wait is bounded: a wait that runs
 // out raises a CTA-wide abort flag, every role leaves its loops, in-flight copies and MMAs are
 // drained (bounded again), tensor memory is freed and NGC_DEV_TIMEOUT is reported.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
+#include "kv_map.cuh"
 #include "ngc_common.cuh"
 #include "ptx.cuh"
 #include "replay_attn.cuh"
@@ -44,24 +52,24 @@ namespace {
 
 constexpr int kQRows = 128;                   // query tokens per item = tensor-memory lanes
 constexpr int kKeys = 64;                     // keys per pipeline stage
-constexpr int kStages = 4;
+constexpr int kStages = 5;
 constexpr int kMmaWarp = 8;                   // warps 0-7: softmax (two groups of four, one query head each)
-constexpr int kProducerWarp0 = 9;             // warps 9, 10
-constexpr int kProducerLanes = 64;
-constexpr int kPlannerWarp = 11;
-constexpr int kThreads = 12 * 32;
+constexpr int kPlannerWarp = 9;
+constexpr int kProducerWarp0 = 10;            // warps 10 .. 13
+constexpr int kProducerWarps = 4;
+constexpr int kProducerLanes = kProducerWarps * 32;
+constexpr int kThreads = (kProducerWarp0 + kProducerWarps) * 32;
 constexpr int kQHalf = kQRows * 128;          // one 64-channel half of a Q tile (128 rows x 128 B)
 constexpr int kQBytes = 2 * kQHalf;           // 32 KB per head
 constexpr int kKBox = kKeys * 128;            // 64 keys x 64 channels
 constexpr int kKTile = 2 * kKBox;             // K (or V) tile, 16 KB
 constexpr int kStageBytes = 2 * kKTile;       // K + V
-constexpr int kPBytes = kQRows * 128;         // P tile of a head: 128 rows x 64 keys of bf16
-constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 2 * kPBytes + 1024;
-constexpr uint32_t kTmemCols = 512;           // S[h][buf] at (2h + buf) * 64, O[h] at 256 + 128 h
+constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 1024;
+constexpr uint32_t kTmemCols = 512;           // S[h][buf] at (2h + buf) * 64 (P over its first 32 columns), O[h] at 256 + 128 h
 constexpr int kMaxSeg = 34;                   // rounds one query tile can straddle (+ the contiguous part)
 constexpr float kLazyRescale = 8.f;           // log2 units the row maximum may grow before O is rescaled
 constexpr int kPlanSlots = 2;
-constexpr int kPlanReaders = 8 + 1 + 2;       // one arrival per softmax warp, the MMA thread, per producer warp
+constexpr int kPlanReaders = 8 + 1 + kProducerWarps;   // one arrival per softmax warp, the MMA thread, per producer warp
 
 // What the roles need to know about one item.
 struct Plan {
@@ -73,7 +81,7 @@ struct Plan {
 };
 
 struct Shared {
-  uint64_t kv_full[kStages], kv_empty[kStages], s_full[2][2], p_full[2], o_done[2];
+  uint64_t kv_full[kStages], kv_empty[kStages], s_full[2][2], p_full[2][2], o_done[2][2];
   uint64_t q_full, q_empty, plan_full[kPlanSlots], plan_empty[kPlanSlots], drain;
   uint32_t tmem;
   int abort;
@@ -101,19 +109,27 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, Shared
   return __all_sync(0xffffffffu, wait_or_abort(bar, parity, sh, dev_status));
 }
 
-// swizzled byte offset of 16-byte piece c (0..15) of row r inside a tile of `half_bytes`-sized 64-channel halves
-__device__ __forceinline__ uint32_t tile_off(int half_bytes, int r, int c) {
-  return (uint32_t)((c >> 3) * half_bytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+// Tensor map of a launch: Q as a 2-D tensor (channel, row over all layers / sequences / heads), box = 64 channels x 128 rows.
+struct Maps { CUtensorMap q; };
+
+// swizzled byte offset of 16-byte piece c (0..15) of key row r inside a K or V tile
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+  return (uint32_t)((c >> 3) * kKBox + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(ptx::smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(ptx::smem_u32(bar))
+               : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAttnParams p, int n_items) {
+__global__ void __launch_bounds__(kThreads, 1)
+replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, int n_items) {
   extern __shared__ uint8_t smem_dyn[];
   __shared__ Shared sh;
 
   uint8_t* base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = base;                                   // [2 heads][32 KB]
   uint8_t* stage = sQ + 2 * kQBytes;                    // [kStages][K 16 KB | V 16 KB]
-  uint8_t* sP = stage + kStages * kStageBytes;          // [2 heads][16 KB]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int pairs = (p.g + 1) >> 1;
 
@@ -123,15 +139,17 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
       ptx::mbar_init(&sh.s_full[hh][0], 1); ptx::mbar_init(&sh.s_full[hh][1], 1);
-      ptx::mbar_init(&sh.p_full[hh], 128); ptx::mbar_init(&sh.o_done[hh], 1);
+      ptx::mbar_init(&sh.p_full[hh][0], 128); ptx::mbar_init(&sh.p_full[hh][1], 128);
+      ptx::mbar_init(&sh.o_done[hh][0], 1); ptx::mbar_init(&sh.o_done[hh][1], 1);
     }
 #pragma unroll
     for (int s = 0; s < kPlanSlots; ++s) { ptx::mbar_init(&sh.plan_full[s], 1); ptx::mbar_init(&sh.plan_empty[s], kPlanReaders); }
-    ptx::mbar_init(&sh.q_full, 32);
+    ptx::mbar_init(&sh.q_full, 1);
     ptx::mbar_init(&sh.q_empty, 1);
     ptx::mbar_init(&sh.drain, 1);
     ptx::fence_barrier_init();
     sh.abort = 0;
+    ptx::prefetch_tensormap(&maps.q);
   }
   if (warp == kMmaWarp) umma::tmem_alloc(&sh.tmem, kTmemCols);
   umma::fence_before_sync();
@@ -227,35 +245,24 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
       // Q tiles of the two heads -> shared memory (rows beyond the sequence: zeros), once the previous item's
       // last S product has read the buffer
       if (n_q >= 1 && !warp_wait(&sh.q_empty, (n_q - 1) & 1, &sh, p.dev_status)) break;
-      const int n_heads = has1 ? 2 : 1;
-      for (int i = lane; i < n_heads * kQRows * 16; i += 32) {
-        const int hh = i / (kQRows * 16), rest = i - hh * kQRows * 16;
-        const int r = rest >> 4, c = rest & 15;
-        uint8_t* dst = sQ + hh * kQBytes + tile_off(kQHalf, r, c);
-        const int t = q0 + r;
-        if (t < T_b) {
-          const __nv_bfloat16* src = p.q + ((((int64_t)l * p.B + b) * p.Hq + hq0 + hh) * (int64_t)p.t_max + t) * 128 + 8 * c;
-          ptx::cp_async_cg_16(ptx::smem_u32(dst), src);
-        } else {
-          *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+      if (lane == 0) {
+        // rows beyond the sequence (or beyond t_max: the next head's rows, zeros past the end of the tensor) only feed
+        // the S rows of queries that do not exist and are never written
+        const int n_heads = has1 ? 2 : 1;
+        ptx::mbar_expect_tx(&sh.q_full, (uint32_t)(n_heads * kQBytes));
+        for (int hh = 0; hh < n_heads; ++hh) {
+          const int y = (int)((((int64_t)l * p.B + b) * p.Hq + hq0 + hh) * (int64_t)p.t_max + q0);
+          tma_load_2d(sQ + hh * kQBytes, &maps.q, 0, y, &sh.q_full);
+          tma_load_2d(sQ + hh * kQBytes + kQHalf, &maps.q, 64, y, &sh.q_full);
         }
       }
-      ptx::cp_async_commit();
-      ptx::cp_async_wait_group<0>();
-      ptx::fence_proxy_async();
-      ptx::mbar_arrive(&sh.q_full);
+      __syncwarp();
       ++n_q;
     }
-    ptx::cp_async_wait_group<0>();
   } else if (warp >= kProducerWarp0) {
-    // ------------------------------------------------------------------ producers
-    const int ptid = tid - kProducerWarp0 * 32;
-    const int pw = ptid >> 5;                           // producer warp w gathers rows 32 w .. 32 w + 31 of a tile
-    int issued = 0, published = 0;                      // tiles, over all items
-    auto publish = [&](int t) {                         // this lane's copies of tile t have landed
-      ptx::fence_proxy_async();
-      ptx::mbar_arrive(&sh.kv_full[t % kStages]);
-    };
+    // ------------------------------------------------------------------ producers: cp.async gathers
+    const int pw = warp - kProducerWarp0;               // producer warp w gathers key rows 16 w .. 16 w + 15 of a tile
+    int issued = 0;                                     // tiles, over all items
     bool ok = true;
     int k = 0;
     for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x, ++k) {
@@ -265,58 +272,50 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
       const int n_tiles = pl.n_tiles, nseg = pl.nseg, c_lo = pl.c_lo, T_b = pl.T_b, b = pl.b, gi = pl.gi;
       const __nv_bfloat16* k_strip = p.k + ((int64_t)(pl.l * p.Hkv + pl.h) * p.rows_R + p.seq_off[b]) * 128;
       const __nv_bfloat16* v_strip = p.v + ((int64_t)(pl.l * p.Hkv + pl.h) * p.rows_R + p.seq_off[b]) * 128;
-      // position of key row 32 pw + lane of tile i (-1: no such key, -2: a kept position outside the sequence);
-      // one coalesced load per lane and tile, fetched one tile ahead
+      // position of key row 16 pw + (lane & 15) of tile i, one coalesced load per tile, fetched one tile ahead.  A row
+      // the tile does not have (beyond the segment's end) is fetched from position 0 of the sequence: live data that
+      // the mask gives weight 0 (every byte of a stage comes through cp.async, so the mbarrier hand-over covers it);
+      // a kept position outside the sequence is reported and treated the same way.
       int sgi = 0;
       auto tile_pos = [&](int i) {
         while (sgi + 1 < nseg && i >= pl.seg_first[sgi + 1]) ++sgi;
         const int rho = pl.seg_rho[sgi], n = pl.seg_n[sgi];
-        const int kidx = (i - pl.seg_first[sgi]) * kKeys + 32 * pw + lane;
-        if (kidx >= n) return -1;
+        const int kidx = (i - pl.seg_first[sgi]) * kKeys + 16 * pw + (lane & 15);
+        if (kidx >= n) return 0;
         const int pos = rho >= 1 ? p.alive_pos[(((int64_t)(rho - 1) * p.B + b) * p.G + gi) * p.kt_max + kidx] : c_lo + kidx;
-        return (pos >= 0 && pos < T_b) ? pos : -2;
+        if (pos >= 0 && pos < T_b) return pos;
+        set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
+        return 0;
       };
-      int pos_next = n_tiles > 0 ? tile_pos(0) : -1;
+      int pos_next = n_tiles > 0 ? tile_pos(0) : 0;
       for (int i = 0; i < n_tiles; ++i) {
         const int s = issued % kStages;
         const int pos_mine = pos_next;
         if (i + 1 < n_tiles) pos_next = tile_pos(i + 1);
-        if (pos_mine == -2) set_dev_status(p.dev_status, NGC_DEV_BAD_KEPT);
         if (issued >= kStages && !warp_wait(&sh.kv_empty[s], ((issued / kStages) - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
         uint8_t* st = stage + s * kStageBytes;
         const int c = lane & 15;
-#pragma unroll 4
-        for (int u = 0; u < 16; ++u) {                  // two rows per step, 16 lanes (16-byte pieces) per row
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {                   // two rows per step, 16 lanes (16-byte pieces) per row
           const int rl = 2 * u + (lane >> 4);
           const int pos = __shfl_sync(0xffffffffu, pos_mine, rl);
-          const int row = 32 * pw + rl;
-          const uint32_t off = tile_off(kKBox, row, c);
-          if (pos >= 0) {
-            ptx::cp_async_cg_16(ptx::smem_u32(st + off), k_strip + (int64_t)pos * 128 + 8 * c);
-            ptx::cp_async_cg_16(ptx::smem_u32(st + kKTile + off), v_strip + (int64_t)pos * 128 + 8 * c);
-          } else {    // past the end of the source: zeros (a stale NaN times P = 0 would poison the sum)
-            *reinterpret_cast<uint4*>(st + off) = make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4*>(st + kKTile + off) = make_uint4(0, 0, 0, 0);
-          }
+          const uint32_t off = tile_off(16 * pw + rl, c);
+          ptx::cp_async_cg_16(ptx::smem_u32(st + off), k_strip + (int64_t)pos * 128 + 8 * c);
+          ptx::cp_async_cg_16(ptx::smem_u32(st + kKTile + off), v_strip + (int64_t)pos * 128 + 8 * c);
         }
-        ptx::cp_async_commit();
+        ptx::cp_async_mbar_arrive_noinc(&sh.kv_full[s]);    // counts as this lane's arrival once its copies have landed
         ++issued;
-        if (issued - published > 1) {                   // everything but the tile just issued has landed
-          ptx::cp_async_wait_group<1>();
-          publish(published++);
-        }
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&sh.plan_empty[slot]);
     }
-    ptx::cp_async_wait_group<0>();
-    if (issued - published == 1) publish(published++);
+    ptx::cp_async_wait_all();
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issue (one thread)
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma::instr_desc(kQRows, kKeys, false);
       constexpr uint32_t idesc_o = umma::instr_desc(kQRows, 128, true);
-      const uint32_t q_addr = ptx::smem_u32(sQ), p_addr = ptx::smem_u32(sP), st_addr = ptx::smem_u32(stage);
+      const uint32_t q_addr = ptx::smem_u32(sQ), st_addr = ptx::smem_u32(stage);
       int t0 = 0, t1 = 0, n_q = 0;                      // tiles so far (head 0 = all, head 1), items with tiles so far
       bool ok = true;
       int k = 0;
@@ -353,20 +352,22 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
             ok = wait_or_abort(&sh.kv_full[(t + 1) % kStages], ((t + 1) / kStages) & 1, &sh, p.dev_status);
             if (!ok) break;
             umma::fence_after_sync();
-            issue_s(i + 1);                             // its S buffer was read out before P of two tiles ago was published
+            issue_s(i + 1);                             // its buffer held S and P of two tiles ago: that P V product was issued
+                                                        // before this one, and the tensor pipe runs them in issue order
           }
           const uint32_t v_addr = st_addr + (t % kStages) * kStageBytes + kKTile;
           for (int hh = 0; hh < n_heads; ++hh) {
-            ok = wait_or_abort(&sh.p_full[hh], ((hh ? t1 : t0) + i) & 1, &sh, p.dev_status);
+            const int th = (hh ? t1 : t0) + i;          // tile count of this head: P sits in S buffer th & 1, use th >> 1 of it
+            ok = wait_or_abort(&sh.p_full[hh][th & 1], (th >> 1) & 1, &sh, p.dev_status);
             if (!ok) break;
             umma::fence_after_sync();
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {            // 16 keys per step
-              const uint64_t a = umma::smem_desc_sw128(p_addr + hh * kPBytes + kk * 32, 16, 1024);
+              const uint32_t a = tmem + (uint32_t)((2 * hh + (th & 1)) * kKeys + 8 * kk);    // 16 keys = 8 packed columns of P
               const uint64_t bd = umma::smem_desc_sw128(v_addr + kk * 2048, kKBox, 1024);   // next 64 channels: one box on
-              umma::mma_bf16(tmem + 256u + 128u * hh, a, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+              umma::mma_bf16_a_tmem(tmem + 256u + 128u * hh, a, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
             }
-            umma::commit(&sh.o_done[hh]);
+            umma::commit(&sh.o_done[hh][th & 1]);
           }
           if (!ok) break;
           umma::commit(&sh.kv_empty[t % kStages]);      // K and V of this stage have been consumed
@@ -386,7 +387,6 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
     const int row = 32 * (warp & 3) + lane;
     const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
     const uint32_t o_addr = tmem + lane_base + 256u + 128u * hh;
-    uint8_t* p_row = sP + hh * kPBytes + row * 128;
     int tc = 0;                                         // tiles this head has been through, over all items
     bool ok = true;
     int k = 0;
@@ -405,7 +405,7 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
           if (tb <= t_q) { blk += 1; lo_row = tb; }
         }
         float m_use = -INFINITY, l_run = 0.f;
-        int o_seen = tc - 1;                            // last tile whose P V product is known to be complete
+        int o_seen = tc - 1;                            // last tile whose P V product is known to be complete (they complete in order)
         int sgi = 0;
         for (int i = 0; i < n_tiles; ++i) {
           const int t = tc + i;
@@ -452,7 +452,7 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
           const bool rescale = grow && m_use != -INFINITY && i > 0;           // O already holds something for this row
           if (__any_sync(0xffffffffu, rescale)) {
             if (o_seen < t - 1) {
-              if (!warp_wait(&sh.o_done[hh], (t - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+              if (!warp_wait(&sh.o_done[hh][(t - 1) & 1], ((t - 1) >> 1) & 1, &sh, p.dev_status)) { ok = false; break; }
               o_seen = t - 1;
               umma::fence_after_sync();
             }
@@ -481,20 +481,15 @@ __global__ void __launch_bounds__(kThreads, 1) replay_attn_umma_kernel(ReplayAtt
               l_run += p0 + p1;
               pk[16 * half + (j >> 1)] = ptx::pack_bf16x2(p0, p1);
             }
-          if (t > 0 && o_seen < t - 1) {                                      // the P tile is free once the previous P V has completed
-            if (!warp_wait(&sh.o_done[hh], (t - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
-            o_seen = t - 1;
-          }
-#pragma unroll
-          for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(p_row + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-          ptx::fence_proxy_async();
+          // P over the first 32 columns of the S buffer this row was just read from (free: the row is in registers)
+          umma::tmem_st32(s_addr, pk);
+          umma::tmem_st_wait();
           umma::fence_before_sync();
-          ptx::mbar_arrive(&sh.p_full[hh]);
+          ptx::mbar_arrive(&sh.p_full[hh][t & 1]);
         }
         if (!ok) break;
         tc += n_tiles;
-        if (!warp_wait(&sh.o_done[hh], (tc - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+        if (!warp_wait(&sh.o_done[hh][(tc - 1) & 1], ((tc - 1) >> 1) & 1, &sh, p.dev_status)) { ok = false; break; }
         umma::fence_after_sync();
         const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
         const int64_t o_base = ((((int64_t)pl.l * p.B + pl.b) * p.Hq + pl.hq0 + hh) * (int64_t)p.t_max + t_q) * 128;
@@ -545,6 +540,9 @@ int launch_replay_attn_umma(const ReplayAttnParams& p, cudaStream_t stream) {
   q.q_tiles = (p.t_max + kQRows - 1) / kQRows;
   const int64_t items = (int64_t)p.L * p.B * p.Hkv * pairs * q.q_tiles;
   if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
+  // TMA coordinates are 32-bit: the queries are addressed by row over all layers, sequences and heads
+  Maps maps;
+  if (!make_rows_map(&maps.q, p.q, (int64_t)p.L * p.B * p.Hq * p.t_max, kQRows)) return NGC_ERR_UNSUPPORTED;
   static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
   static int sm_count[kMaxDevices] = {0};
   int dev = -1;
@@ -560,7 +558,7 @@ int launch_replay_attn_umma(const ReplayAttnParams& p, cudaStream_t stream) {
   // One CTA per SM by construction (226 KB of shared memory each): a CTA owns all 512 columns of its SM's tensor
   // memory, and walks the items blockIdx.x, blockIdx.x + gridDim.x, ...
   const int grid = (int)(items < sm_count[dev] ? items : sm_count[dev]);
-  replay_attn_umma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(q, (int)items);
+  replay_attn_umma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(maps, q, (int)items);
   return launch_status();
 }
 
