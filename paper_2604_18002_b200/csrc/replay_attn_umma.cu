@@ -20,7 +20,8 @@
 //                        ties a tile's visibility to the issue of a later tile: the ring then runs in
 //                        lockstep with the consumer.  TMA row gathers, tile::gather4, were measured too:
 //                        about 80 cycles per four-row instruction, one 32 KB tile per 5000 cycles.)
-//   MMA warp (1 thread)  S_h = Q_h K^T (tcgen05.mma, M = 128, N = 64, both operands K-major in shared
+//   MMA warps (2 x 1 thread, one per head)
+//                        S_h = Q_h K^T (tcgen05.mma, M = 128, N = 64, both operands K-major in shared
 //                        memory) into a double-buffered S in tensor memory, and O_h += P_h V (M = 128,
 //                        N = 128, P read from TENSOR MEMORY as the A operand, V as MN-major B operand);
 //                        completion is committed to mbarriers;
@@ -53,9 +54,10 @@ namespace {
 constexpr int kQRows = 128;                   // query tokens per item = tensor-memory lanes
 constexpr int kKeys = 64;                     // keys per pipeline stage
 constexpr int kStages = 5;
-constexpr int kMmaWarp = 8;                   // warps 0-7: softmax (two groups of four, one query head each)
-constexpr int kPlannerWarp = 9;
-constexpr int kProducerWarp0 = 10;            // warps 10 .. 13
+constexpr int kMmaWarp = 8;                   // warps 0-7: softmax (two groups of four, one query head each);
+                                              // warps 8, 9: one MMA-issuing thread per head
+constexpr int kPlannerWarp = 10;
+constexpr int kProducerWarp0 = 11;            // warps 11 .. 14
 constexpr int kProducerWarps = 4;
 constexpr int kProducerLanes = kProducerWarps * 32;
 constexpr int kThreads = (kProducerWarp0 + kProducerWarps) * 32;
@@ -69,7 +71,7 @@ constexpr uint32_t kTmemCols = 512;           // S[h][buf] at (2h + buf) * 64 (P
 constexpr int kMaxSeg = 34;                   // rounds one query tile can straddle (+ the contiguous part)
 constexpr float kLazyRescale = 8.f;           // log2 units the row maximum may grow before O is rescaled
 constexpr int kPlanSlots = 2;
-constexpr int kPlanReaders = 8 + 1 + kProducerWarps;   // one arrival per softmax warp, the MMA thread, per producer warp
+constexpr int kPlanReaders = 8 + 2 + kProducerWarps;   // one arrival per softmax warp, per MMA thread, per producer warp
 
 // What the roles need to know about one item.
 struct Plan {
@@ -82,7 +84,7 @@ struct Plan {
 
 struct Shared {
   uint64_t kv_full[kStages], kv_empty[kStages], s_full[2][2], p_full[2][2], o_done[2][2];
-  uint64_t q_full, q_empty, plan_full[kPlanSlots], plan_empty[kPlanSlots], drain;
+  uint64_t q_full, q_empty, plan_full[kPlanSlots], plan_empty[kPlanSlots], drain[2];
   uint32_t tmem;
   int abort;
   Plan plan[kPlanSlots];
@@ -135,7 +137,7 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
 
   if (tid == 0) {
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&sh.kv_full[s], kProducerLanes); ptx::mbar_init(&sh.kv_empty[s], 1); }
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&sh.kv_full[s], kProducerLanes); ptx::mbar_init(&sh.kv_empty[s], 2); }
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
       ptx::mbar_init(&sh.s_full[hh][0], 1); ptx::mbar_init(&sh.s_full[hh][1], 1);
@@ -145,8 +147,9 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
 #pragma unroll
     for (int s = 0; s < kPlanSlots; ++s) { ptx::mbar_init(&sh.plan_full[s], 1); ptx::mbar_init(&sh.plan_empty[s], kPlanReaders); }
     ptx::mbar_init(&sh.q_full, 1);
-    ptx::mbar_init(&sh.q_empty, 1);
-    ptx::mbar_init(&sh.drain, 1);
+    ptx::mbar_init(&sh.q_empty, 2);
+    ptx::mbar_init(&sh.drain[0], 1);
+    ptx::mbar_init(&sh.drain[1], 1);
     ptx::fence_barrier_init();
     sh.abort = 0;
     ptx::prefetch_tensormap(&maps.q);
@@ -310,75 +313,87 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
       if (lane == 0) ptx::mbar_arrive(&sh.plan_empty[slot]);
     }
     ptx::cp_async_wait_all();
-  } else if (warp == kMmaWarp) {
-    // ------------------------------------------------------------------ MMA issue (one thread)
+  } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
+    // ------------------------------------------------------------------ MMA issue: one thread per head
+    // Two issuing threads halve the serial issue path (descriptors, waits, fences, commits) per tile; the tensor
+    // pipe takes their instructions as they come.  Both threads release a K/V stage and the Q buffer (two
+    // arrivals each); for an item without a second head the thread of head 1 just passes the arrivals on.
+    const int hh = warp - kMmaWarp;
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma::instr_desc(kQRows, kKeys, false);
       constexpr uint32_t idesc_o = umma::instr_desc(kQRows, 128, true);
-      const uint32_t q_addr = ptx::smem_u32(sQ), st_addr = ptx::smem_u32(stage);
-      int t0 = 0, t1 = 0, n_q = 0;                      // tiles so far (head 0 = all, head 1), items with tiles so far
+      const uint32_t q_addr = ptx::smem_u32(sQ) + hh * kQBytes, st_addr = ptx::smem_u32(stage);
+      const uint32_t o_tmem = tmem + 256u + 128u * hh;
+      int t0 = 0, th = 0, n_q = 0;                      // tiles so far (all items / items with this head), items with tiles so far
       bool ok = true;
       int k = 0;
       for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x, ++k) {
         const int slot = k & 1;
         if (!wait_or_abort(&sh.plan_full[slot], (k >> 1) & 1, &sh, p.dev_status)) break;
         const int n_tiles = sh.plan[slot].n_tiles;
-        const int n_heads = sh.plan[slot].has1 ? 2 : 1;
+        const bool mine = hh == 0 || sh.plan[slot].has1;
         ptx::mbar_arrive(&sh.plan_empty[slot]);         // nothing else of the table is needed here
         if (n_tiles == 0) continue;
-        auto issue_s = [&](int i) {                     // S_h = Q_h K^T for tile i of this item, into the head's next S buffer
-          const uint32_t k_addr = st_addr + ((t0 + i) % kStages) * kStageBytes;
-          for (int hh = 0; hh < n_heads; ++hh) {
-            const int buf = ((hh ? t1 : t0) + i) & 1;
-            const uint32_t d = tmem + (uint32_t)((2 * hh + buf) * kKeys);
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              const uint64_t a = umma::smem_desc_sw128(q_addr + hh * kQBytes + (ks >> 2) * kQHalf + (ks & 3) * 32, 16, 1024);
-              const uint64_t bd = umma::smem_desc_sw128(k_addr + (ks >> 2) * kKBox + (ks & 3) * 32, 16, 1024);
-              umma::mma_bf16(d, a, bd, idesc_s, ks > 0);
-            }
-            umma::commit(&sh.s_full[hh][buf]);
+        ok = wait_or_abort(&sh.q_full, n_q & 1, &sh, p.dev_status);      // (also: the previous use of q_empty is over)
+        if (!ok) break;
+        if (!mine) {
+          // nothing to multiply: hand on this thread's share of the releases, each after the tile has landed (so
+          // that the arrival cannot fall into an earlier phase of the stage's barrier)
+          ptx::mbar_arrive(&sh.q_empty);
+          for (int i = 0; i < n_tiles && ok; ++i) {
+            const int t = t0 + i;
+            ok = wait_or_abort(&sh.kv_full[t % kStages], (t / kStages) & 1, &sh, p.dev_status);
+            if (ok) ptx::mbar_arrive(&sh.kv_empty[t % kStages]);
           }
+          t0 += n_tiles;
+          ++n_q;
+          continue;
+        }
+        auto issue_s = [&](int i) {                     // S = Q K^T for tile i of this item, into the head's next S buffer
+          const uint32_t k_addr = st_addr + ((t0 + i) % kStages) * kStageBytes;
+          const int buf = (th + i) & 1;
+          const uint32_t d = tmem + (uint32_t)((2 * hh + buf) * kKeys);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint64_t a = umma::smem_desc_sw128(q_addr + (ks >> 2) * kQHalf + (ks & 3) * 32, 16, 1024);
+            const uint64_t bd = umma::smem_desc_sw128(k_addr + (ks >> 2) * kKBox + (ks & 3) * 32, 16, 1024);
+            umma::mma_bf16(d, a, bd, idesc_s, ks > 0);
+          }
+          umma::commit(&sh.s_full[hh][buf]);
           if (i == n_tiles - 1) umma::commit(&sh.q_empty);     // the item's last product that reads Q
         };
-        ok = wait_or_abort(&sh.q_full, n_q & 1, &sh, p.dev_status) &&
-             wait_or_abort(&sh.kv_full[t0 % kStages], (t0 / kStages) & 1, &sh, p.dev_status);
+        ok = wait_or_abort(&sh.kv_full[t0 % kStages], (t0 / kStages) & 1, &sh, p.dev_status);
         if (!ok) break;
-        umma::fence_after_sync();
         issue_s(0);
         for (int i = 0; i < n_tiles; ++i) {
           const int t = t0 + i;
           if (i + 1 < n_tiles) {
             ok = wait_or_abort(&sh.kv_full[(t + 1) % kStages], ((t + 1) / kStages) & 1, &sh, p.dev_status);
             if (!ok) break;
-            umma::fence_after_sync();
             issue_s(i + 1);                             // its buffer held S and P of two tiles ago: that P V product was issued
                                                         // before this one, and the tensor pipe runs them in issue order
           }
           const uint32_t v_addr = st_addr + (t % kStages) * kStageBytes + kKTile;
-          for (int hh = 0; hh < n_heads; ++hh) {
-            const int th = (hh ? t1 : t0) + i;          // tile count of this head: P sits in S buffer th & 1, use th >> 1 of it
-            ok = wait_or_abort(&sh.p_full[hh][th & 1], (th >> 1) & 1, &sh, p.dev_status);
-            if (!ok) break;
-            umma::fence_after_sync();
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {            // 16 keys per step
-              const uint32_t a = tmem + (uint32_t)((2 * hh + (th & 1)) * kKeys + 8 * kk);    // 16 keys = 8 packed columns of P
-              const uint64_t bd = umma::smem_desc_sw128(v_addr + kk * 2048, kKBox, 1024);   // next 64 channels: one box on
-              umma::mma_bf16_a_tmem(tmem + 256u + 128u * hh, a, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
-            }
-            umma::commit(&sh.o_done[hh][th & 1]);
-          }
+          const int tt = th + i;                        // tile count of this head: P sits in S buffer tt & 1, use tt >> 1 of it
+          ok = wait_or_abort(&sh.p_full[hh][tt & 1], (tt >> 1) & 1, &sh, p.dev_status);
           if (!ok) break;
-          umma::commit(&sh.kv_empty[t % kStages]);      // K and V of this stage have been consumed
+          umma::fence_after_sync();                     // P was written with tcgen05.st by the softmax threads
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {              // 16 keys per step
+            const uint32_t a = tmem + (uint32_t)((2 * hh + (tt & 1)) * kKeys + 8 * kk);     // 16 keys = 8 packed columns of P
+            const uint64_t bd = umma::smem_desc_sw128(v_addr + kk * 2048, kKBox, 1024);    // next 64 channels: one box on
+            umma::mma_bf16_a_tmem(o_tmem, a, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma::commit(&sh.o_done[hh][tt & 1]);
+          umma::commit(&sh.kv_empty[t % kStages]);      // this head is done with K and V of the stage
         }
         t0 += n_tiles;
-        if (n_heads == 2) t1 += n_tiles;
+        th += n_tiles;
         ++n_q;
       }
       // everything issued has completed before tensor memory is released
-      umma::commit(&sh.drain);
-      wait_or_abort(&sh.drain, 0, &sh, p.dev_status);
+      umma::commit(&sh.drain[hh]);
+      wait_or_abort(&sh.drain[hh], 0, &sh, p.dev_status);
     }
     __syncwarp();
   } else {
