@@ -300,7 +300,10 @@ int replay_attn_impl(const ngc_cache* c, const void* q, int t_max,
   p.G = lists_G(lists, c->L, c->Hkv); p.kt_max = kt_max; p.lists = lists; p.out_bf16 = out_dtype == NGC_BF16;
   p.q_tiles = (t_max + kQTile - 1) / kQTile;
   p.scale_log2 = scale * 1.4426950408889634f;
-  if (variant != NGC_REPLAY_ATTN_MMA_SYNC) return launch_replay_attn_umma(p, stream);
+  // the tcgen05 kernel takes row maxima on the raw scores, which needs a positive scale; anything else (and an
+  // explicit request) runs on the warp-level kernel
+  if (variant == NGC_REPLAY_ATTN_TCGEN05 && !(scale > 0.f)) return NGC_ERR_UNSUPPORTED;
+  if (variant != NGC_REPLAY_ATTN_MMA_SYNC && scale > 0.f) return launch_replay_attn_umma(p, stream);
   const int64_t ctas = (int64_t)c->L * c->B * c->Hq * p.q_tiles;
   if (ctas > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
   const int smem = 2 * kStageBytes + 1024;

@@ -90,6 +90,29 @@ struct Shared {
   Plan plan[kPlanSlots];
 };
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// two floats in one 64-bit register for the packed fp32 instructions (fma / add on both halves at once)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // Bounded wait that also gives up as soon as another thread of the CTA has given up.
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Shared* sh, int32_t* dev_status) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
@@ -437,7 +460,8 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
           // a tile needs no mask when every query of the item lies in one block and the tile is a full tile of that
           // block's kept list, or lies entirely before the first query
           const bool need_mask = !uniform || (rho >= 1 ? n_here < kKeys : c_lo + kt * kKeys + kKeys - 1 > q0);
-          float mx = -INFINITY;
+          // raw scores stay as they are; invisible ones become -inf.  The row maximum is taken on the raw values
+          // (the scale is positive) with three-input max over four independent chains.
           if (need_mask) {
             const int j0 = c_lo + kt * kKeys;
 #pragma unroll
@@ -448,20 +472,19 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
                 bool vis;
                 if (rho >= 1) vis = jj < n_here && blk == rho;                 // a kept entry of the round before this row's block
                 else vis = j0 + jj >= lo_row && j0 + jj <= t_q;                // a token of the row's own block, causal
-                const float z = vis ? __uint_as_float(zr[half][j]) * p.scale_log2 : -INFINITY;
-                zr[half][j] = __float_as_uint(z);
-                mx = fmaxf(mx, z);
-              }
-          } else {
-#pragma unroll
-            for (int half = 0; half < 2; ++half)
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float z = __uint_as_float(zr[half][j]) * p.scale_log2;
-                zr[half][j] = __float_as_uint(z);
-                mx = fmaxf(mx, z);
+                if (!vis) zr[half][j] = 0xff800000u;                           // -inf
               }
           }
+          float mxc[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+#pragma unroll
+              for (int c = 0; c < 4; ++c)
+                mxc[c] = max3(mxc[c], __uint_as_float(zr[half][j + 2 * c]), __uint_as_float(zr[half][j + 2 * c + 1]));
+            }
+          const float mx = fmaxf(fmaxf(mxc[0], mxc[1]), fmaxf(mxc[2], mxc[3])) * p.scale_log2;
           // the maximum used for the exponentials follows the true one lazily
           const bool grow = mx > m_use + kLazyRescale;                        // also the first visible key (m_use = -inf)
           const bool rescale = grow && m_use != -INFINITY && i > 0;           // O already holds something for this row
@@ -486,16 +509,26 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
           }
           if (grow) m_use = mx;
           const float m_eff = m_use == -INFINITY ? 0.f : m_use;               // nothing visible yet: every exponential is 0
+          // p = 2^(z * scale - m): one packed fused multiply-add per pair of scores, then the exponentials; the row sum
+          // in four independent packed chains
+          const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_eff, -m_eff);
+          uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
           uint32_t pk[32];
 #pragma unroll
           for (int half = 0; half < 2; ++half)
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
-              const float p0 = ptx::ex2_approx(__uint_as_float(zr[half][j]) - m_eff);
-              const float p1 = ptx::ex2_approx(__uint_as_float(zr[half][j + 1]) - m_eff);
-              l_run += p0 + p1;
+              float x0, x1;
+              unpack2(fma2(pack2(__uint_as_float(zr[half][j]), __uint_as_float(zr[half][j + 1])), sc2, nm2), x0, x1);
+              const float p0 = ptx::ex2_approx(x0), p1 = ptx::ex2_approx(x1);
+              acc2[(j >> 1) & 3] = add2(acc2[(j >> 1) & 3], pack2(p0, p1));
               pk[16 * half + (j >> 1)] = ptx::pack_bf16x2(p0, p1);
             }
+          {
+            float s0, s1;
+            unpack2(add2(add2(acc2[0], acc2[1]), add2(acc2[2], acc2[3])), s0, s1);
+            l_run += s0 + s1;
+          }
           // P over the first 32 columns of the S buffer this row was just read from (free: the row is in registers)
           umma::tmem_st32(s_addr, pk);
           umma::tmem_st_wait();
