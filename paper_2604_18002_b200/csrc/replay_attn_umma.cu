@@ -345,9 +345,16 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma::instr_desc(kQRows, kKeys, false);
       constexpr uint32_t idesc_o = umma::instr_desc(kQRows, 128, true);
-      const uint32_t q_addr = ptx::smem_u32(sQ) + hh * kQBytes, st_addr = ptx::smem_u32(stage);
+      const uint32_t st_addr = ptx::smem_u32(stage);
       const uint32_t o_tmem = tmem + 256u + 128u * hh;
+      // Operand descriptors differ only in their low word (start address / 16): the Q descriptors of the eight
+      // 16-channel steps are fixed, those of K and V follow the stage.  High word: stride 1024 bytes between 8-row
+      // groups, descriptor version 1, 128-byte swizzle.
+      const uint64_t desc_hi = (uint64_t)umma::smem_desc_sw128(0, 0, 1024) & 0xffffffff00000000ull;
+      const uint32_t q_lo = ((ptx::smem_u32(sQ) + hh * kQBytes) >> 4) | (1u << 16);      // leading offset 16 bytes (unused with swizzle)
+      const uint32_t v_lbo = (uint32_t)(kKBox >> 4) << 16;                                // V: the next 64 channels are one box on
       int t0 = 0, th = 0, n_q = 0;                      // tiles so far (all items / items with this head), items with tiles so far
+      int st_cur = 0, ph_cur = 0;                       // stage and phase parity of tile t0
       bool ok = true;
       int k = 0;
       for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x, ++k) {
@@ -364,51 +371,51 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
           // that the arrival cannot fall into an earlier phase of the stage's barrier)
           ptx::mbar_arrive(&sh.q_empty);
           for (int i = 0; i < n_tiles && ok; ++i) {
-            const int t = t0 + i;
-            ok = wait_or_abort(&sh.kv_full[t % kStages], (t / kStages) & 1, &sh, p.dev_status);
-            if (ok) ptx::mbar_arrive(&sh.kv_empty[t % kStages]);
+            ok = wait_or_abort(&sh.kv_full[st_cur], ph_cur, &sh, p.dev_status);
+            if (ok) ptx::mbar_arrive(&sh.kv_empty[st_cur]);
+            if (++st_cur == kStages) { st_cur = 0; ph_cur ^= 1; }
           }
           t0 += n_tiles;
           ++n_q;
           continue;
         }
-        auto issue_s = [&](int i) {                     // S = Q K^T for tile i of this item, into the head's next S buffer
-          const uint32_t k_addr = st_addr + ((t0 + i) % kStages) * kStageBytes;
-          const int buf = (th + i) & 1;
+        auto issue_s = [&](int stg, int buf, bool last) {      // S = Q K^T for the tile in stage stg, into S buffer buf
+          const uint32_t k_lo = ((st_addr + stg * kStageBytes) >> 4) | (1u << 16);
           const uint32_t d = tmem + (uint32_t)((2 * hh + buf) * kKeys);
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t a = umma::smem_desc_sw128(q_addr + (ks >> 2) * kQHalf + (ks & 3) * 32, 16, 1024);
-            const uint64_t bd = umma::smem_desc_sw128(k_addr + (ks >> 2) * kKBox + (ks & 3) * 32, 16, 1024);
+            const uint64_t a = desc_hi | (uint64_t)(q_lo + (uint32_t)(((ks >> 2) * kQHalf + (ks & 3) * 32) >> 4));
+            const uint64_t bd = desc_hi | (uint64_t)(k_lo + (uint32_t)(((ks >> 2) * kKBox + (ks & 3) * 32) >> 4));
             umma::mma_bf16(d, a, bd, idesc_s, ks > 0);
           }
           umma::commit(&sh.s_full[hh][buf]);
-          if (i == n_tiles - 1) umma::commit(&sh.q_empty);     // the item's last product that reads Q
+          if (last) umma::commit(&sh.q_empty);          // the item's last product that reads Q
         };
-        ok = wait_or_abort(&sh.kv_full[t0 % kStages], (t0 / kStages) & 1, &sh, p.dev_status);
+        ok = wait_or_abort(&sh.kv_full[st_cur], ph_cur, &sh, p.dev_status);
         if (!ok) break;
-        issue_s(0);
+        issue_s(st_cur, th & 1, n_tiles == 1);
         for (int i = 0; i < n_tiles; ++i) {
-          const int t = t0 + i;
-          if (i + 1 < n_tiles) {
-            ok = wait_or_abort(&sh.kv_full[(t + 1) % kStages], ((t + 1) / kStages) & 1, &sh, p.dev_status);
-            if (!ok) break;
-            issue_s(i + 1);                             // its buffer held S and P of two tiles ago: that P V product was issued
-                                                        // before this one, and the tensor pipe runs them in issue order
-          }
-          const uint32_t v_addr = st_addr + (t % kStages) * kStageBytes + kKTile;
+          int st_nxt = st_cur + 1, ph_nxt = ph_cur;
+          if (st_nxt == kStages) { st_nxt = 0; ph_nxt ^= 1; }
           const int tt = th + i;                        // tile count of this head: P sits in S buffer tt & 1, use tt >> 1 of it
+          if (i + 1 < n_tiles) {
+            ok = wait_or_abort(&sh.kv_full[st_nxt], ph_nxt, &sh, p.dev_status);
+            if (!ok) break;
+            issue_s(st_nxt, (tt + 1) & 1, i + 2 == n_tiles);   // its buffer held S and P of two tiles ago: that P V product was issued
+                                                               // before this one, and the tensor pipe runs them in issue order
+          }
           ok = wait_or_abort(&sh.p_full[hh][tt & 1], (tt >> 1) & 1, &sh, p.dev_status);
           if (!ok) break;
           umma::fence_after_sync();                     // P was written with tcgen05.st by the softmax threads
+          const uint32_t v_lo = ((st_addr + st_cur * kStageBytes + kKTile) >> 4) | v_lbo;
+          const uint32_t p_tmem = tmem + (uint32_t)((2 * hh + (tt & 1)) * kKeys);
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {              // 16 keys per step
-            const uint32_t a = tmem + (uint32_t)((2 * hh + (tt & 1)) * kKeys + 8 * kk);     // 16 keys = 8 packed columns of P
-            const uint64_t bd = umma::smem_desc_sw128(v_addr + kk * 2048, kKBox, 1024);    // next 64 channels: one box on
-            umma::mma_bf16_a_tmem(o_tmem, a, bd, idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
-          }
+          for (int kk = 0; kk < 4; ++kk)                // 16 keys per step: 8 packed columns of P, two 8-row groups of V
+            umma::mma_bf16_a_tmem(o_tmem, p_tmem + 8 * kk, desc_hi | (uint64_t)(v_lo + (uint32_t)((kk * 2048) >> 4)), idesc_o,
+                                  (i > 0 || kk > 0) ? 1u : 0u);
           umma::commit(&sh.o_done[hh][tt & 1]);
-          umma::commit(&sh.kv_empty[t % kStages]);      // this head is done with K and V of the stage
+          umma::commit(&sh.kv_empty[st_cur]);           // this head is done with K and V of the stage
+          st_cur = st_nxt; ph_cur = ph_nxt;
         }
         t0 += n_tiles;
         th += n_tiles;
