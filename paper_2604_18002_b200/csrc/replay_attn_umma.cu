@@ -12,7 +12,7 @@
 //                        shared memory by tiled TMA as soon as the previous item's last S product has
 //                        read them;
 //   producer warps (4)   gather 64-key K/V tiles by position (kept lists, then the contiguous block)
-//                        with 16-byte cp.async into a 5-stage ring, 128-byte swizzled.  Every lane hands
+//                        with 16-byte cp.async into a 4-stage ring, 128-byte swizzled.  Every lane hands
 //                        its copies of a tile to the stage's mbarrier with cp.async.mbarrier.arrive.noinc:
 //                        the arrival fires when the copies have landed, nobody waits for it, so the
 //                        producers run a full ring ahead and a tile becomes visible to the MMA warp the
@@ -53,7 +53,7 @@ namespace {
 
 constexpr int kQRows = 128;                   // query tokens per item = tensor-memory lanes
 constexpr int kKeys = 64;                     // keys per pipeline stage
-constexpr int kStages = 5;
+constexpr int kStages = 4;
 constexpr int kMmaWarp = 8;                   // warps 0-7: softmax (two groups of four, one query head each);
                                               // warps 8, 9: one MMA-issuing thread per head
 constexpr int kPlannerWarp = 10;
@@ -66,7 +66,8 @@ constexpr int kQBytes = 2 * kQHalf;           // 32 KB per head
 constexpr int kKBox = kKeys * 128;            // 64 keys x 64 channels
 constexpr int kKTile = 2 * kKBox;             // K (or V) tile, 16 KB
 constexpr int kStageBytes = 2 * kKTile;       // K + V
-constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 1024;
+constexpr int kOutStage = 4096;                // per softmax warp: 32 rows x 32 columns of the output on their way out
+constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 8 * kOutStage + 1024;
 constexpr uint32_t kTmemCols = 512;           // S[h][buf] at (2h + buf) * 64 (P over its first 32 columns), O[h] at 256 + 128 h
 constexpr int kMaxSeg = 34;                   // rounds one query tile can straddle (+ the contiguous part)
 constexpr float kLazyRescale = 8.f;           // log2 units the row maximum may grow before O is rescaled
@@ -155,6 +156,7 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
   uint8_t* base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = base;                                   // [2 heads][32 KB]
   uint8_t* stage = sQ + 2 * kQBytes;                    // [kStages][K 16 KB | V 16 KB]
+  uint8_t* sOut = stage + kStages * kStageBytes;        // [8 softmax warps][4 KB]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int pairs = (p.g + 1) >> 1;
 
@@ -470,17 +472,18 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
           // raw scores stay as they are; invisible ones become -inf.  The row maximum is taken on the raw values
           // (the scale is positive) with three-input max over four independent chains.
           if (need_mask) {
-            const int j0 = c_lo + kt * kKeys;
+            // the visible keys of this row are one index range of the tile: the whole kept tile (up to its end) if the
+            // row's block follows that round, else nothing; or the causal part of the row's own block
+            int jlo, jhi;
+            if (rho >= 1) { jlo = blk == rho ? 0 : kKeys; jhi = n_here - 1; }
+            else { const int j0 = c_lo + kt * kKeys; jlo = max(lo_row - j0, 0); jhi = t_q - j0; }
+            const uint32_t width = jhi >= jlo ? (uint32_t)(jhi - jlo) : 0u;
+            if (jhi < jlo) jlo = 2 * kKeys;                                    // nothing visible
 #pragma unroll
             for (int half = 0; half < 2; ++half)
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const int jj = 32 * half + j;
-                bool vis;
-                if (rho >= 1) vis = jj < n_here && blk == rho;                 // a kept entry of the round before this row's block
-                else vis = j0 + jj >= lo_row && j0 + jj <= t_q;                // a token of the row's own block, causal
-                if (!vis) zr[half][j] = 0xff800000u;                           // -inf
-              }
+              for (int j = 0; j < 32; ++j)
+                if ((uint32_t)(32 * half + j - jlo) > width) zr[half][j] = 0xff800000u;   // -inf
           }
           float mxc[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -547,27 +550,47 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
         if (!warp_wait(&sh.o_done[hh][(tc - 1) & 1], ((tc - 1) >> 1) & 1, &sh, p.dev_status)) { ok = false; break; }
         umma::fence_after_sync();
         const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-        const int64_t o_base = ((((int64_t)pl.l * p.B + pl.b) * p.Hq + pl.hq0 + hh) * (int64_t)p.t_max + t_q) * 128;
+        // The thread owns a whole output row, but a store instruction should cover whole rows' worth of consecutive
+        // bytes: every 32-column chunk goes through the warp's 4 KB of shared memory (own row in, 16-byte pieces of
+        // several rows out), so that eight (fp32) or four (bf16) lanes write one row's chunk side by side.
+        uint8_t* so = sOut + warp * kOutStage;
+        const int t_w0 = q0 + 32 * (warp & 3);                                // query token of this warp's row 0
+        const int64_t o_row0 = ((((int64_t)pl.l * p.B + pl.b) * p.Hq + pl.hq0 + hh) * (int64_t)p.t_max + t_w0) * 128;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 32) {
           uint32_t o[32];
           umma::tmem_ld32(o_addr + c0, o);
           umma::tmem_ld_wait();
-          if (t_q < T_b) {
-            if (p.out_bf16) {
-              uint4* dst = reinterpret_cast<uint4*>((__nv_bfloat16*)p.out + o_base + c0);
+          __syncwarp();                                                       // the previous chunk has left the staging area
+          if (p.out_bf16) {
 #pragma unroll
-              for (int j = 0; j < 4; ++j)
-                dst[j] = make_uint4(ptx::pack_bf16x2(__uint_as_float(o[8 * j]) * inv, __uint_as_float(o[8 * j + 1]) * inv),
-                                    ptx::pack_bf16x2(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv),
-                                    ptx::pack_bf16x2(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv),
-                                    ptx::pack_bf16x2(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv));
-            } else {
-              float4* dst = reinterpret_cast<float4*>((float*)p.out + o_base + c0);
+            for (int c = 0; c < 4; ++c)
+              *reinterpret_cast<uint4*>(so + lane * 64 + ((c ^ ((lane >> 1) & 3)) << 4)) =
+                  make_uint4(ptx::pack_bf16x2(__uint_as_float(o[8 * c]) * inv, __uint_as_float(o[8 * c + 1]) * inv),
+                             ptx::pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv),
+                             ptx::pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv),
+                             ptx::pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv));
+            __syncwarp();
 #pragma unroll
-              for (int j = 0; j < 8; ++j)
-                dst[j] = make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
-                                     __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
+            for (int u = 0; u < 4; ++u) {                                     // eight rows per store, four lanes per row
+              const int r = 8 * u + (lane >> 2), c = lane & 3;
+              const uint4 v = *reinterpret_cast<const uint4*>(so + r * 64 + ((c ^ ((r >> 1) & 3)) << 4));
+              if (t_w0 + r < T_b)
+                *reinterpret_cast<uint4*>((__nv_bfloat16*)p.out + o_row0 + (int64_t)r * 128 + c0 + 8 * c) = v;
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              *reinterpret_cast<float4*>(so + lane * 128 + ((c ^ (lane & 7)) << 4)) =
+                  make_float4(__uint_as_float(o[4 * c]) * inv, __uint_as_float(o[4 * c + 1]) * inv,
+                              __uint_as_float(o[4 * c + 2]) * inv, __uint_as_float(o[4 * c + 3]) * inv);
+            __syncwarp();
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {                                     // four rows per store, eight lanes per row
+              const int r = 4 * u + (lane >> 3), c = lane & 7;
+              const float4 v = *reinterpret_cast<const float4*>(so + r * 128 + ((c ^ (r & 7)) << 4));
+              if (t_w0 + r < T_b)
+                *reinterpret_cast<float4*>((float*)p.out + o_row0 + (int64_t)r * 128 + c0 + 4 * c) = v;
             }
           }
         }
