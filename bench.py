@@ -221,6 +221,7 @@ def run_ngc(args):
     noise_seed = cfg["noise_seed"]
 
     ev_marks = []
+    score_kernels = ngc.score_launches(ro.cache, W_RECENT)
 
     def one_step(step_idx, timed=False):
         """The whole hot path once.  Timed steps drop an event between the calls (score | sample | log-prob | compact |
@@ -243,7 +244,7 @@ def run_ngc(args):
         mark()
         ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, cfg["lists"], 1, status=ro.status)
         mark()
-        ro.launches += 7          # score 3, sample 1, log-prob 1, compaction 2
+        ro.launches += score_kernels + 4          # score (group by group), sample 1, log-prob 1, compaction 2
         for s in range(steps):
             ro.decode_step(q[s], out[s], nk[s], nv[s])
         mark()
@@ -456,6 +457,8 @@ def measure_other(args):
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
+    score_kernels = ngc.score_launches(ro.cache, W_RECENT)
+
     def eviction(rnd, t):
         e = [ev() for _ in range(5)]
         e[0].record()
@@ -476,7 +479,7 @@ def measure_other(args):
         else:
             ngc.ngc_compact_kv(ro.cache, ro.kept_sorted, k_t, lists, block, status=ro.status)
         e[4].record()
-        ro.launches += 7 + (1 if G > 1 and not per_list and paged is None else 0)   # score 3, sample 1, log-prob 1, compaction 2 (+ check)
+        ro.launches += score_kernels + 4 + (1 if G > 1 and not per_list and paged is None else 0)   # score, sample 1, log-prob 1, compaction 2 (+ check)
         t.append(e)
 
     graph = None

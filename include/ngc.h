@@ -153,6 +153,10 @@ int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, 
                     int log_transform, float* logits, int n_max, int32_t* n_units_out,
                     void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream);
 
+/* Number of kernels one ngc_score_evict call enqueues for this cache and window (host-only planning query, for
+ * launch counting). */
+int ngc_score_evict_launches(const ngc_cache* c, int w);
+
 /*
  * Gradient of the eviction scores with respect to the recent queries and the
  * keys -- Sections 4.4 and 4.5: the eviction loss reaches the model through

@@ -25,7 +25,7 @@ OP_SCORE, OP_SAMPLE, OP_LOGPROB, OP_COMPACT, OP_DECODE, OP_SCORE_BACKWARD = rang
 DEV_STATUS = {0: "ok", 1: "bad counts", 2: "NaN logit", 3: "bad kept list", 4: "strip full",
               5: "lists disagree", 6: "timeout", 7: "index out of bounds (bounds-checking build)"}
 
-EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict",
+EXPORTS = ["ngc_version", "ngc_strerror", "ngc_last_cuda_error", "ngc_workspace_bytes", "ngc_decode_splits", "ngc_score_evict", "ngc_score_evict_launches",
            "ngc_sample_evict", "ngc_evict_logprob", "ngc_evict_logprob_backward", "ngc_compact_kv", "ngc_decode_attn_ragged",
            "ngc_decode_attn_ragged_static", "ngc_evict_pages", "ngc_decode_attn_paged", "ngc_score_evict_paged", "ngc_replay_visibility", "ngc_score_evict_backward", "ngc_replay_attn", "ngc_replay_attn_variant", "ngc_selftest_bounded_wait"]
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -65,6 +65,8 @@ def _load(path: str = LIB_PATH):
     lib.ngc_workspace_bytes.argtypes = [i32, C.POINTER(CacheDesc), i32, i32, i32]
     lib.ngc_decode_splits.restype = i32
     lib.ngc_decode_splits.argtypes = [C.POINTER(CacheDesc), i32]
+    lib.ngc_score_evict_launches.restype = i32
+    lib.ngc_score_evict_launches.argtypes = [C.POINTER(CacheDesc), i32]
     lib.ngc_score_evict.restype = i32
     lib.ngc_score_evict.argtypes = [C.POINTER(CacheDesc), vp, i32, i32, i32, i32, vp, i32, vp, vp, sz, vp, vp]
     lib.ngc_sample_evict.restype = i32
@@ -199,6 +201,12 @@ def workspace_bytes(op: int, cache: Optional[NgcCache] = None, G: int = 1, n_max
 def decode_splits(cache: NgcCache, layers: Optional[int] = None, append: bool = True) -> int:
     d = cache.desc(1 if append else 0)
     return int(lib.ngc_decode_splits(C.byref(d), cache.L if layers is None else layers))
+
+
+def score_launches(cache: NgcCache, w: int) -> int:
+    """Kernels one ngc_score_evict call enqueues (launch counting)."""
+    d = cache.desc()
+    return int(lib.ngc_score_evict_launches(C.byref(d), w))
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> Optional[torch.Tensor]:

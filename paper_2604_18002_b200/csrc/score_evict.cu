@@ -617,6 +617,12 @@ int score_impl(const ngc_cache* c, const PagedView& pv, const void* q_recent, in
 }  // namespace
 }  // namespace ngc
 
+extern "C" int ngc_score_evict_launches(const ngc_cache* c, int w) {
+  using namespace ngc;
+  if (!valid_cache(c) || w <= 0 || c->rows == 0 || c->max_len == 0) return 0;
+  return 3;      // statistics, probabilities, list reduction
+}
+
 extern "C" int ngc_score_evict(const ngc_cache* c, const void* q_recent, int w, int block, int lists,
                                int log_transform, float* logits, int n_max, int32_t* n_units_out,
                                void* ws, size_t ws_bytes, int32_t* dev_status, ngc_stream stream) {

@@ -66,7 +66,7 @@ class NgcRollout:
             target = self.score_logits if logits is not None else self.logits
             ngc.ngc_score_evict(self.cache, q_recent, self.block, self.lists, target, ws=self.ws_score, status=self.status,
                                 n_units_out=self.n_units)
-            self.launches += 3
+            self.launches += ngc.score_launches(self.cache, q_recent.shape[3])
             if self.cache.lens_lists and logits is None:
                 n = self.n_units        # a length per list: the library reports the unit count of each rollout's longest list
         src = logits if logits is not None else self.logits
