@@ -67,7 +67,7 @@ METRIC = "evict+compact+decode tokens/sec at B=64"
 W_RECENT = 5
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic K/V bytes for decode_stream_t_kernel, from the ncu
 # capture summarised in profiles/decode_stream_t_kernel_config2.md (small case, scaled by tokens processed)
-NCU_TRAFFIC_RATIO = 1.0141
+NCU_TRAFFIC_RATIO = 1.0118
 
 
 def peaks():
