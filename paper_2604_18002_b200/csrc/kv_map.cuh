@@ -54,4 +54,20 @@ inline bool make_rows_map(CUtensorMap* map, const void* base, int64_t rows, int 
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A row-major matrix of `rows` rows of 128 elements (bf16 or fp32) as a 2-D tensor for TMA stores of 32-column,
+// `box_rows`-row boxes; the shared-memory side uses the swizzle whose span equals the box's row (64 bytes for bf16,
+// 128 bytes for fp32), so that a thread per row can fill the box without bank conflicts.
+inline bool make_out_map(CUtensorMap* map, void* base, bool bf16, int64_t rows, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn || rows <= 0 || rows > 0x7fffffffLL) return false;
+  const cuuint64_t elt = bf16 ? 2 : 4;
+  cuuint64_t dims[2] = {128, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {128 * elt};
+  cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace ngc

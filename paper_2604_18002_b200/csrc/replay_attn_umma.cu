@@ -135,8 +135,15 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, Shared
   return __all_sync(0xffffffffu, wait_or_abort(bar, parity, sh, dev_status));
 }
 
-// Tensor map of a launch: Q as a 2-D tensor (channel, row over all layers / sequences / heads), box = 64 channels x 128 rows.
-struct Maps { CUtensorMap q; };
+// Tensor maps of a launch: Q as a 2-D tensor (channel, row over all layers / sequences / heads), box = 64 channels x
+// 128 rows; the output over the same rows, box = 32 channels x 32 rows (one warp's chunk).
+struct Maps { CUtensorMap q, out; };
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(ptx::smem_u32(src))
+               : "memory");
+}
 
 // swizzled byte offset of 16-byte piece c (0..15) of key row r inside a K or V tile
 __device__ __forceinline__ uint32_t tile_off(int r, int c) {
@@ -178,6 +185,7 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
     ptx::fence_barrier_init();
     sh.abort = 0;
     ptx::prefetch_tensormap(&maps.q);
+    ptx::prefetch_tensormap(&maps.out);
   }
   if (warp == kMmaWarp) umma::tmem_alloc(&sh.tmem, kTmemCols);
   umma::fence_before_sync();
@@ -550,18 +558,21 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
         if (!warp_wait(&sh.o_done[hh][(tc - 1) & 1], ((tc - 1) >> 1) & 1, &sh, p.dev_status)) { ok = false; break; }
         umma::fence_after_sync();
         const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-        // The thread owns a whole output row, but a store instruction should cover whole rows' worth of consecutive
-        // bytes: every 32-column chunk goes through the warp's 4 KB of shared memory (own row in, 16-byte pieces of
-        // several rows out), so that eight (fp32) or four (bf16) lanes write one row's chunk side by side.
+        // The thread owns a whole output row.  Every 32-column chunk goes through the warp's 4 KB of shared memory (each
+        // thread its own row, in the swizzle TMA expects for a box of that row width) and leaves as ONE asynchronous TMA
+        // store per warp: the load/store unit, busy with the producers' gathers, is not involved.  A warp whose 32 rows
+        // reach beyond the sequence must not write those rows: it stores with ordinary instructions, several lanes per row.
         uint8_t* so = sOut + warp * kOutStage;
         const int t_w0 = q0 + 32 * (warp & 3);                                // query token of this warp's row 0
         const int64_t o_row0 = ((((int64_t)pl.l * p.B + pl.b) * p.Hq + pl.hq0 + hh) * (int64_t)p.t_max + t_w0) * 128;
+        const bool whole = t_w0 + 32 <= T_b;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 32) {
           uint32_t o[32];
           umma::tmem_ld32(o_addr + c0, o);
           umma::tmem_ld_wait();
-          __syncwarp();                                                       // the previous chunk has left the staging area
+          if (lane == 0) ptx::bulk_wait_read<0>();                            // the previous chunk's store has read the staging area
+          __syncwarp();
           if (p.out_bf16) {
 #pragma unroll
             for (int c = 0; c < 4; ++c)
@@ -570,6 +581,21 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
                              ptx::pack_bf16x2(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv),
                              ptx::pack_bf16x2(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv),
                              ptx::pack_bf16x2(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv));
+          } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              *reinterpret_cast<float4*>(so + lane * 128 + ((c ^ (lane & 7)) << 4)) =
+                  make_float4(__uint_as_float(o[4 * c]) * inv, __uint_as_float(o[4 * c + 1]) * inv,
+                              __uint_as_float(o[4 * c + 2]) * inv, __uint_as_float(o[4 * c + 3]) * inv);
+          }
+          if (whole) {
+            ptx::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&maps.out, c0, (int)(o_row0 >> 7), so);
+              ptx::bulk_commit();
+            }
+          } else if (p.out_bf16) {
             __syncwarp();
 #pragma unroll
             for (int u = 0; u < 4; ++u) {                                     // eight rows per store, four lanes per row
@@ -579,11 +605,6 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
                 *reinterpret_cast<uint4*>((__nv_bfloat16*)p.out + o_row0 + (int64_t)r * 128 + c0 + 8 * c) = v;
             }
           } else {
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-              *reinterpret_cast<float4*>(so + lane * 128 + ((c ^ (lane & 7)) << 4)) =
-                  make_float4(__uint_as_float(o[4 * c]) * inv, __uint_as_float(o[4 * c + 1]) * inv,
-                              __uint_as_float(o[4 * c + 2]) * inv, __uint_as_float(o[4 * c + 3]) * inv);
             __syncwarp();
 #pragma unroll
             for (int u = 0; u < 8; ++u) {                                     // four rows per store, eight lanes per row
@@ -600,6 +621,7 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&sh.plan_empty[slot]);
     }
+    if (lane == 0) ptx::bulk_wait<0>();                 // this warp's output stores have completed
   }
   // ---- teardown: every role has left its loops; nothing of this CTA is in flight any more
   umma::fence_before_sync();
@@ -618,9 +640,11 @@ int launch_replay_attn_umma(const ReplayAttnParams& p, cudaStream_t stream) {
   q.q_tiles = (p.t_max + kQRows - 1) / kQRows;
   const int64_t items = (int64_t)p.L * p.B * p.Hkv * pairs * q.q_tiles;
   if (items > 0x7fffffffLL) return NGC_ERR_UNSUPPORTED;
-  // TMA coordinates are 32-bit: the queries are addressed by row over all layers, sequences and heads
+  // TMA coordinates are 32-bit: queries and outputs are addressed by row over all layers, sequences and heads
   Maps maps;
-  if (!make_rows_map(&maps.q, p.q, (int64_t)p.L * p.B * p.Hq * p.t_max, kQRows)) return NGC_ERR_UNSUPPORTED;
+  if (!make_rows_map(&maps.q, p.q, (int64_t)p.L * p.B * p.Hq * p.t_max, kQRows) ||
+      !make_out_map(&maps.out, p.out, p.out_bf16 != 0, (int64_t)p.L * p.B * p.Hq * p.t_max, 32))
+    return NGC_ERR_UNSUPPORTED;
   static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
   static int sm_count[kMaxDevices] = {0};
   int dev = -1;
