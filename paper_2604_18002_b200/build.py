@@ -23,7 +23,7 @@ INCLUDE = os.path.join(ROOT, "include")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libngc_b200.so")
 
-SOURCES = ["api.cu", "compact_kv.cu", "sample_evict.cu", "evict_logprob.cu", "decode_attn.cu", "score_evict.cu", "replay_visibility.cu", "score_backward.cu", "replay_attn.cu", "replay_attn_umma.cu", "selftest.cu"]
+SOURCES = ["api.cu", "compact_kv.cu", "sample_evict.cu", "evict_logprob.cu", "decode_attn.cu", "score_evict.cu", "replay_visibility.cu", "score_backward.cu", "score_backward_umma.cu", "replay_attn.cu", "replay_attn_umma.cu", "selftest.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",

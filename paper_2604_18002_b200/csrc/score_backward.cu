@@ -19,12 +19,14 @@
 //      Per-range dQ partials go to the workspace; a third small kernel adds the ranges of a strip
 //      in a fixed order (no float atomics: results are reproducible).
 #include <cuda_bf16.h>
+#include <stdlib.h>
 
 
 #include "kv_map.cuh"
 #include "ngc_common.cuh"
 #include "ngc_plan.h"
 #include "ptx.cuh"
+#include "score_backward.cuh"
 
 namespace ngc {
 namespace {
@@ -36,57 +38,11 @@ constexpr int kBoxBytes = kTileT * 128;           // 64 tokens x 64 channels of 
 constexpr int kStageBytes = 2 * kBoxBytes;
 constexpr int kStagesA = 4;                       // statistics pass, two CTAs per SM
 constexpr int kStagesB = 4;                       // gradient pass, two CTAs per SM
-constexpr int kMaxRows = 40;
+constexpr int kMaxRows = kBwdMaxRows;
 constexpr int kQRowBytes = 272;                   // query row in shared memory: 256 bytes + 16 (conflict-free ldmatrix)
 constexpr int kQBytes = 48 * kQRowBytes;          // rows padded to 48 (three 16-row MMA steps)
 constexpr int kDzRowBytes = 112;                  // dz row (one token, 48 rows of bf16 = 96 bytes) + 16
 constexpr int kDzBytes = kTileT * kDzRowBytes;
-
-struct BwdParams {
-  const void* k;
-  const void* q_recent;
-  const int64_t* seq_off;
-  const int32_t* lens;
-  const float* logits;         // forward output (log variant only)
-  const float* grad_logits;    // [B][G][n_max]
-  float4* stats;               // [strips][n_split][kMaxRows] (max, sum e, sum e*P, -)
-  float* dq_part;              // [strips][n_split][kMaxRows][128]
-  float* grad_q;               // [L][B][Hq][w][128]
-  void* grad_k;                // [L][Hkv][R][128] bf16
-  int32_t* dev_status;
-  int64_t rows_R;
-  int L, B, Hq, Hkv, g, w, n_rows, block, lists, G, n_max, log_transform, n_split, lens_lists;
-  float scale_log2, inv_sqrt_d;
-};
-
-// (m, s, n) <- merge of two partial (max, sum 2^(z-max), sum 2^(z-max) P) triples
-__device__ __forceinline__ void merge3(float& m, float& s, float& n, float mo, float so, float no) {
-  const float mn = fmaxf(m, mo);
-  if (mn == -INFINITY) { s = 0.f; n = 0.f; return; }
-  const float fa = ptx::ex2_approx(m - mn), fb = ptx::ex2_approx(mo - mn);
-  s = s * fa + so * fb;
-  n = n * fa + no * fb;
-  m = mn;
-}
-
-// dL/dA of a token for the rows of list gi (0 beyond the sequence)
-__device__ __forceinline__ float token_weight(const BwdParams& p, int b, int gi, int t, int T_b, float inv_rows) {
-  if (t >= T_b) return 0.f;
-  const int u = p.block == 1 ? t : t / p.block;
-  if (u >= p.n_max) return 0.f;
-  const int size = p.block == 1 ? 1 : min((u + 1) * p.block, T_b) - u * p.block;
-  const int64_t idx = ((int64_t)b * p.G + gi) * p.n_max + u;
-  float up = p.grad_logits[idx];
-  if (p.log_transform) up *= __expf(-p.logits[idx]);        // d log s = ds / s
-  return up * inv_rows / (float)size;
-}
-
-// rows of list gi: layers x KV heads feeding it x group size x window queries that exist
-__device__ __forceinline__ float inv_list_rows(const BwdParams& p, int T_b) {
-  const int w_eff = min(p.w, T_b);
-  const int strips = p.lists == NGC_LISTS_SHARED ? p.L * p.Hkv : (p.lists == NGC_LISTS_PER_LAYER ? p.Hkv : 1);
-  return 1.f / (float)(strips * p.g * w_eff);
-}
 
 // Item decoding and token range shared by both passes.
 struct Item { int split, strip, h, b, l, T_b, tile_lo, n_tiles, gi; };
@@ -124,12 +80,6 @@ __device__ __forceinline__ void produce_k_tiles(const CUtensorMap* map_k, const 
     ptx::tma_load_3d(sp, map_k, 0, y, plane, &bar_full[s]);
     ptx::tma_load_3d(sp + kBoxBytes, map_k, 64, y, plane, &bar_full[s]);
   }
-}
-
-// Last visible token of column c of S (row c of the strip = head-in-group c / w, window slot c % w); -1: unused.
-__device__ __forceinline__ int column_limit(const BwdParams& p, int c, int T_b) {
-  const int jc = c % p.w;
-  return (c < p.n_rows && jc >= p.w - min(p.w, T_b)) ? T_b - p.w + jc : -1;
 }
 
 // ---------------------------------------------------------------- pass 1: row statistics
@@ -511,7 +461,7 @@ int bwd_n_split(const ngc_cache* c) {
 }
 
 template <int NT>
-int launch_bwd(const CUtensorMap& map_k, const CUtensorMap& map_gk, const BwdParams& p, unsigned grid, cudaStream_t stream) {
+int launch_bwd(const CUtensorMap& map_k, const CUtensorMap& map_gk, const BwdParams& p, unsigned grid, bool use_umma, cudaStream_t stream) {
   const int smem_a = kStagesA * kStageBytes + 1024;
   const int smem_b = kStagesB * kStageBytes + 1024 + kStageBytes + kQBytes + 2 * kDzBytes;
   static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
@@ -522,7 +472,7 @@ int launch_bwd(const CUtensorMap& map_k, const CUtensorMap& map_gk, const BwdPar
   });
   if (attr_rc != NGC_OK) return attr_rc;
   score_bwd_stats_kernel<NT><<<grid, kThreads, smem_a, stream>>>(map_k, p);
-  score_bwd_kernel<NT><<<grid, kThreads, smem_b, stream>>>(map_k, map_gk, p);
+  if (!use_umma) score_bwd_kernel<NT><<<grid, kThreads, smem_b, stream>>>(map_k, map_gk, p);
   return launch_status();
 }
 
@@ -577,15 +527,20 @@ extern "C" int ngc_score_evict_backward(const ngc_cache* c, const void* q_recent
   if (!make_kv_map(&map_k, c->k, c->rows, c->L * c->Hkv, kTileT) || !make_kv_map(&map_gk, grad_k, c->rows, c->L * c->Hkv, kTileT))
     return NGC_ERR_UNSUPPORTED;
   const unsigned grid = (unsigned)items;
+  const bool use_umma = getenv("NGC_BWD_LEGACY") == nullptr;
   int rc;
   switch ((p.n_rows + 7) / 8) {
-    case 1: rc = launch_bwd<1>(map_k, map_gk, p, grid, stream); break;
-    case 2: rc = launch_bwd<2>(map_k, map_gk, p, grid, stream); break;
-    case 3: rc = launch_bwd<3>(map_k, map_gk, p, grid, stream); break;
-    case 4: rc = launch_bwd<4>(map_k, map_gk, p, grid, stream); break;
-    default: rc = launch_bwd<5>(map_k, map_gk, p, grid, stream); break;
+    case 1: rc = launch_bwd<1>(map_k, map_gk, p, grid, use_umma, stream); break;
+    case 2: rc = launch_bwd<2>(map_k, map_gk, p, grid, use_umma, stream); break;
+    case 3: rc = launch_bwd<3>(map_k, map_gk, p, grid, use_umma, stream); break;
+    case 4: rc = launch_bwd<4>(map_k, map_gk, p, grid, use_umma, stream); break;
+    default: rc = launch_bwd<5>(map_k, map_gk, p, grid, use_umma, stream); break;
   }
   if (rc != NGC_OK) return rc;
+  if (use_umma) {
+    rc = launch_score_bwd_umma(p, c->k, grad_k, c->rows, c->L * c->Hkv, (int64_t)items, stream);
+    if (rc != NGC_OK) return rc;
+  }
   score_bwd_reduce_kernel<<<(unsigned)(c->L * c->B * c->Hkv * p.n_rows), 128, 0, stream>>>(p);
   return launch_status();
 }

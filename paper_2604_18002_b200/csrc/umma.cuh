@@ -21,9 +21,9 @@
 namespace ngc {
 namespace umma {
 
-constexpr uint32_t kF32Acc = 1u << 4, kBf16A = 1u << 7, kBf16B = 1u << 10, kBMajorMN = 1u << 16;
-__host__ __device__ constexpr uint32_t instr_desc(uint32_t M, uint32_t N, bool b_mn_major) {
-  return kF32Acc | kBf16A | kBf16B | (b_mn_major ? kBMajorMN : 0u) | ((N >> 3) << 17) | ((M >> 4) << 24);
+constexpr uint32_t kF32Acc = 1u << 4, kBf16A = 1u << 7, kBf16B = 1u << 10, kAMajorMN = 1u << 15, kBMajorMN = 1u << 16;
+__host__ __device__ constexpr uint32_t instr_desc(uint32_t M, uint32_t N, bool b_mn_major, bool a_mn_major = false) {
+  return kF32Acc | kBf16A | kBf16B | (a_mn_major ? kAMajorMN : 0u) | (b_mn_major ? kBMajorMN : 0u) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
 // 128-byte-swizzled operand at shared address `saddr` (the tile it belongs to is 1024-byte aligned).
@@ -77,6 +77,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
 }
+// 16 consecutive columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
@@ -87,6 +95,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
         "r"(r[30]), "r"(r[31])
       : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
