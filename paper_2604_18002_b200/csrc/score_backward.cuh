@@ -39,16 +39,30 @@ __device__ __forceinline__ void merge3(float& m, float& s, float& n, float mo, f
   m = mn;
 }
 
-// dL/dA of a token for the rows of list gi (0 beyond the sequence)
-__device__ __forceinline__ float token_weight(const BwdParams& p, int b, int gi, int t, int T_b, float inv_rows) {
-  if (t >= T_b) return 0.f;
-  const int u = p.block == 1 ? t : t / p.block;
-  if (u >= p.n_max) return 0.f;
-  const int size = p.block == 1 ? 1 : min((u + 1) * p.block, T_b) - u * p.block;
-  const int64_t idx = ((int64_t)b * p.G + gi) * p.n_max + u;
-  float up = p.grad_logits[idx];
-  if (p.log_transform) up *= __expf(-p.logits[idx]);        // d log s = ds / s
-  return up * inv_rows / (float)size;
+// dL/dA of a token for the rows of list gi (0 beyond the sequence), in two steps for software pipelining:
+// `issue` starts the loads for a token of a LATER tile, `finish`
+// turns them into the weight where it is needed.  The empty asm pins the first use of the loaded values to that
+// place (otherwise the arithmetic is scheduled right behind the loads and the warp stalls on them at once).
+struct TokenWeightRaw { float up, lg, f; };
+__device__ __forceinline__ TokenWeightRaw token_weight_issue(const BwdParams& p, int b, int gi, int t, int T_b, float inv_rows) {
+  TokenWeightRaw raw = {0.f, 0.f, 0.f};
+  if (t < T_b) {
+    const int u = p.block == 1 ? t : t / p.block;
+    if (u < p.n_max) {
+      const int size = p.block == 1 ? 1 : min((u + 1) * p.block, T_b) - u * p.block;
+      const int64_t idx = ((int64_t)b * p.G + gi) * p.n_max + u;
+      raw.f = inv_rows / (float)size;
+      raw.up = p.grad_logits[idx];
+      if (p.log_transform) raw.lg = p.logits[idx];
+    }
+  }
+  return raw;
+}
+__device__ __forceinline__ float token_weight_finish(const BwdParams& p, TokenWeightRaw raw) {
+  asm volatile("" : "+f"(raw.up), "+f"(raw.lg));
+  float up = raw.up;
+  if (p.log_transform) up *= __expf(-raw.lg);                 // d log s = ds / s
+  return up * raw.f;
 }
 
 // rows of list gi: layers x KV heads feeding it x group size x window queries that exist

@@ -57,23 +57,23 @@ struct Shared {
 };
 
 // Bounded wait that also gives up as soon as another thread of the CTA has given up.
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Shared* sh, int32_t* dev_status) {
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, int* abort_flag, int32_t* dev_status) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = ptx::globaltimer_ns();
   for (uint32_t spins = 0;; ++spins) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     if ((spins & 63u) == 63u) {
-      if (*(volatile int*)&sh->abort) return false;
+      if (*(volatile int*)abort_flag) return false;
       if (ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs) {
-        *(volatile int*)&sh->abort = 1;
+        *(volatile int*)abort_flag = 1;
         set_dev_status(dev_status, NGC_DEV_TIMEOUT);
         return false;
       }
     }
   }
 }
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, Shared* sh, int32_t* dev_status) {
-  return __all_sync(0xffffffffu, wait_or_abort(bar, parity, sh, dev_status));
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, int* abort_flag, int32_t* dev_status) {
+  return __all_sync(0xffffffffu, wait_or_abort(bar, parity, abort_flag, dev_status));
 }
 
 // One item: a token range of one strip, in tiles of 128 tokens.
@@ -158,7 +158,7 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
         const int row0 = (int)p.seq_off[it.b];
         for (int i = 0; i < it.n_tiles; ++i, ++t) {
           const int s = t % kStages;
-          if (t >= kStages && !wait_or_abort(&sh.k_empty[s], ((t / kStages) - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+          if (t >= kStages && !wait_or_abort(&sh.k_empty[s], ((t / kStages) - 1) & 1, &sh.abort, p.dev_status)) { ok = false; break; }
           uint8_t* sp = stage + s * kStageBytes;
           ptx::mbar_expect_tx(&sh.k_full[s], kStageBytes);
           const int y = row0 + (it.tile_lo + i) * kTok;
@@ -187,7 +187,7 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
         const Item it = decode_item(p, item);
         const int n = it.n_tiles;
         if (n == 0) continue;
-        ok = wait_or_abort(&sh.q_ready, nq & 1, &sh, p.dev_status);      // Q rows in place, dQ^T of the previous item read
+        ok = wait_or_abort(&sh.q_ready, nq & 1, &sh.abort, p.dev_status);      // Q rows in place, dQ^T of the previous item read
         if (!ok) break;
         umma::fence_after_sync();
         auto issue_s = [&](int tt) {                                   // S = K Q^T of tile tt into S buffer tt & 1
@@ -201,18 +201,18 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
           }
           umma::commit(&sh.s_full[tt & 1]);
         };
-        ok = wait_or_abort(&sh.k_full[t % kStages], (t / kStages) & 1, &sh, p.dev_status);
+        ok = wait_or_abort(&sh.k_full[t % kStages], (t / kStages) & 1, &sh.abort, p.dev_status);
         if (!ok) break;
         issue_s(t);
         for (int i = 0; i < n; ++i) {
           const int tt = t + i, buf = tt & 1;
           if (i + 1 < n) {
-            ok = wait_or_abort(&sh.k_full[(tt + 1) % kStages], ((tt + 1) / kStages) & 1, &sh, p.dev_status);
+            ok = wait_or_abort(&sh.k_full[(tt + 1) % kStages], ((tt + 1) / kStages) & 1, &sh.abort, p.dev_status);
             if (!ok) break;
             issue_s(tt + 1);      // its buffer held S and dz of tile tt - 1, whose dK product was issued before this one
           }
-          ok = wait_or_abort(&sh.dz_full[buf], (tt >> 1) & 1, &sh, p.dev_status);
-          if (ok && tt >= 2) ok = wait_or_abort(&sh.dk_empty[buf], ((tt >> 1) - 1) & 1, &sh, p.dev_status);
+          ok = wait_or_abort(&sh.dz_full[buf], (tt >> 1) & 1, &sh.abort, p.dev_status);
+          if (ok && tt >= 2) ok = wait_or_abort(&sh.dk_empty[buf], ((tt >> 1) - 1) & 1, &sh.abort, p.dev_status);
           if (!ok) break;
           umma::fence_after_sync();
           // dK = dz Q: 16 rows per step = 8 packed columns of dz, two 8-row groups of Q
@@ -236,7 +236,7 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
         ++nq;
       }
       umma::commit(&sh.drain);          // everything issued has completed before tensor memory is released
-      wait_or_abort(&sh.drain, 0, &sh, p.dev_status);
+      wait_or_abort(&sh.drain, 0, &sh.abort, p.dev_status);
     }
     __syncwarp();
   } else if (warp < kDkWarp0) {
@@ -248,7 +248,7 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
     bool ok = true;
     float* prev_part = nullptr;                                        // where the dQ^T in tensor memory belongs
     auto flush_dq = [&]() {                                            // the finished item's dQ partial: rows x 128 channels, fp32
-      if (!warp_wait(&sh.dq_full, (nq - 1) & 1, &sh, p.dev_status)) return false;
+      if (!warp_wait(&sh.dq_full, (nq - 1) & 1, &sh.abort, p.dev_status)) return false;
       umma::fence_after_sync();
       uint32_t v[NC];
 #pragma unroll
@@ -262,7 +262,9 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
     };
     for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
       const Item it = decode_item(p, item);
-      float* part = p.dq_part + ((int64_t)it.strip * p.n_split + it.split) * kBwdMaxRows * 128;
+      // with one token range per strip the partial is the gradient itself (the strip's rows are contiguous in grad_q)
+      float* part = p.n_split == 1 ? p.grad_q + ((((int64_t)it.l * p.B + it.b) * p.Hq + it.h * p.g) * p.w) * 128
+                                   : p.dq_part + ((int64_t)it.strip * p.n_split + it.split) * kBwdMaxRows * 128;
       if (it.n_tiles == 0) {                                           // an empty range still owns a partial
         for (int r = 0; r < p.n_rows; ++r) part[r * 128 + row] = 0.f;
         continue;
@@ -303,12 +305,15 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
       bar_sync(1);                                                     // rowc is visible to the four warps
       ++nq;
       const float inv_rows = inv_list_rows(p, T_b);
+      // upstream weights: loaded one tile ahead, turned into P at the end of the tile before
+      float P_next = token_weight_finish(p, token_weight_issue(p, it.b, it.gi, it.tile_lo * kTok + row, T_b, inv_rows));
       for (int i = 0; i < it.n_tiles; ++i) {
         const int tt = t + i, buf = tt & 1;
         const int t_tile = (it.tile_lo + i) * kTok;
         const int t_tok = t_tile + row;
-        const float P = token_weight(p, it.b, it.gi, t_tok, T_b, inv_rows);      // fetched ahead of the wait
-        if (!warp_wait(&sh.s_full[buf], (tt >> 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+        const float P = P_next;
+        const TokenWeightRaw raw_next = token_weight_issue(p, it.b, it.gi, i + 1 < it.n_tiles ? t_tok + kTok : T_b, T_b, inv_rows);
+        if (!warp_wait(&sh.s_full[buf], (tt >> 1) & 1, &sh.abort, p.dev_status)) { ok = false; break; }
         umma::fence_after_sync();
         uint32_t sv[NC];
         const uint32_t s_addr = tmem + lane_base + 64u * buf;
@@ -329,7 +334,7 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
           pk[r >> 1] = ptx::pack_bf16x2(d0, d1);
         }
         // the shared-memory copy below is free once the dQ^T product of two tiles ago has read it
-        if (tt >= 2 && !warp_wait(&sh.dzs_empty[buf], ((tt >> 1) - 1) & 1, &sh, p.dev_status)) { ok = false; break; }
+        if (tt >= 2 && !warp_wait(&sh.dzs_empty[buf], ((tt >> 1) - 1) & 1, &sh.abort, p.dev_status)) { ok = false; break; }
         // dz over the first NC / 2 columns of the S buffer it came from: the A operand of dK ...
 #pragma unroll
         for (int c = 0; c < NC / 2; c += 8) umma::tmem_st8(s_addr + c, pk + c);
@@ -351,6 +356,7 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
         umma::fence_before_sync();
         ptx::fence_proxy_async();
         ptx::mbar_arrive(&sh.dz_full[buf]);
+        P_next = token_weight_finish(p, raw_next);
       }
       t += it.n_tiles;
     }
@@ -371,7 +377,7 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
         const int tt = t + i, buf = tt & 1;
         const int t_tile = (it.tile_lo + i) * kTok;
         const bool full = t_tile + kTok <= T_b;
-        ok = group_all(2, warp_wait(&sh.dk_full[buf], (tt >> 1) & 1, &sh, p.dev_status));
+        ok = group_all(2, warp_wait(&sh.dk_full[buf], (tt >> 1) & 1, &sh.abort, p.dev_status));
         if (!ok) break;
         umma::fence_after_sync();
         const uint32_t d_addr = tmem + lane_base + kTmemDk + 128u * buf;
@@ -426,6 +432,237 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
   }
 }
 
+// ---------------------------------------------------------------- first pass: row statistics
+//
+// The transposed product S^T = Q K^T puts the rows on the lanes of tensor memory and the 128 tokens of a tile on its
+// columns, so that a thread keeps the running (maximum, sum of exponentials, sum of exponentials times P) of ONE row in
+// registers and walks along its tokens without any exchange between threads.  The query rows are stacked 128 / RQ
+// times in the A operand (RQ = 32 or 64 rows, zero padded): copy c of a row sits on lane RQ c + r and its thread takes
+// tokens (128 / copies) c ... of every tile, so all four warps share the exponentials of a tile.  The copies of a row
+// are merged when the item ends.
+struct StatsShared {
+  uint64_t k_full[kStages], k_empty[kStages], s_full[2], s_empty[2], q_ready, drain;
+  uint32_t tmem;
+  int abort;
+  alignas(16) float pw[2][kTok];                  // upstream weights P of the tokens of a tile (read four at a time)
+  float4 part[kTok];                              // per lane: (max, sum, sum * P) at the end of an item
+};
+constexpr int kStatsSmemBytes = kStages * kStageBytes + kStageBytes + 1024;      // K ring + the stacked Q tile
+constexpr int kStatsThreads = 6 * 32;             // producer, MMA, four statistics warps
+constexpr uint32_t kStatsTmemCols = 256;          // S^T [2] at 128 b
+
+template <int RQ>
+__global__ void __launch_bounds__(kStatsThreads, 1)
+score_bwd_stats_umma_kernel(const __grid_constant__ CUtensorMap map_k, BwdParams p, int n_items) {
+  extern __shared__ uint8_t smem_dyn[];
+  __shared__ StatsShared sh;
+  constexpr int kCopies = kTok / RQ, kTpt = kTok / kCopies;      // tokens of a tile per thread
+
+  uint8_t* base = (uint8_t*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage = base;                                 // [kStages][2 boxes of 128 tokens x 64 channels]
+  uint8_t* sQ = stage + kStages * kStageBytes;           // [2 boxes][128 stacked rows x 64 channels]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&sh.k_full[s], 1); ptx::mbar_init(&sh.k_empty[s], 1); }
+#pragma unroll
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&sh.s_full[b], 1); ptx::mbar_init(&sh.s_empty[b], 128); }
+    ptx::mbar_init(&sh.q_ready, 128);
+    ptx::mbar_init(&sh.drain, 1);
+    ptx::fence_barrier_init();
+    sh.abort = 0;
+    ptx::prefetch_tensormap(&map_k);
+  }
+  if (warp == kMmaWarp) umma::tmem_alloc(&sh.tmem, kStatsTmemCols);
+  umma::fence_before_sync();
+  __syncthreads();
+  umma::fence_after_sync();
+  const uint32_t tmem = sh.tmem;
+
+  if (warp == kProducerWarp) {
+    if (lane == 0) {
+      int t = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        const Item it = decode_item(p, item);
+        const int plane = it.l * p.Hkv + it.h;
+        const int row0 = (int)p.seq_off[it.b];
+        for (int i = 0; i < it.n_tiles; ++i, ++t) {
+          const int s = t % kStages;
+          if (t >= kStages && !wait_or_abort(&sh.k_empty[s], ((t / kStages) - 1) & 1, &sh.abort, p.dev_status)) { ok = false; break; }
+          uint8_t* sp = stage + s * kStageBytes;
+          ptx::mbar_expect_tx(&sh.k_full[s], kStageBytes);
+          const int y = row0 + (it.tile_lo + i) * kTok;
+          ptx::tma_load_3d(sp, &map_k, 0, y, plane, &sh.k_full[s]);
+          ptx::tma_load_3d(sp + kBox, &map_k, 64, y, plane, &sh.k_full[s]);
+        }
+      }
+      for (int u = max(0, t - kStages); u < t; ++u) ptx::mbar_wait_bounded(&sh.k_full[u % kStages], (u / kStages) & 1);
+    }
+    __syncwarp();
+  } else if (warp == kMmaWarp) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma::instr_desc(kTok, kTok, false);
+      const uint64_t desc_hi = (uint64_t)umma::smem_desc_sw128(0, 0, 1024) & 0xffffffff00000000ull;
+      const uint32_t st_addr = ptx::smem_u32(stage);
+      const uint32_t q_lo = (ptx::smem_u32(sQ) >> 4) | (1u << 16);
+      int t = 0, nq = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        const Item it = decode_item(p, item);
+        if (it.n_tiles == 0) continue;
+        ok = wait_or_abort(&sh.q_ready, nq & 1, &sh.abort, p.dev_status);
+        if (!ok) break;
+        umma::fence_after_sync();
+        for (int i = 0; i < it.n_tiles; ++i, ++t) {
+          const int buf = t & 1, s = t % kStages;
+          ok = wait_or_abort(&sh.k_full[s], (t / kStages) & 1, &sh.abort, p.dev_status);
+          if (ok && t >= 2) ok = wait_or_abort(&sh.s_empty[buf], ((t >> 1) - 1) & 1, &sh.abort, p.dev_status);
+          if (!ok) break;
+          umma::fence_after_sync();
+          const uint32_t k_lo = ((st_addr + s * kStageBytes) >> 4) | (1u << 16);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (uint32_t)(((ks >> 2) * kBox + (ks & 3) * 32) >> 4);
+            umma::mma_bf16(tmem + 128u * buf, desc_hi | (uint64_t)(q_lo + off), desc_hi | (uint64_t)(k_lo + off), idesc, ks > 0);
+          }
+          umma::commit(&sh.s_full[buf]);
+          umma::commit(&sh.k_empty[s]);
+        }
+        ++nq;
+      }
+      umma::commit(&sh.drain);
+      wait_or_abort(&sh.drain, 0, &sh.abort, p.dev_status);
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ statistics: one thread per (row, copy)
+    const int m = 32 * (warp & 3) + lane;                              // lane of tensor memory
+    const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
+    const int r = m % RQ, tok_lo = (m / RQ) * kTpt;
+    int t = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+      const Item it = decode_item(p, item);
+      float4* out = p.stats + ((int64_t)it.strip * p.n_split + it.split) * kBwdMaxRows;
+      if (it.n_tiles == 0) {
+        if (m < kBwdMaxRows) out[m] = make_float4(-INFINITY, 0.f, 0.f, 0.f);
+        continue;
+      }
+      const int T_b = it.T_b;
+      const float inv_rows = inv_list_rows(p, T_b);
+      // the stacked query tile: stacked row x = copy * RQ + r, 16 pieces of 16 bytes each (every S^T product of the
+      // previous item has completed: its last tile has been read below)
+      const __nv_bfloat16* q_rows = (const __nv_bfloat16*)p.q_recent + ((((int64_t)it.l * p.B + it.b) * p.Hq + it.h * p.g) * p.w) * 128;
+      uint4 qv[RQ / 8];                                                 // RQ rows x 16 pieces over 128 threads, all loads in flight
+#pragma unroll
+      for (int u = 0; u < RQ / 8; ++u) {
+        const int rr = (m + 128 * u) >> 4, piece = m & 15;
+        qv[u] = make_uint4(0, 0, 0, 0);
+        if (rr < p.n_rows) qv[u] = ((const uint4*)(q_rows + (int64_t)rr * 128))[piece];
+      }
+#pragma unroll
+      for (int u = 0; u < RQ / 8; ++u) {
+        const int rr = (m + 128 * u) >> 4, piece = m & 15;
+#pragma unroll
+        for (int c = 0; c < kCopies; ++c) {
+          const int x = c * RQ + rr;
+          *reinterpret_cast<uint4*>(sQ + (piece >> 3) * kBox + x * 128 + (((piece & 7) ^ (x & 7)) << 4)) = qv[u];
+        }
+      }
+      sh.pw[t & 1][m] = token_weight_finish(p, token_weight_issue(p, it.b, it.gi, it.tile_lo * kTok + m, T_b, inv_rows));
+      ptx::fence_proxy_async();
+      ptx::mbar_arrive(&sh.q_ready);
+      const int lim = column_limit(p, r, T_b);
+      float m_run = -INFINITY, s_run = 0.f, n_run = 0.f;              // maximum in raw score units
+      for (int i = 0; i < it.n_tiles; ++i, ++t) {
+        const int buf = t & 1;
+        const int t_tile = (it.tile_lo + i) * kTok;
+        // the next tile's upstream weights: loads now, arithmetic and hand-over at the end of this tile
+        const TokenWeightRaw raw_next = token_weight_issue(p, it.b, it.gi, i + 1 < it.n_tiles ? t_tile + kTok + m : T_b, T_b, inv_rows);
+        ok = group_all(1, warp_wait(&sh.s_full[buf], (t >> 1) & 1, &sh.abort, p.dev_status));   // also: pw[buf] is complete
+        if (!ok) break;
+        umma::fence_after_sync();
+        const bool masked = t_tile + kTok > T_b - p.w;
+#pragma unroll
+        for (int c0 = 0; c0 < kTpt; c0 += 32) {
+          uint32_t v[32];
+          umma::tmem_ld32(tmem + lane_base + 128u * buf + tok_lo + c0, v);
+          umma::tmem_ld_wait();
+          if (c0 + 32 == kTpt) {                          // the thread's share of the buffer is in registers
+            umma::fence_before_sync();
+            ptx::mbar_arrive(&sh.s_empty[buf]);
+          }
+          float z[32];
+          float mx = m_run;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            z[j] = __uint_as_float(v[j]);
+            if (masked && t_tile + tok_lo + c0 + j > lim) z[j] = -INFINITY;
+            mx = fmaxf(mx, z[j]);
+          }
+          if (mx == -INFINITY) continue;                  // nothing visible so far
+          const float neg = -mx * p.scale_log2;
+          const float e_old = ptx::ex2_approx(fmaf(m_run, p.scale_log2, neg));
+          float s_acc = 0.f, n_acc = 0.f;
+          const float4* pw4 = reinterpret_cast<const float4*>(&sh.pw[buf][tok_lo + c0]);
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 P4 = pw4[j >> 2];
+            const float e0 = ptx::ex2_approx(fmaf(z[j], p.scale_log2, neg)), e1 = ptx::ex2_approx(fmaf(z[j + 1], p.scale_log2, neg));
+            const float e2 = ptx::ex2_approx(fmaf(z[j + 2], p.scale_log2, neg)), e3 = ptx::ex2_approx(fmaf(z[j + 3], p.scale_log2, neg));
+            s_acc += (e0 + e1) + (e2 + e3);
+            n_acc = fmaf(e0, P4.x, fmaf(e1, P4.y, fmaf(e2, P4.z, fmaf(e3, P4.w, n_acc))));
+          }
+          s_run = fmaf(s_run, e_old, s_acc);
+          n_run = fmaf(n_run, e_old, n_acc);
+          m_run = mx;
+        }
+        sh.pw[buf ^ 1][m] = token_weight_finish(p, raw_next);        // every thread is past the tile that used this buffer
+      }
+      if (!ok) break;
+      // merge the copies of a row
+      sh.part[m] = make_float4(m_run * p.scale_log2, s_run, n_run, 0.f);
+      bar_sync(1);
+      if (m < kBwdMaxRows) {
+        float mm = -INFINITY, sum = 0.f, num = 0.f;
+        if (m < p.n_rows) {
+#pragma unroll
+          for (int c = 0; c < kCopies; ++c) merge3(mm, sum, num, sh.part[c * RQ + m].x, sh.part[c * RQ + m].y, sh.part[c * RQ + m].z);
+        }
+        out[m] = make_float4(mm, sum, num, 0.f);
+      }
+      bar_sync(1);                                                      // part[] is free again
+    }
+  }
+  umma::fence_before_sync();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    umma::fence_after_sync();
+    umma::tmem_dealloc(tmem, kStatsTmemCols);
+  }
+}
+
+template <int RQ>
+int launch_stats_rq(const CUtensorMap& map_k, const BwdParams& p, int64_t items, cudaStream_t stream) {
+  static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
+  static int sm_count[kMaxDevices] = {0};
+  int dev = -1;
+  const int rc = attr_once.run([&] {
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count[cur], cudaDevAttrMultiProcessorCount, cur);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(score_bwd_stats_umma_kernel<RQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmemBytes);
+    return e;
+  }, &dev);
+  if (rc != NGC_OK) return rc;
+  const int grid = (int)(items < sm_count[dev] ? items : sm_count[dev]);
+  score_bwd_stats_umma_kernel<RQ><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(map_k, p, (int)items);
+  return launch_status();
+}
+
 template <int NC>
 int launch_nc(const Maps& maps, const BwdParams& p, int64_t items, cudaStream_t stream) {
   static PerDeviceOnce attr_once;      // the shared-memory opt-in is stored per device
@@ -451,6 +688,8 @@ int launch_score_bwd_umma(const BwdParams& p, const void* k, void* grad_k, int64
   Maps maps;
   if (!make_kv_map(&maps.k, const_cast<void*>(k), rows, planes, kTok) || !make_kv_map(&maps.gk, grad_k, rows, planes, kTok))
     return NGC_ERR_UNSUPPORTED;
+  const int rc = p.n_rows <= 32 ? launch_stats_rq<32>(maps.k, p, items, stream) : launch_stats_rq<64>(maps.k, p, items, stream);
+  if (rc != NGC_OK) return rc;
   if (p.n_rows <= 16) return launch_nc<16>(maps, p, items, stream);
   if (p.n_rows <= 32) return launch_nc<32>(maps, p, items, stream);
   return launch_nc<48>(maps, p, items, stream);

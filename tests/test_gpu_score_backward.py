@@ -70,6 +70,16 @@ def test_score_backward_token_ranges_and_unsupported_shapes():
         b.ngc_score_evict_backward(dc, qr, 1, 1, torch.zeros((1, 1, 10), device="cuda"), torch.zeros_like(qr), torch.zeros_like(dc.k))
 
 
+def test_score_backward_many_short_strips_write_grad_q_directly():
+    """More strips than the kernels want items: no strip is cut into token ranges and the gradient pass writes
+    grad_q itself (no partials, no reduction launch)."""
+    rng = np.random.default_rng(7)
+    lens = [int(x) for x in rng.integers(0, 300, size=80)]
+    lens[3] = 0
+    lens[5] = 128
+    run_case(4, 80, 4, 2, 3, lens, 1, 32, 0, seed=11)
+
+
 def test_score_backward_with_a_length_per_layer():
     """Per-layer lists whose layers hold different numbers of tokens: every layer against the oracle run on it alone."""
     b = ngc()
