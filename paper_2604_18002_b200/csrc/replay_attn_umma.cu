@@ -566,11 +566,16 @@ replay_attn_umma_kernel(const __grid_constant__ Maps maps, ReplayAttnParams p, i
         const int t_w0 = q0 + 32 * (warp & 3);                                // query token of this warp's row 0
         const int64_t o_row0 = ((((int64_t)pl.l * p.B + pl.b) * p.Hq + pl.hq0 + hh) * (int64_t)p.t_max + t_w0) * 128;
         const bool whole = t_w0 + 32 <= T_b;
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t o[32];
-          umma::tmem_ld32(o_addr + c0, o);
+        // The chunk after the current one is already on its way out of tensor memory while this one is scaled,
+        // packed and handed to the TMA unit.
+        uint32_t ob[2][32];
+        umma::tmem_ld32(o_addr, ob[0]);
+#pragma unroll
+        for (int ci = 0; ci < 4; ++ci) {
+          const int c0 = 32 * ci;
+          uint32_t (&o)[32] = ob[ci & 1];
           umma::tmem_ld_wait();
+          if (ci < 3) umma::tmem_ld32(o_addr + c0 + 32, ob[(ci + 1) & 1]);
           if (lane == 0) ptx::bulk_wait_read<0>();                            // the previous chunk's store has read the staging area
           __syncwarp();
           if (p.out_bf16) {
