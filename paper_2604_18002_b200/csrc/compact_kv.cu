@@ -20,6 +20,7 @@
 // 256 bytes each, are limited by the copy engine's request rate; a cp.async
 // gather into a shared-memory ring with one bulk store per 16 KB tile.)
 #include "ngc_common.cuh"
+#include "ptx.cuh"
 
 namespace ngc {
 namespace {
@@ -213,7 +214,9 @@ __global__ void compact_check_kernel(CompactParams p) {
 
 // After all strips moved: the lengths become the kept token counts (one CTA per sequence, a warp per
 // list; every list is re-validated).  With one length per sequence the lists must agree; with a
-// length per list each list gets its own count.
+// length per list each list gets its own count.  Launched as a programmatic dependent of the strip
+// kernel: the lists are checked while the last strips are still moving (neither kernel writes what the
+// other reads there), the lengths are written only after the strip kernel has completed.
 __global__ void compact_lens_kernel(CompactParams p) {
   __shared__ int s_bad, s_min, s_max;
   const int b = blockIdx.x;
@@ -221,6 +224,7 @@ __global__ void compact_lens_kernel(CompactParams p) {
   const bool per_list = p.lens_lists != 0;          // then lens_lists == lists: every list has its own length
   if (!per_list && p.lens[b] < 0) {                 // marked by the check kernel: put the length back, nothing moved
     __syncthreads();                                // (every thread has read the entry)
+    ptx::grid_dep_wait();
     if (threadIdx.x == 0) const_cast<int32_t*>(p.lens)[b] = ~p.lens[b];
     return;
   }
@@ -230,12 +234,14 @@ __global__ void compact_lens_kernel(CompactParams p) {
   for (int gi = warp; gi < p.G; gi += n_warps) {
     int32_t* len_p = const_cast<int32_t*>(p.lens) + (per_list ? (int64_t)b * p.G + gi : b);
     const int t = validate_list_warp(p.kept_sorted + ((int64_t)b * p.G + gi) * p.k_max, K, p.k_max, *len_p, p.block);
+    ptx::grid_dep_wait();                        // every strip has moved (and read its length)
     if ((threadIdx.x & 31) == 0) {
       if (t < 0) atomicOr(&s_bad, 1);            // already reported by the strip kernel
       else if (per_list) *len_p = t;             // lists may keep different token counts (a short last unit)
       else { atomicMin(&s_min, t); atomicMax(&s_max, t); }
     }
   }
+  ptx::grid_dep_wait();
   __syncthreads();
   if (threadIdx.x == 0 && !per_list && !s_bad) {
     if (s_min != s_max) set_dev_status(p.dev_status, NGC_DEV_LISTS_DISAGREE);
@@ -354,7 +360,7 @@ extern "C" int ngc_compact_kv(ngc_cache* c, const int32_t* kept_sorted, const in
   else compact_kernel<32><<<(unsigned)strips, kThreads, 0, (cudaStream_t)stream>>>(p);
   int rc = launch_status();
   if (rc != NGC_OK) return rc;
-  compact_lens_kernel<<<c->B, lens_threads, 0, (cudaStream_t)stream>>>(p);
+  NGC_CUDA_TRY(launch_pdl(compact_lens_kernel, dim3((unsigned)c->B), dim3(lens_threads), 0, (cudaStream_t)stream, p));
   return launch_status();
 }
 
