@@ -70,6 +70,17 @@ def test_score_backward_token_ranges_and_unsupported_shapes():
         b.ngc_score_evict_backward(dc, qr, 1, 1, torch.zeros((1, 1, 10), device="cuda"), torch.zeros_like(qr), torch.zeros_like(dc.k))
 
 
+@pytest.mark.parametrize("Hq,Hkv,w,lens", [
+    (16, 2, 5, [127, 128, 129, 255, 256, 257, 1, 4]),      # 40 rows, the widest strip; lengths around the 128-token tiles;
+                                                           # fewer tokens than window queries
+    (4, 2, 16, [15, 16, 17, 384]),                         # exactly 32 rows with the longest window
+    (12, 2, 5, [0, 2, 640]),                               # an empty sequence beside live ones
+])
+def test_score_backward_tile_edges_and_row_counts(Hq, Hkv, w, lens):
+    run_case(2, len(lens), Hq, Hkv, w, lens, 1, 1, 0, seed=3 * Hq + w)
+    run_case(1, len(lens), Hq, Hkv, w, lens, 2, 8, 1, seed=5 * Hq + w)
+
+
 def test_score_backward_many_short_strips_write_grad_q_directly():
     """More strips than the kernels want items: no strip is cut into token ranges and the gradient pass writes
     grad_q itself (no partials, no reduction launch)."""
