@@ -115,22 +115,31 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
   const int64_t cap = p.seq_off[b + 1] - p.seq_off[b];        // rows this sequence owns in the plane
 #endif
   uint4 cur[kVecPerThread], nxt[kVecPerThread];
+  int src_nxt[kVecPerThread];          // source rows of the tile whose data is fetched next (-1: no such row)
 
-  auto load_tile = [&](int t0, uint4 (&r)[kVecPerThread]) {
+  // The source row of an output row comes from the kept list, which may itself come from HBM (a list per layer and
+  // head): the indices are fetched one tile ahead of the rows they address, the rows one tile ahead of their store.
+  auto load_sources = [&](int t0, int (&src)[kVecPerThread]) {
 #pragma unroll
     for (int u = 0; u < kVecPerThread; ++u) {
       const int jt = t0 + u * kRowsPerPass + my_row;
+      src[u] = -1;
       if (jt < tokens) {
-        int64_t src;
         if (block == 1) {
-          src = kept[jt];
+          src[u] = __ldg(kept + jt);
         } else {
           const int unit = jt / block;
-          src = (int64_t)kept[unit] * block + (jt - unit * block);
+          src[u] = __ldg(kept + unit) * block + (jt - unit * block);      // < len: validated above
         }
-        // a kept row never lies in front of its destination, and always inside the live part of the strip
-        if (NGC_IN_BOUNDS(p.dev_status, src >= jt && src < len && src < cap)) r[u] = __ldcs(strip + src * RV);
       }
+    }
+  };
+  auto load_tile = [&](int t0, const int (&src)[kVecPerThread], uint4 (&r)[kVecPerThread]) {
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) {
+      const int jt = t0 + u * kRowsPerPass + my_row;
+      // a kept row never lies in front of its destination, and always inside the live part of the strip
+      if (src[u] >= 0 && NGC_IN_BOUNDS(p.dev_status, src[u] >= jt && src[u] < len && src[u] < cap)) r[u] = __ldcs(strip + (int64_t)src[u] * RV);
     }
   };
   auto store_tile = [&](int t0, const uint4 (&r)[kVecPerThread]) {
@@ -143,9 +152,14 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactParams p) {
 
   int t0 = first_moved;
   if (t0 >= tokens) return;
-  load_tile(t0, cur);
+  load_sources(t0, src_nxt);
+  load_tile(t0, src_nxt, cur);
+  load_sources(t0 + kTileRows, src_nxt);
   for (; t0 < tokens; t0 += kTileRows) {
-    if (t0 + kTileRows < tokens) load_tile(t0 + kTileRows, nxt);
+    if (t0 + kTileRows < tokens) {
+      load_tile(t0 + kTileRows, src_nxt, nxt);
+      load_sources(t0 + 2 * kTileRows, src_nxt);
+    }
     __syncthreads();            // every load of this tile has completed
     store_tile(t0, cur);
 #pragma unroll
@@ -160,16 +174,17 @@ __device__ int validate_list_warp(const int32_t* kept, int K, int k_max, int len
   const int n_units = (len + block - 1) / block;
   if (K < 0 || K > k_max || K > n_units) return -1;
   bool bad = false;
-  for (int jb = 0; jb < K; jb += 128) {          // four independent loads per lane in flight
-    int u[4];
+  constexpr int kE = 16;                          // independent loads per lane in flight: a list may come from HBM
+  for (int jb = 0; jb < K; jb += 32 * kE) {
+    int u[kE];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
+    for (int e = 0; e < kE; ++e) {
       const int j = jb + 32 * e + lane;
       u[e] = j < K ? kept[j] : 0x7fffffff;
     }
-    int edge = (lane < 4 && jb + 32 * lane > 0 && jb + 32 * lane < K) ? kept[jb + 32 * lane - 1] : -1;
+    int edge = (lane < kE && jb + 32 * lane > 0 && jb + 32 * lane < K) ? kept[jb + 32 * lane - 1] : -1;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
+    for (int e = 0; e < kE; ++e) {
       const int j = jb + 32 * e + lane;
       int prev = __shfl_up_sync(0xffffffffu, u[e], 1);
       const int first_prev = __shfl_sync(0xffffffffu, edge, e);
