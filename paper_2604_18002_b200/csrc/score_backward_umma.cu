@@ -405,14 +405,14 @@ score_bwd_umma_kernel(const __grid_constant__ Maps maps, BwdParams p, int n_item
                                           ptx::pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7])));
               if (full)
                 *reinterpret_cast<uint4*>(so + row * 128 + (((4 * cc + q) ^ (row & 7)) << 4)) = w4;
-              else if (t_tile + row < T_b)
+              else if (t_tile + row < T_b && NGC_IN_BOUNDS(p.dev_status, row0 + t_tile + row < p.rows_R))
                 *reinterpret_cast<uint4*>(gk_strip + (int64_t)(t_tile + row) * 128 + 64 * half + 32 * cc + 8 * q) = w4;
             }
           }
           if (full) {
             ptx::fence_proxy_async();                     // written through the generic proxy, read by the TMA store
             bar_sync(2);
-            if (leader) {
+            if (leader && NGC_IN_BOUNDS(p.dev_status, row0 + t_tile + kTok <= p.rows_R && plane < p.L * p.Hkv)) {
               ptx::tma_store_3d(&maps.gk, 64 * half, row0 + t_tile, plane, so);
               ptx::bulk_commit();
             }
