@@ -722,6 +722,13 @@ def run_reference(args):
         return
     import oracle
     oracle.build()
+    if "LOCAL_RANK" in os.environ and oracle.threads() == 1:
+        # the multi-rank launcher pins OpenMP to one thread per rank; this arm runs on rank 0 alone, on the host's cores
+        import ctypes
+        try:
+            ctypes.CDLL("libgomp.so.1").omp_set_num_threads(len(os.sched_getaffinity(0)))
+        except OSError:
+            pass
     n_seqs, dsteps = args.cpu_seqs, args.cpu_decode_steps
     data = make_cpu_sample(n_seqs, dsteps)
     for w in range(args.warmup):
