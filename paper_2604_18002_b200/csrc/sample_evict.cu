@@ -91,6 +91,7 @@ __global__ void sample_kernel(SampleParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int s_flag;
   __shared__ int s_warp_tot[32];
+  __shared__ int s_sel[2][32];
   __shared__ int s_carry;
 
   const int li = blockIdx.x;
@@ -182,23 +183,97 @@ __global__ void sample_kernel(SampleParams p) {
     // Thread t owns the `per` consecutive positions [t*per, (t+1)*per) of the order (per a power of
     // two); position i is STORED at (i % per) * nthr + i / per, so that the lanes of a warp walking
     // their runs in step touch consecutive shared-memory words.
-    int per_log = 0;
-    while ((nthr << per_log) < n_cand) ++per_log;
-    const int per = 1 << per_log;
     uint16_t* src = idx_a;
     uint16_t* dst = idx_b;
-    for (int k = 0; k < per; ++k) {
-      const int i = tid * per + k;
-      if (i < n_cand) src[k * nthr + tid] = (uint16_t)i;
+    uint32_t* cnt_words = reinterpret_cast<uint32_t*>(hist);
+    int n_sort = n_cand;                 // candidates that take part in the sort
+    uint32_t img_base = 0;               // the sort runs on img - img_base ...
+    int n_bits = 32;                     // ... whose values need this many bits
+    // Long lists of which at most three quarters are drawn: only candidates that can be drawn are sorted.  The
+    // Kp-th largest image is found bit by bit (32 counting rounds over values held in registers); the candidates
+    // at or above it are laid out in index order, so the stable sort below treats equal keys exactly as a sort
+    // of the whole list would, and the sort keys are taken relative to that image, which shortens them.
+    const bool preselect = nthr == 1024 && n_cand > 8192 && Kp > 0 && 4 * (int64_t)Kp <= 3 * (int64_t)n_cand;
+    if (preselect) {
+      uint32_t v[16];                    // candidates tid, tid + 1024, ...: images (0 = no such candidate; real images are > 0)
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int i = tid + (k << 10);
+        v[k] = i < n_cand ? img[i] : 0u;
+      }
+      uint32_t piv = 0, mx = 0;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) mx = max(mx, v[k]);
+      mx = __reduce_max_sync(0xffffffffu, mx);
+      if (lane == 0) s_warp_tot[warp] = (int)mx;
+      __syncthreads();
+      mx = __reduce_max_sync(0xffffffffu, (uint32_t)s_warp_tot[lane]);
+      for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t tr = piv | (1u << bit);
+        int c = 0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) c += v[k] >= tr ? 1 : 0;
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (lane == 0) s_sel[bit & 1][warp] = c;
+        __syncthreads();                 // (the other half of s_sel is rewritten only after the next barrier)
+        if (__reduce_add_sync(0xffffffffu, s_sel[bit & 1][lane]) >= Kp) piv = tr;
+      }
+      // positions of the surviving candidates in index order: index = 1024 k + 32 warp + lane
+      int* s_cnt = reinterpret_cast<int*>(cnt_words);          // [16][32 warps]; free until the sort starts
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const uint32_t bal = __ballot_sync(0xffffffffu, v[k] >= piv);
+        if (lane == 0) s_cnt[k * 32 + warp] = __popc(bal);
+      }
+      __syncthreads();
+      {
+        const int x = tid < 512 ? s_cnt[tid] : 0;
+        int incl = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_warp_tot[warp] = incl;
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int w2 = 0; w2 < 16; ++w2) { const int t = s_warp_tot[w2]; total += t; if (w2 < warp) before += t; }
+        if (tid < 512) s_cnt[tid] = before + incl - x;
+        n_sort = total;
+        __syncthreads();
+      }
+      img_base = piv;
+      n_bits = 32 - __clz(mx - piv);                           // 0: every survivor has the same key
+    }
+    int per_log = 0;
+    while ((nthr << per_log) < n_sort) ++per_log;
+    const int per = 1 << per_log;
+    if (preselect) {
+      const int* s_cnt = reinterpret_cast<const int*>(cnt_words);
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int i = tid + (k << 10);
+        const bool keep = i < n_cand && img[i] >= img_base;
+        const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+        if (keep) {
+          const int pos = s_cnt[k * 32 + warp] + __popc(bal & ((1u << lane) - 1u));
+          src[(pos & (per - 1)) * nthr + (pos >> per_log)] = (uint16_t)i;
+        }
+      }
+      __syncthreads();                   // s_cnt is read before the counters are cleared
+    } else {
+      for (int k = 0; k < per; ++k) {
+        const int i = tid * per + k;
+        if (i < n_cand) src[k * nthr + tid] = (uint16_t)i;
+      }
     }
     // counter x = digit * nthr + thread sits at cnt[x + 2 * (x >> 5)]: one pad word per 32 counters, so that
     // the 32 consecutive counters a thread scans start in a different bank for every lane
-    uint32_t* cnt_words = reinterpret_cast<uint32_t*>(hist);
-    for (int shift = 0; shift < 32 && Kp > 0; shift += 5) {
+    for (int shift = 0; shift < n_bits && Kp > 0; shift += 5) {
       for (int i = tid; i < 17 * nthr; i += nthr) cnt_words[i] = 0u;
       __syncthreads();
-      for (int k = 0; k < per && tid * per + k < n_cand; ++k) {
-        const uint32_t d = 31u - ((img[src[k * nthr + tid]] >> shift) & 31u);
+      for (int k = 0; k < per && tid * per + k < n_sort; ++k) {
+        const uint32_t d = 31u - (((img[src[k * nthr + tid]] - img_base) >> shift) & 31u);
         const uint32_t x = d * nthr + tid;
         hist[x + 2 * (x >> 5)] += 1;
       }
@@ -227,9 +302,9 @@ __global__ void sample_kernel(SampleParams p) {
         }
       }
       __syncthreads();
-      for (int k = 0; k < per && tid * per + k < n_cand; ++k) {
+      for (int k = 0; k < per && tid * per + k < n_sort; ++k) {
         const uint16_t cand = src[k * nthr + tid];
-        const uint32_t d = 31u - ((img[cand] >> shift) & 31u);
+        const uint32_t d = 31u - (((img[cand] - img_base) >> shift) & 31u);
         const uint32_t x = d * nthr + tid;
         const uint32_t pos = hist[x + 2 * (x >> 5)]++;
         dst[(pos & (per - 1)) * nthr + (pos >> per_log)] = cand;

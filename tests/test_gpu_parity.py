@@ -43,6 +43,35 @@ def test_sample_bit_exact(B, G, n_max, std):
         assert np.array_equal(got[2], ref[2]), "keep_mask"
 
 
+@pytest.mark.parametrize("kind", ["quantised", "constant", "infinite", "few_distinct"])
+def test_sample_long_lists_with_ties_around_the_selection_threshold(kind):
+    """Lists long enough for the pre-selection of drawable candidates (more than 8192 candidates, at most three
+    quarters drawn): equal keys at the threshold must still go to the smaller index, and budgets on both sides of
+    the three-quarter rule take both code paths."""
+    B, G, n_max = 6, 2, 16384
+    rng = np.random.default_rng(5)
+    logits = synth.make_logits(B, G, n_max, seed=21).numpy()
+    if kind == "quantised":
+        logits = np.round(logits * 4.0).astype(np.float32) / 4.0          # many exact ties (greedy), few in sampled mode
+    elif kind == "constant":
+        logits[:] = -1.5
+    elif kind == "infinite":
+        logits[:, :, ::3] = -np.inf
+        logits[:, :, 5::97] = np.inf
+    else:
+        logits = rng.integers(0, 3, logits.shape).astype(np.float32)      # three distinct values
+    n = np.array([16384, 16384, 12000, 8193, 9000, 16000], np.int32)
+    P = np.array([0, 100, 0, 1, 0, 4000], np.int32)
+    K = np.array([8192, 8292, 9000, 4097, 6751, 13000], np.int32)          # list 4: just over three quarters; list 5: P > 0
+    k_max = int(K.max())
+    for greedy in (1, 0):
+        ref = oracle.sample_evict(logits, n, P, K, k_max, seed=9, rnd=3, greedy=greedy, list_base=2)
+        got = gpu_sample(logits, n, P, K, k_max, seed=9, rnd=3, greedy=greedy, list_base=2)
+        assert got[3] == 0 and not ref[3].any()
+        for i in range(3):
+            assert np.array_equal(got[i], ref[i]), (kind, greedy, i)
+
+
 def test_sample_large_list_uses_workspace():
     B, G, n_max = 2, 1, 40000
     logits = synth.make_logits(B, G, n_max, seed=3).numpy()
