@@ -354,6 +354,9 @@ __global__ void sample_kernel(SampleParams p) {
   __syncthreads();
 
   // ---- ascending kept list from the prefix popcounts of the bitmap ----
+  // (radix path: assembled in shared memory over the order arrays, which are dead by now, and written out in one
+  // coalesced sweep; a thread's own run of up to 32 entries would otherwise go out as 32 strided stores)
+  uint16_t* ks_stage = kRadix ? idx_b : nullptr;
   if (tid == 0) s_carry = 0;
   __syncthreads();
   for (int base = 0; base < n_words; base += nthr) {
@@ -375,7 +378,10 @@ __global__ void sample_kernel(SampleParams p) {
     while (mm) {
       const int bit = __ffs(mm) - 1;
       mm &= mm - 1;
-      if (NGC_IN_BOUNDS(p.dev_status, pos >= 0 && pos < p.k_max)) ks[pos] = (wd << 5) + bit;
+      if (NGC_IN_BOUNDS(p.dev_status, pos >= 0 && pos < p.k_max)) {
+        if (kRadix) ks_stage[pos] = (uint16_t)((wd << 5) + bit);
+        else ks[pos] = (wd << 5) + bit;
+      }
       ++pos;
     }
     __syncthreads();
@@ -386,6 +392,8 @@ __global__ void sample_kernel(SampleParams p) {
     }
     __syncthreads();
   }
+  if (kRadix)
+    for (int j = tid; j < K && j < p.k_max; j += nthr) ks[j] = (int)ks_stage[j];
   for (int j = K + tid; j < p.k_max; j += nthr) ks[j] = -1;
   if (km) {
     for (int i = tid; i < p.n_max; i += nthr)
