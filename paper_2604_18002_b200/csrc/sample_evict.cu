@@ -174,25 +174,28 @@ __global__ void sample_kernel(SampleParams p) {
     return;
   }
 
-  int order_per_log = 0, order_per = 1;        // how the sorted order is laid out (radix path)
+  int order_per = 1;                           // how the sorted order is laid out (radix path)
+  uint32_t order_inv = 0;
   if (kRadix) {
     // ---- stable LSD radix sort of the candidate order, descending image: 7 passes of 5 bits ----
     // Thread t owns the consecutive candidates [t*per, (t+1)*per) and a private counter per digit,
     // cnt[digit][t]; in (digit, thread) order the counters' prefix sums are the stable output
     // offsets.  No atomics, no inter-thread traffic inside the counting and scattering walks.
-    // Thread t owns the `per` consecutive positions [t*per, (t+1)*per) of the order (per a power of
-    // two); position i is STORED at (i % per) * nthr + i / per, so that the lanes of a warp walking
-    // their runs in step touch consecutive shared-memory words.
+    // Thread t owns the `per` consecutive positions [t*per, (t+1)*per) of the order; position i is
+    // STORED at (i % per) * nthr + i / per, so that the lanes of a warp walking their runs in step
+    // touch consecutive shared-memory words (the division is a multiplication by ceil(2^32 / per)).
     uint16_t* src = idx_a;
     uint16_t* dst = idx_b;
     uint32_t* cnt_words = reinterpret_cast<uint32_t*>(hist);
     int n_sort = n_cand;                 // candidates that take part in the sort
     uint32_t img_base = 0;               // the sort runs on img - img_base ...
     int n_bits = 32;                     // ... whose values need this many bits
-    // Long lists of which at most three quarters are drawn: only candidates that can be drawn are sorted.  The
-    // Kp-th largest image is found bit by bit (32 counting rounds over values held in registers); the candidates
-    // at or above it are laid out in index order, so the stable sort below treats equal keys exactly as a sort
-    // of the whole list would, and the sort keys are taken relative to that image, which shortens them.
+    // Long lists of which at most three quarters are drawn: only candidates that can be drawn are sorted.  An
+    // image at or below the Kp-th largest is found bit by bit (counting rounds over values held in registers) and
+    // the search stops as soon as at most Kp + Kp / 16 candidates lie at or above it: the few extra candidates cost
+    // less in the sort than the remaining rounds would.  The survivors are laid out in index order, so the stable
+    // sort below treats equal keys exactly as a sort of the whole list would, and the sort keys are taken relative
+    // to that image, which shortens them.
     const bool preselect = nthr == 1024 && n_cand > 8192 && Kp > 0 && 4 * (int64_t)Kp <= 3 * (int64_t)n_cand;
     if (preselect) {
       uint32_t v[16];                    // candidates tid, tid + 1024, ...: images (0 = no such candidate; real images are > 0)
@@ -208,6 +211,7 @@ __global__ void sample_kernel(SampleParams p) {
       if (lane == 0) s_warp_tot[warp] = (int)mx;
       __syncthreads();
       mx = __reduce_max_sync(0xffffffffu, (uint32_t)s_warp_tot[lane]);
+      int cnt_piv = n_cand;
       for (int bit = 31; bit >= 0; --bit) {
         const uint32_t tr = piv | (1u << bit);
         int c = 0;
@@ -216,7 +220,9 @@ __global__ void sample_kernel(SampleParams p) {
         c = __reduce_add_sync(0xffffffffu, c);
         if (lane == 0) s_sel[bit & 1][warp] = c;
         __syncthreads();                 // (the other half of s_sel is rewritten only after the next barrier)
-        if (__reduce_add_sync(0xffffffffu, s_sel[bit & 1][lane]) >= Kp) piv = tr;
+        const int tot = __reduce_add_sync(0xffffffffu, s_sel[bit & 1][lane]);
+        if (tot >= Kp) { piv = tr; cnt_piv = tot; }
+        if (cnt_piv <= Kp + (Kp >> 4)) break;            // close enough: a few more candidates than needed go into the sort
       }
       // positions of the surviving candidates in index order: index = 1024 k + 32 warp + lane
       int* s_cnt = reinterpret_cast<int*>(cnt_words);          // [16][32 warps]; free until the sort starts
@@ -245,9 +251,12 @@ __global__ void sample_kernel(SampleParams p) {
       img_base = piv;
       n_bits = 32 - __clz(mx - piv);                           // 0: every survivor has the same key
     }
-    int per_log = 0;
-    while ((nthr << per_log) < n_sort) ++per_log;
-    const int per = 1 << per_log;
+    const int per = max(1, (n_sort + nthr - 1) / nthr);
+    const uint32_t per_inv = per > 1 ? 0xFFFFFFFFu / (uint32_t)per + 1u : 0u;
+    auto slot = [&](uint32_t pos) {
+      const uint32_t t = per > 1 ? __umulhi(pos, per_inv) : pos;
+      return (pos - t * (uint32_t)per) * (uint32_t)nthr + t;
+    };
     if (preselect) {
       const int* s_cnt = reinterpret_cast<const int*>(cnt_words);
 #pragma unroll
@@ -257,7 +266,7 @@ __global__ void sample_kernel(SampleParams p) {
         const uint32_t bal = __ballot_sync(0xffffffffu, keep);
         if (keep) {
           const int pos = s_cnt[k * 32 + warp] + __popc(bal & ((1u << lane) - 1u));
-          src[(pos & (per - 1)) * nthr + (pos >> per_log)] = (uint16_t)i;
+          src[slot((uint32_t)pos)] = (uint16_t)i;
         }
       }
       __syncthreads();                   // s_cnt is read before the counters are cleared
@@ -307,13 +316,13 @@ __global__ void sample_kernel(SampleParams p) {
         const uint32_t d = 31u - (((img[cand] - img_base) >> shift) & 31u);
         const uint32_t x = d * nthr + tid;
         const uint32_t pos = hist[x + 2 * (x >> 5)]++;
-        dst[(pos & (per - 1)) * nthr + (pos >> per_log)] = cand;
+        dst[slot(pos)] = cand;
       }
       __syncthreads();
       uint16_t* t = src; src = dst; dst = t;
     }
     idx_a = src;        // the sorted order
-    order_per_log = per_log; order_per = per;
+    order_per = per; order_inv = per_inv;
   } else {
     // ---- bitonic sort, descending ----
     for (int k = 2; k <= pad; k <<= 1) {
@@ -344,7 +353,8 @@ __global__ void sample_kernel(SampleParams p) {
   for (int j = tid; j < p.k_max; j += nthr) {
     int idx = -1;
     if (j < Kp) {
-      idx = kRadix ? P + (int)idx_a[(j & (order_per - 1)) * nthr + (j >> order_per_log)]
+      const uint32_t jt = order_per > 1 ? __umulhi((uint32_t)j, order_inv) : (uint32_t)j;
+      idx = kRadix ? P + (int)idx_a[((uint32_t)j - jt * (uint32_t)order_per) * (uint32_t)nthr + jt]
                    : (int)(0xFFFFFFFFu - (uint32_t)(keys[j] & 0xFFFFFFFFull));
       if (NGC_IN_BOUNDS(p.dev_status, idx >= P && idx < n)) atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
       else idx = -1;
