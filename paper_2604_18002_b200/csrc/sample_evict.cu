@@ -111,16 +111,18 @@ __global__ void sample_kernel(SampleParams p) {
   uint16_t* idx_a = nullptr;           // [n_max] candidate order, ping
   uint16_t* idx_b = nullptr;           // [n_max] pong
   uint16_t* hist = nullptr;            // [32 digits][threads] private digit counts, then output offsets (padded)
+  uint8_t* dig = nullptr;              // [n_max] digit of the candidate at each position of the order, kept from the counting walk
   unsigned long long* keys = nullptr;  // composite keys (bitonic)
   uint32_t* bitmap;
   if (kRadix) {
     const int n_al = (p.n_max + 7) & ~7;
-    const int n_slots = max(p.pad_max, nthr);          // order arrays: a power-of-two run per thread
+    const int n_slots = max(p.pad_max, nthr) + 64;     // order arrays: a run per thread, rows of nthr + 2 entries
     img = reinterpret_cast<uint32_t*>(smem_raw);
     idx_a = reinterpret_cast<uint16_t*>(smem_raw + (size_t)n_al * 4);
     idx_b = idx_a + n_slots;
     hist = idx_b + n_slots;
     bitmap = reinterpret_cast<uint32_t*>(hist + 34 * nthr);
+    dig = reinterpret_cast<uint8_t*>(bitmap + ((p.n_max + 31) >> 5));
   } else {
     keys = p.ws_keys + (int64_t)li * p.pad_max;
     bitmap = reinterpret_cast<uint32_t*>(smem_raw);
@@ -182,8 +184,10 @@ __global__ void sample_kernel(SampleParams p) {
     // cnt[digit][t]; in (digit, thread) order the counters' prefix sums are the stable output
     // offsets.  No atomics, no inter-thread traffic inside the counting and scattering walks.
     // Thread t owns the `per` consecutive positions [t*per, (t+1)*per) of the order; position i is
-    // STORED at (i % per) * nthr + i / per, so that the lanes of a warp walking their runs in step
-    // touch consecutive shared-memory words (the division is a multiplication by ceil(2^32 / per)).
+    // STORED at (i % per) * (nthr + 2) + i / per, so that the lanes of a warp walking their runs in step
+    // touch consecutive shared-memory words, and consecutive positions (survivors laid out in order, the
+    // ranks read at the end) fall into consecutive banks: row stride nthr + 2 entries = one bank more per row.
+    // (The division is a multiplication by ceil(2^32 / per).)
     uint16_t* src = idx_a;
     uint16_t* dst = idx_b;
     uint32_t* cnt_words = reinterpret_cast<uint32_t*>(hist);
@@ -255,7 +259,7 @@ __global__ void sample_kernel(SampleParams p) {
     const uint32_t per_inv = per > 1 ? 0xFFFFFFFFu / (uint32_t)per + 1u : 0u;
     auto slot = [&](uint32_t pos) {
       const uint32_t t = per > 1 ? __umulhi(pos, per_inv) : pos;
-      return (pos - t * (uint32_t)per) * (uint32_t)nthr + t;
+      return (pos - t * (uint32_t)per) * (uint32_t)(nthr + 2) + t;
     };
     if (preselect) {
       const int* s_cnt = reinterpret_cast<const int*>(cnt_words);
@@ -273,7 +277,7 @@ __global__ void sample_kernel(SampleParams p) {
     } else {
       for (int k = 0; k < per; ++k) {
         const int i = tid * per + k;
-        if (i < n_cand) src[k * nthr + tid] = (uint16_t)i;
+        if (i < n_cand) src[k * (nthr + 2) + tid] = (uint16_t)i;
       }
     }
     // counter x = digit * nthr + thread sits at cnt[x + 2 * (x >> 5)]: one pad word per 32 counters, so that
@@ -282,7 +286,8 @@ __global__ void sample_kernel(SampleParams p) {
       for (int i = tid; i < 17 * nthr; i += nthr) cnt_words[i] = 0u;
       __syncthreads();
       for (int k = 0; k < per && tid * per + k < n_sort; ++k) {
-        const uint32_t d = 31u - (((img[src[k * nthr + tid]] - img_base) >> shift) & 31u);
+        const uint32_t d = 31u - (((img[src[k * (nthr + 2) + tid]] - img_base) >> shift) & 31u);
+        dig[k * nthr + tid] = (uint8_t)d;                       // the scattering walk below needs no second gather
         const uint32_t x = d * nthr + tid;
         hist[x + 2 * (x >> 5)] += 1;
       }
@@ -312,8 +317,8 @@ __global__ void sample_kernel(SampleParams p) {
       }
       __syncthreads();
       for (int k = 0; k < per && tid * per + k < n_sort; ++k) {
-        const uint16_t cand = src[k * nthr + tid];
-        const uint32_t d = 31u - (((img[cand] - img_base) >> shift) & 31u);
+        const uint16_t cand = src[k * (nthr + 2) + tid];
+        const uint32_t d = dig[k * nthr + tid];
         const uint32_t x = d * nthr + tid;
         const uint32_t pos = hist[x + 2 * (x >> 5)]++;
         dst[slot(pos)] = cand;
@@ -354,7 +359,7 @@ __global__ void sample_kernel(SampleParams p) {
     int idx = -1;
     if (j < Kp) {
       const uint32_t jt = order_per > 1 ? __umulhi((uint32_t)j, order_inv) : (uint32_t)j;
-      idx = kRadix ? P + (int)idx_a[((uint32_t)j - jt * (uint32_t)order_per) * (uint32_t)nthr + jt]
+      idx = kRadix ? P + (int)idx_a[((uint32_t)j - jt * (uint32_t)order_per) * (uint32_t)(nthr + 2) + jt]
                    : (int)(0xFFFFFFFFu - (uint32_t)(keys[j] & 0xFFFFFFFFull));
       if (NGC_IN_BOUNDS(p.dev_status, idx >= P && idx < n)) atomicOr(&bitmap[idx >> 5], 1u << (idx & 31));
       else idx = -1;
@@ -509,8 +514,8 @@ extern "C" int ngc_sample_evict(const float* logits, const int32_t* n, const int
     sample_tiny_kernel<<<(grid + kTinyWarps - 1) / kTinyWarps, kTinyWarps * 32, 0, (cudaStream_t)stream>>>(p, (int)grid);
   } else if (n_max <= kSampleSmemMaxUnits) {
     const size_t n_al = (size_t)((n_max + 7) & ~7);
-    const size_t n_slots = (size_t)(p.pad_max > threads ? p.pad_max : threads);
-    const size_t smem = n_al * 4 + 2 * n_slots * 2 + (size_t)34 * threads * 2 + bitmap_bytes;
+    const size_t n_slots = (size_t)(p.pad_max > threads ? p.pad_max : threads) + 64;
+    const size_t smem = n_al * 4 + 2 * n_slots * 2 + (size_t)34 * threads * 2 + bitmap_bytes + n_slots;
     if (smem > 48 * 1024)
       NGC_CUDA_TRY(cudaFuncSetAttribute(sample_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     sample_kernel<true><<<grid, threads, smem, (cudaStream_t)stream>>>(p);
