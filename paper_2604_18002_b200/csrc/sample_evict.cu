@@ -307,7 +307,17 @@ __global__ void sample_kernel(SampleParams p) {
         if (lane == 31) s_warp_tot[warp] = incl;
         __syncthreads();
         int run = incl - sum;
-        for (int w2 = 0; w2 < warp; ++w2) run += s_warp_tot[w2];
+        {
+          // counters in front of this warp's: a scan over the warp totals (one per lane) instead of a serial walk
+          const int wt = lane < n_warps ? s_warp_tot[lane] : 0;
+          int wincl = wt;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, wincl, o);
+            if (lane >= o) wincl += t;
+          }
+          run += __shfl_sync(0xffffffffu, wincl - wt, warp);
+        }
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           const int c0 = (int)(wv[e] & 0xFFFFu), c1 = (int)(wv[e] >> 16);
