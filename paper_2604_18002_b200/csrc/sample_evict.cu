@@ -270,7 +270,7 @@ __global__ void sample_kernel(SampleParams p) {
         const uint32_t bal = __ballot_sync(0xffffffffu, keep);
         if (keep) {
           const int pos = s_cnt[k * 32 + warp] + __popc(bal & ((1u << lane) - 1u));
-          src[slot((uint32_t)pos)] = (uint16_t)i;
+          if (NGC_IN_BOUNDS(p.dev_status, pos >= 0 && pos < n_sort)) src[slot((uint32_t)pos)] = (uint16_t)i;
         }
       }
       __syncthreads();                   // s_cnt is read before the counters are cleared
@@ -331,7 +331,7 @@ __global__ void sample_kernel(SampleParams p) {
         const uint32_t d = dig[k * nthr + tid];
         const uint32_t x = d * nthr + tid;
         const uint32_t pos = hist[x + 2 * (x >> 5)]++;
-        dst[slot(pos)] = cand;
+        if (NGC_IN_BOUNDS(p.dev_status, pos < (uint32_t)n_sort)) dst[slot(pos)] = cand;
       }
       __syncthreads();
       uint16_t* t = src; src = dst; dst = t;

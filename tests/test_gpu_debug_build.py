@@ -33,6 +33,8 @@ bf16, f32 = torch.bfloat16, torch.float32
 CASES = [
     (t_par.test_sample_bit_exact, (3, 2, 100, 1.0)),
     (t_par.test_sample_bit_exact, (2, 3, 4096, 1.4142)),
+    (t_par.test_sample_bit_exact, (2, 2, 16384, 1.0)),
+    (t_par.test_sample_long_lists_with_ties_around_the_selection_threshold, ("quantised",)),
     (t_par.test_sample_edge_cases_and_status, ()),
     (t_par.test_tiny_lists_sample_and_logprob, (19, 28, 22)),
     (t_par.test_logprob_matches_oracle, (4, 2, 3, 768, 1 / 3)),
