@@ -81,6 +81,12 @@ def test_score_backward_tile_edges_and_row_counts(Hq, Hkv, w, lens):
     run_case(1, len(lens), Hq, Hkv, w, lens, 2, 8, 1, seed=5 * Hq + w)
 
 
+def test_score_backward_cache_smaller_than_one_tile():
+    """A whole cache plane shorter than one 128-token tile (the tensor-map boxes reach beyond the tensor)."""
+    run_case(1, 1, 4, 2, 2, [10], 1, 1, 0, seed=2)
+    run_case(2, 2, 12, 2, 5, [1, 7], 2, 4, 1, seed=3)
+
+
 def test_score_backward_many_short_strips_write_grad_q_directly():
     """More strips than the kernels want items: no strip is cut into token ranges and the gradient pass writes
     grad_q itself (no partials, no reduction launch)."""
